@@ -1,0 +1,159 @@
+/*
+ * lookm.h -- C ABI of the B200 (sm_100a) implementation of LOOK-M's one-shot, prefill-time
+ * KV-cache compression (arXiv 2406.18139, Section 3).
+ *
+ * Per layer, per request and per KV head the library
+ *   1. scores every prompt key by the column sum of the prompt's causal softmax attention (Eq. 4),
+ *   2. keeps the recent window and the Top-N of the other tokens with text ranked before image
+ *      tokens (Eq. 5-8),
+ *   3. matches every evicted key to its most cosine-similar kept key (Eq. 9),
+ *   4. folds the evicted K/V rows into their kept rows by averaged, pivotal or weighted merging
+ *      (Eq. 10-12) and writes the kept rows as a dense cache ordered by position (Eq. 6-7).
+ *
+ * Conventions common to every entry point
+ *   - All tensors are DEVICE memory unless the parameter name ends in `_host`.  Q/K/V and the
+ *     output caches are bf16; head_dim must be 128; the feature index is contiguous.
+ *   - Batches are packed along the token axis: request r owns tokens
+ *     [cu_seqlens_host[r], cu_seqlens_host[r+1]).  A single prompt is n_requests = 1.
+ *   - "kept"/"evicted" lists hold positions relative to the request start, ascending.  With
+ *     B_r = min(budget_r, L_r) and E_r = L_r - B_r, the list of (request r, KV head h) starts at
+ *     element  n_kv_heads * sum_{r'<r} B_r' + h * B_r   (kept lists) or
+ *              n_kv_heads * sum_{r'<r} E_r' + h * E_r   (evicted, assign and sim arrays).
+ *   - Every buffer is owned by the caller.  The library allocates nothing, keeps no state between
+ *     calls, never modifies inputs; outputs and workspace must not overlap inputs.  `workspace`
+ *     must be 256-byte aligned and at least lookm_workspace_size() bytes; its first bytes hold
+ *     the device status word.  Calls that share a workspace must not overlap on the GPU.
+ *   - Work is enqueued on `cuda_stream` (a cudaStream_t; NULL = default stream) and the call
+ *     returns without synchronising.  Host outputs (`*_host`) are computed from the arguments and
+ *     are valid on return.
+ *   - Return value: a lookm_status.  Argument errors are found before anything is enqueued.
+ *     Device-side waits are bounded; if one expires the kernel finishes without its results and
+ *     lookm_device_status() reports LOOKM_ERR_DEVICE_TIMEOUT.  Nothing traps.
+ *   - Edge rules: seq_len <= budget copies the prompt unchanged (out_len = seq_len);
+ *     recent_window >= budget keeps only the last `budget` tokens; budget <= 0, seq_len <= 0 or
+ *     recent_window < 0 is LOOKM_ERR_INVALID_ARG.
+ */
+#ifndef LOOKM_H_
+#define LOOKM_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    LOOKM_OK = 0,
+    LOOKM_ERR_INVALID_ARG = 1,
+    LOOKM_ERR_UNSUPPORTED = 2,        /* e.g. head_dim != 128, or a device that is not sm_100 */
+    LOOKM_ERR_WORKSPACE_TOO_SMALL = 3,
+    LOOKM_ERR_CUDA = 4,               /* a CUDA runtime/driver call failed */
+    LOOKM_ERR_DEVICE_TIMEOUT = 5,     /* a bounded device-side wait expired */
+    LOOKM_ERR_DEVICE_BAD_INDEX = 6    /* a caller-supplied index list held an out-of-range entry */
+} lookm_status;
+
+typedef enum {
+    LOOKM_MERGE_AVERAGE = 0,          /* Eq. 10 */
+    LOOKM_MERGE_PIVOTAL = 1,          /* Eq. 11 */
+    LOOKM_MERGE_WEIGHTED = 2          /* Eq. 12 */
+} lookm_merge_mode;
+
+/* Shapes and strides (in elements) of Q [tokens, n_q_heads, head_dim] and of K and V
+ * [tokens, n_kv_heads, head_dim] (K and V share strides).  Strides must be multiples of 8
+ * elements and the base pointers 16-byte aligned (TMA requirements).  n_q_heads must be a
+ * multiple of n_kv_heads; query heads [h*g, (h+1)*g) share KV head h and their scores are
+ * summed.  softmax_scale = 0 selects 1/sqrt(head_dim); it must not be negative. */
+typedef struct {
+    int n_q_heads, n_kv_heads, head_dim;
+    long long q_stride_tok, q_stride_head;
+    long long kv_stride_tok, kv_stride_head;
+    float softmax_scale;
+} lookm_layout;
+
+/* Bytes of workspace that any entry point below needs for this batch (host arrays of
+ * n_requests entries).  Returns 0 on invalid arguments. */
+size_t lookm_workspace_size(const lookm_layout* layout, int n_requests, const int* seq_lens_host,
+                            const int* budgets_host);
+
+/* The whole path for one prompt (Section 3.2-3.3, Eq. 4-12).
+ *   q, k, v        [seq_len, heads, 128] bf16 with the strides of `layout`
+ *   modality_mask  [seq_len] bytes, 1 = image token, 0 = text token
+ *   out_k, out_v   [n_kv_heads, out_len, 128] bf16, contiguous; row order = ascending position,
+ *                  the Top-N tokens first, then the recent window (Eq. 6-7)
+ *   out_len_host   receives min(seq_len, budget) */
+int lookm_compress_layer(const void* q, const void* k, const void* v, const uint8_t* modality_mask,
+                         int seq_len, int budget, int recent_window, int merge_mode,
+                         const lookm_layout* layout, void* out_k, void* out_v, int* out_len_host,
+                         void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* The whole path for a packed ragged batch; each request has its own budget, window and merge
+ * mode (host arrays of n_requests entries).
+ *   out_k, out_v          [sum_r out_len_r, n_kv_heads, 128] bf16, requests in order
+ *   out_cu_seqlens_host   [n_requests + 1] prefix sums of out_len_r */
+int lookm_compress_varlen(const void* q, const void* k, const void* v, const uint8_t* modality_mask,
+                          const int* cu_seqlens_host, int n_requests, const int* budgets_host,
+                          const int* windows_host, const int* merge_modes_host,
+                          const lookm_layout* layout, void* out_k, void* out_v,
+                          int* out_cu_seqlens_host, void* workspace, size_t workspace_bytes,
+                          void* cuda_stream);
+
+/* Step 1 alone (Eq. 4): scores[h, t] = sum over the query heads of KV head h and over the rows
+ * i >= t of the same request of softmax_row_i(q_i . k * scale)[t].
+ *   scores  [n_kv_heads, total_tokens] fp32
+ *   lse     [n_q_heads, total_tokens] fp32, natural-log row log-sum-exp.  If lse_is_input != 0
+ *           it is read (e.g. produced by the caller's prefill attention) and the first sweep is
+ *           skipped; otherwise it is written.  May be NULL when lse_is_input == 0 (the workspace
+ *           then holds it). */
+int lookm_score(const void* q, const void* k, const int* cu_seqlens_host, int n_requests,
+                const lookm_layout* layout, float* scores, float* lse, int lse_is_input,
+                void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* The selection alone (Eq. 5-8), fed with given scores [n_kv_heads, total_tokens] (fp32; the
+ * method's scores are positive, other finite values are ordered numerically).
+ *   kept_idx    kept positions, ascending (layout above)
+ *   evict_idx   evicted positions, ascending
+ *   rank        [n_kv_heads, total_tokens]: evicted token -> its index in the evicted list,
+ *               kept token -> -1 - slot.  May be NULL. */
+int lookm_select(const float* scores, const uint8_t* modality_mask, const int* cu_seqlens_host,
+                 int n_requests, const int* budgets_host, const int* windows_host, int n_kv_heads,
+                 int* kept_idx, int* evict_idx, int* rank, void* workspace, size_t workspace_bytes,
+                 void* cuda_stream);
+
+/* The matching alone (Eq. 9): for every evicted key the kept slot of largest cosine similarity
+ * on the original keys (lowest slot on ties) and that similarity. */
+int lookm_match(const void* k, const int* kept_idx, const int* evict_idx, const int* cu_seqlens_host,
+                int n_requests, const int* budgets_host, const lookm_layout* layout, int* assign,
+                float* sim, void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* The decision part of the matching alone: row argmax (lowest slot on ties) of given similarity
+ * matrices.  sim_matrix holds, per (request, head) in the order of the evicted lists, a dense
+ * row-major [E_r, B_r] fp32 block (block of (r, h) starts at element
+ * n_kv_heads * sum_{r'<r} E_r' B_r' + h * E_r * B_r). */
+int lookm_match_from_sim(const float* sim_matrix, const int* cu_seqlens_host, int n_requests,
+                         const int* budgets_host, int n_kv_heads, int* assign, float* sim,
+                         void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* The merging alone (Eq. 10-12 and the compaction of Eq. 6-7), fed with given lists.
+ * varlen_output = 0: out [n_kv_heads, out_len, 128] (requires n_requests == 1);
+ * varlen_output = 1: out [sum_r out_len_r, n_kv_heads, 128]. */
+int lookm_merge(const void* k, const void* v, const int* kept_idx, const int* evict_idx,
+                const int* assign, const float* sim, const int* cu_seqlens_host, int n_requests,
+                const int* budgets_host, const int* merge_modes_host, const lookm_layout* layout,
+                int varlen_output, void* out_k, void* out_v, void* workspace,
+                size_t workspace_bytes, void* cuda_stream);
+
+/* Synchronises `cuda_stream`, then returns and clears the device status word kept at the start
+ * of `workspace` (LOOKM_OK if no kernel reported a problem since the last call that used this
+ * workspace began). */
+int lookm_device_status(void* workspace, void* cuda_stream);
+
+/* Number of kernels the last call on this host thread enqueued (for launch accounting). */
+int lookm_last_launch_count(void);
+
+const char* lookm_strerror(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LOOKM_H_ */

@@ -1,0 +1,83 @@
+// Internal declarations shared by the host planner (api.cu) and the kernel files.
+#pragma once
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "../../include/lookm.h"
+
+namespace lookm {
+
+constexpr int kTile = 128;      // tokens per tile on either operand of the tensor-core kernels
+constexpr int kHeadDim = 128;   // only supported head_dim
+
+// One request of the packed batch as the kernels see it (device copy lives in the workspace).
+// Requests are stored longest first so that the heaviest work items are issued first.
+struct Req {
+    int tok_begin;        // first token of the request on the packed token axis
+    int L;                // prompt length
+    int B;                // kept rows  = min(budget, L)
+    int M;                // recent window, clamped to B
+    int E;                // evicted rows = L - B
+    int mode;             // lookm_merge_mode
+    int nblk;             // ceil(L / kTile)
+    int out_begin;        // sum of B over the requests before this one (caller order)
+    long long kept_off;   // n_kv_heads * out_begin          (start of this request's kept lists)
+    long long ev_off;     // n_kv_heads * sum of E before    (start of this request's evicted lists)
+    long long sim_off;    // n_kv_heads * sum of E*B before  (start of its similarity blocks)
+    int item_begin[3];    // first work item of this request in sweep 1 / sweep 2 / match order
+    int slot_begin;       // first (head, slot) row of this request in merge order (table order)
+};
+
+enum TileKind { kSweep1 = 0, kSweep2 = 1, kMatch = 2 };
+
+struct TileParams {
+    const Req* reqs;
+    int n_req;
+    int n_items;
+    int n_q_heads, n_kv_heads, group;
+    long long T;                 // total packed tokens
+    float scale_log2;            // softmax scale * log2(e)
+    float* lse;                  // [n_q_heads, T] natural log (sweep 1 writes, sweep 2 reads)
+    float* scores;               // [n_kv_heads, T]
+    const int* rank;             // [n_kv_heads, T]      (match)
+    const float* rnorm_all;      // [n_kv_heads, T]      (match)
+    const float* rnorm_kept;     // kept-list layout     (match)
+    int* assign;                 // evicted-list layout  (match)
+    float* sim;                  // evicted-list layout  (match)
+    int* status;                 // device status word
+};
+
+// ---- launchers (each enqueues on `stream` and returns the CUDA error of the launch) -----------
+cudaError_t launch_tile_kernel(int kind, const CUtensorMap& map_a, const CUtensorMap& map_b,
+                               const TileParams& p, int num_sms, cudaStream_t stream);
+
+cudaError_t launch_select(const float* scores, const uint8_t* mask, const Req* reqs, int n_req,
+                          int n_kv_heads, long long T, int* kept_idx, int* evict_idx, int* rank,
+                          cudaStream_t stream);
+
+cudaError_t launch_key_norms(const void* k, long long stride_tok, long long stride_head,
+                             int n_kv_heads, long long T, float* rnorm_all, cudaStream_t stream);
+
+cudaError_t launch_gather_kept(const void* k, long long stride_tok, long long stride_head,
+                               const Req* reqs, int n_req, int n_kv_heads, long long T,
+                               long long total_kept_rows, const int* kept_idx,
+                               const float* rnorm_all, void* kept_keys, float* rnorm_kept,
+                               int* status, cudaStream_t stream);
+
+cudaError_t launch_argmax_rows(const float* sim_matrix, const Req* reqs, int n_req, int n_kv_heads,
+                               int* assign, float* sim, cudaStream_t stream);
+
+cudaError_t launch_invert_assignment(const int* assign, const Req* reqs, int n_req, int n_kv_heads,
+                                     int* row_ptr, int* members, unsigned* sort_a, unsigned* sort_b,
+                                     int* status, cudaStream_t stream);
+
+cudaError_t launch_merge(const void* k, const void* v, long long stride_tok, long long stride_head,
+                         const Req* reqs, int n_req, int n_kv_heads, long long T,
+                         long long total_kept_rows, const int* kept_idx, const int* evict_idx,
+                         const float* sim, const int* row_ptr, const int* members,
+                         int varlen_output, void* out_k, void* out_v, int* status,
+                         cudaStream_t stream);
+
+}  // namespace lookm
