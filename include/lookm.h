@@ -71,8 +71,9 @@ typedef struct {
     float softmax_scale;
 } lookm_layout;
 
-/* Bytes of workspace that any entry point below needs for this batch (host arrays of
- * n_requests entries).  Returns 0 on invalid arguments. */
+/* Bytes of workspace that any entry point below needs for this batch (seq_lens_host: n_requests
+ * entries).  The size covers every budget, so budgets_host is only validated and may be NULL.
+ * Returns 0 on invalid arguments. */
 size_t lookm_workspace_size(const lookm_layout* layout, int n_requests, const int* seq_lens_host,
                             const int* budgets_host);
 

@@ -1,0 +1,182 @@
+"""Thin ctypes binding of liblookm.so: same names as the C ABI, argument marshalling only.
+
+Device buffers are torch CUDA tensors (PyTorch is used for device memory and streams, nothing
+else); host arrays are Python sequences of ints.  Every function returns the library's status
+code unless stated otherwise and raises nothing for device-side results; :func:`check` turns a
+non-zero status into an exception.  Loading fails loudly if the library has not been built:
+there is no fallback path.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional, Sequence
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "liblookm.so")
+_lib = None
+
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE_TOO_SMALL, ERR_CUDA, ERR_DEVICE_TIMEOUT, \
+    ERR_DEVICE_BAD_INDEX = range(7)
+MERGE_AVERAGE, MERGE_PIVOTAL, MERGE_WEIGHTED = 0, 1, 2
+
+EXPORTS = ["lookm_workspace_size", "lookm_compress_layer", "lookm_compress_varlen", "lookm_score",
+           "lookm_select", "lookm_match", "lookm_match_from_sim", "lookm_merge",
+           "lookm_device_status", "lookm_last_launch_count", "lookm_strerror"]
+
+
+class Layout(C.Structure):
+    _fields_ = [("n_q_heads", C.c_int), ("n_kv_heads", C.c_int), ("head_dim", C.c_int),
+                ("q_stride_tok", C.c_longlong), ("q_stride_head", C.c_longlong),
+                ("kv_stride_tok", C.c_longlong), ("kv_stride_head", C.c_longlong),
+                ("softmax_scale", C.c_float)]
+
+
+def lib():
+    """The loaded library; raises if liblookm.so is missing (build it with build.py)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError("liblookm.so is not built: run `python -m paper_2406_18139_b200.build` "
+                               "(there is no CPU or eager fallback)")
+        L = C.CDLL(LIB_PATH)
+        vp, ip, sz = C.c_void_p, C.POINTER(C.c_int), C.c_size_t
+        lp = C.POINTER(Layout)
+        L.lookm_workspace_size.argtypes = [lp, C.c_int, ip, ip]
+        L.lookm_workspace_size.restype = sz
+        L.lookm_compress_layer.argtypes = [vp, vp, vp, vp, C.c_int, C.c_int, C.c_int, C.c_int, lp,
+                                           vp, vp, ip, vp, sz, vp]
+        L.lookm_compress_varlen.argtypes = [vp, vp, vp, vp, ip, C.c_int, ip, ip, ip, lp, vp, vp, ip,
+                                            vp, sz, vp]
+        L.lookm_score.argtypes = [vp, vp, ip, C.c_int, lp, vp, vp, C.c_int, vp, sz, vp]
+        L.lookm_select.argtypes = [vp, vp, ip, C.c_int, ip, ip, C.c_int, vp, vp, vp, vp, sz, vp]
+        L.lookm_match.argtypes = [vp, vp, vp, ip, C.c_int, ip, lp, vp, vp, vp, sz, vp]
+        L.lookm_match_from_sim.argtypes = [vp, ip, C.c_int, ip, C.c_int, vp, vp, vp, sz, vp]
+        L.lookm_merge.argtypes = [vp, vp, vp, vp, vp, vp, ip, C.c_int, ip, ip, lp, C.c_int, vp, vp,
+                                  vp, sz, vp]
+        L.lookm_device_status.argtypes = [vp, vp]
+        L.lookm_last_launch_count.argtypes = []
+        L.lookm_strerror.argtypes = [C.c_int]
+        L.lookm_strerror.restype = C.c_char_p
+        for name in ("lookm_compress_layer", "lookm_compress_varlen", "lookm_score", "lookm_select",
+                     "lookm_match", "lookm_match_from_sim", "lookm_merge", "lookm_device_status",
+                     "lookm_last_launch_count"):
+            getattr(L, name).restype = C.c_int
+        _lib = L
+    return _lib
+
+
+def _ints(seq: Optional[Sequence[int]]):
+    if seq is None:
+        return None
+    seq = [int(x) for x in seq]
+    return (C.c_int * len(seq))(*seq)
+
+
+def _ptr(t):
+    return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def _stream(stream) -> C.c_void_p:
+    if stream is None:
+        import torch
+        stream = torch.cuda.current_stream()
+    return C.c_void_p(stream.cuda_stream)
+
+
+def lookm_strerror(status: int) -> str:
+    return lib().lookm_strerror(int(status)).decode()
+
+
+def check(status: int) -> None:
+    if status != OK:
+        raise RuntimeError("lookm: %s (status %d)" % (lookm_strerror(status), status))
+
+
+def make_layout(q, k, softmax_scale: float = 0.0) -> Layout:
+    """Layout of Q [T, Hq, 128] and K/V [T, Hkv, 128] tensors (any strides, last dim contiguous)."""
+    assert k.stride(2) == 1 and (q is None or q.stride(2) == 1)
+    qq = q if q is not None else k
+    return Layout(qq.shape[1], k.shape[1], k.shape[2], qq.stride(0), qq.stride(1), k.stride(0),
+                  k.stride(1), float(softmax_scale))
+
+
+def lookm_workspace_size(layout: Layout, seq_lens: Sequence[int], budgets: Optional[Sequence[int]] = None) -> int:
+    return int(lib().lookm_workspace_size(C.byref(layout), len(seq_lens), _ints(seq_lens), _ints(budgets)))
+
+
+def lookm_compress_layer(q, k, v, modality_mask, seq_len, budget, recent_window, merge_mode, layout,
+                         out_k, out_v, workspace, stream=None):
+    """Returns (status, out_len)."""
+    out_len = C.c_int(0)
+    st = lib().lookm_compress_layer(_ptr(q), _ptr(k), _ptr(v), _ptr(modality_mask), int(seq_len),
+                                    int(budget), int(recent_window), int(merge_mode), C.byref(layout),
+                                    _ptr(out_k), _ptr(out_v), C.byref(out_len), _ptr(workspace),
+                                    workspace.numel() * workspace.element_size(), _stream(stream))
+    return st, out_len.value
+
+
+def lookm_compress_varlen(q, k, v, modality_mask, cu_seqlens, budgets, windows, merge_modes, layout,
+                          out_k, out_v, workspace, stream=None):
+    """Returns (status, out_cu_seqlens list)."""
+    n = len(cu_seqlens) - 1
+    out_cu = (C.c_int * (n + 1))()
+    st = lib().lookm_compress_varlen(_ptr(q), _ptr(k), _ptr(v), _ptr(modality_mask), _ints(cu_seqlens),
+                                     n, _ints(budgets), _ints(windows), _ints(merge_modes),
+                                     C.byref(layout), _ptr(out_k), _ptr(out_v), out_cu, _ptr(workspace),
+                                     workspace.numel() * workspace.element_size(), _stream(stream))
+    return st, list(out_cu)
+
+
+def lookm_score(q, k, cu_seqlens, layout, scores, lse, lse_is_input, workspace, stream=None):
+    return lib().lookm_score(_ptr(q), _ptr(k), _ints(cu_seqlens), len(cu_seqlens) - 1, C.byref(layout),
+                             _ptr(scores), _ptr(lse), int(bool(lse_is_input)), _ptr(workspace),
+                             workspace.numel() * workspace.element_size(), _stream(stream))
+
+
+def lookm_select(scores, modality_mask, cu_seqlens, budgets, windows, n_kv_heads, kept_idx, evict_idx,
+                 rank, workspace, stream=None):
+    return lib().lookm_select(_ptr(scores), _ptr(modality_mask), _ints(cu_seqlens), len(cu_seqlens) - 1,
+                              _ints(budgets), _ints(windows), int(n_kv_heads), _ptr(kept_idx),
+                              _ptr(evict_idx), _ptr(rank), _ptr(workspace),
+                              workspace.numel() * workspace.element_size(), _stream(stream))
+
+
+def lookm_match(k, kept_idx, evict_idx, cu_seqlens, budgets, layout, assign, sim, workspace, stream=None):
+    return lib().lookm_match(_ptr(k), _ptr(kept_idx), _ptr(evict_idx), _ints(cu_seqlens),
+                             len(cu_seqlens) - 1, _ints(budgets), C.byref(layout), _ptr(assign),
+                             _ptr(sim), _ptr(workspace), workspace.numel() * workspace.element_size(),
+                             _stream(stream))
+
+
+def lookm_match_from_sim(sim_matrix, cu_seqlens, budgets, n_kv_heads, assign, sim, workspace, stream=None):
+    return lib().lookm_match_from_sim(_ptr(sim_matrix), _ints(cu_seqlens), len(cu_seqlens) - 1,
+                                      _ints(budgets), int(n_kv_heads), _ptr(assign), _ptr(sim),
+                                      _ptr(workspace), workspace.numel() * workspace.element_size(),
+                                      _stream(stream))
+
+
+def lookm_merge(k, v, kept_idx, evict_idx, assign, sim, cu_seqlens, budgets, merge_modes, layout,
+                varlen_output, out_k, out_v, workspace, stream=None):
+    return lib().lookm_merge(_ptr(k), _ptr(v), _ptr(kept_idx), _ptr(evict_idx), _ptr(assign), _ptr(sim),
+                             _ints(cu_seqlens), len(cu_seqlens) - 1, _ints(budgets), _ints(merge_modes),
+                             C.byref(layout), int(bool(varlen_output)), _ptr(out_k), _ptr(out_v),
+                             _ptr(workspace), workspace.numel() * workspace.element_size(),
+                             _stream(stream))
+
+
+def lookm_device_status(workspace, stream=None) -> int:
+    return lib().lookm_device_status(_ptr(workspace), _stream(stream))
+
+
+def lookm_last_launch_count() -> int:
+    return lib().lookm_last_launch_count()
+
+
+def alloc_workspace(layout: Layout, seq_lens: Sequence[int], device="cuda"):
+    """A torch uint8 buffer of lookm_workspace_size bytes (torch allocations are 256-byte aligned)."""
+    import torch
+    n = lookm_workspace_size(layout, seq_lens)
+    if n == 0:
+        raise ValueError("lookm_workspace_size rejected the layout")
+    return torch.empty(n, dtype=torch.uint8, device=device)

@@ -1,0 +1,519 @@
+// Host side of the C ABI: argument checks, workspace carving, the request table, TMA tensor maps
+// and the launch sequence.  Nothing here synchronises with the device or allocates device memory.
+#include <algorithm>
+#include <cmath>
+#include <cstring>
+#include <mutex>
+#include <vector>
+
+#include <cudaTypedefs.h>
+
+#include "internal.h"
+
+namespace lookm {
+namespace {
+
+thread_local int g_launches = 0;
+
+size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+struct Plan {
+    int n_req = 0, n_q_heads = 0, n_kv_heads = 0, group = 1;
+    long long T = 0, sum_B = 0, sum_E = 0, sum_EB = 0;
+    int max_L = 0, max_E = 0;
+    int n_items[3] = {0, 0, 0};
+    long long total_slots = 0;              // n_kv_heads * sum_B
+    std::vector<Req> reqs;                  // table order (longest first)
+    std::vector<int> out_len;               // caller order
+    // workspace offsets (bytes)
+    size_t o_status, o_reqs, o_lse, o_scores, o_rank, o_rnorm_all, o_kept, o_evict, o_kept_keys,
+        o_rnorm_kept, o_assign, o_sim, o_row_ptr, o_members, o_sort_a, o_sort_b, total;
+};
+
+// Returns LOOKM_OK or the status describing the first bad argument.
+int build_plan(Plan& pl, const lookm_layout* lay, int n_req, const int* cu_seqlens,
+               const int* seq_lens, const int* budgets, const int* windows, const int* modes) {
+    if (!lay || n_req <= 0 || (!cu_seqlens && !seq_lens)) return LOOKM_ERR_INVALID_ARG;
+    if (lay->head_dim != kHeadDim) return LOOKM_ERR_UNSUPPORTED;
+    if (lay->n_kv_heads <= 0 || lay->n_q_heads <= 0 || lay->n_q_heads % lay->n_kv_heads)
+        return LOOKM_ERR_INVALID_ARG;
+    if (lay->n_kv_heads > 65535 || n_req > 65535) return LOOKM_ERR_UNSUPPORTED;
+    pl.n_req = n_req;
+    pl.n_q_heads = lay->n_q_heads;
+    pl.n_kv_heads = lay->n_kv_heads;
+    pl.group = lay->n_q_heads / lay->n_kv_heads;
+    pl.reqs.resize(n_req);
+    pl.out_len.resize(n_req);
+    long long tok = 0, out = 0, ev = 0, eb = 0;
+    for (int r = 0; r < n_req; ++r) {
+        const long long begin = cu_seqlens ? cu_seqlens[r] : tok;
+        const long long L = cu_seqlens ? (long long)cu_seqlens[r + 1] - cu_seqlens[r] : seq_lens[r];
+        if (begin != tok || L <= 0 || L > (1 << 30)) return LOOKM_ERR_INVALID_ARG;
+        const int budget = budgets ? budgets[r] : (int)L;
+        const int window = windows ? windows[r] : 0;
+        const int mode = modes ? modes[r] : 0;
+        if (budget <= 0 || window < 0 || mode < 0 || mode > 2) return LOOKM_ERR_INVALID_ARG;
+        Req& q = pl.reqs[r];
+        q.tok_begin = (int)begin;
+        q.L = (int)L;
+        q.B = (int)std::min<long long>(budget, L);
+        q.M = std::min(window, q.B);
+        q.E = q.L - q.B;
+        q.mode = mode;
+        q.nblk = (q.L + kTile - 1) / kTile;
+        q.out_begin = (int)out;
+        q.kept_off = (long long)pl.n_kv_heads * out;
+        q.ev_off = (long long)pl.n_kv_heads * ev;
+        q.sim_off = (long long)pl.n_kv_heads * eb;
+        q.rp_off = q.kept_off + (long long)pl.n_kv_heads * r;
+        pl.out_len[r] = q.B;
+        tok += L;
+        out += q.B;
+        ev += q.E;
+        eb += (long long)q.E * q.B;
+        pl.max_L = std::max(pl.max_L, q.L);
+        pl.max_E = std::max(pl.max_E, q.E);
+    }
+    pl.T = tok;
+    pl.sum_B = out;
+    pl.sum_E = ev;
+    pl.sum_EB = eb;
+    pl.total_slots = (long long)pl.n_kv_heads * out;
+    if (pl.T + kTile >= (1ll << 31) || pl.total_slots + kTile >= (1ll << 31) ||
+        (long long)pl.n_q_heads * ((pl.T + kTile - 1) / kTile + n_req) >= (1ll << 31))
+        return LOOKM_ERR_UNSUPPORTED;
+    // table order: longest request first
+    std::stable_sort(pl.reqs.begin(), pl.reqs.end(), [](const Req& a, const Req& b) { return a.L > b.L; });
+    long long it0 = 0, it1 = 0, it2 = 0, slots = 0;
+    for (Req& q : pl.reqs) {
+        q.item_begin[kSweep1] = (int)it0;
+        q.item_begin[kSweep2] = (int)it1;
+        q.item_begin[kMatch] = (int)it2;
+        q.slot_begin = (int)slots;
+        it0 += (long long)q.nblk * pl.n_q_heads;
+        it1 += (long long)q.nblk * pl.n_kv_heads;
+        it2 += q.E > 0 ? (long long)q.nblk * pl.n_kv_heads : 0;
+        slots += (long long)q.B * pl.n_kv_heads;
+    }
+    pl.n_items[kSweep1] = (int)it0;
+    pl.n_items[kSweep2] = (int)it1;
+    pl.n_items[kMatch] = (int)it2;
+
+    size_t o = 0;
+    auto carve = [&](size_t bytes) { size_t at = o; o = align_up(o + bytes, 256); return at; };
+    const size_t Hq = pl.n_q_heads, Hkv = pl.n_kv_heads, T = (size_t)pl.T;
+    // Every list is sized for the worst case over budgets (at most T kept and T evicted rows per
+    // head), so the carving depends only on the prompt lengths and head counts.
+    pl.o_status = carve(256);
+    pl.o_reqs = carve(sizeof(Req) * n_req);
+    pl.o_lse = carve(4 * Hq * T);
+    pl.o_scores = carve(4 * Hkv * T);
+    pl.o_rank = carve(4 * Hkv * T);
+    pl.o_rnorm_all = carve(4 * Hkv * T);
+    pl.o_kept = carve(4 * Hkv * T);
+    pl.o_evict = carve(4 * Hkv * T);
+    pl.o_kept_keys = carve(2 * (size_t)kHeadDim * Hkv * T);
+    pl.o_rnorm_kept = carve(4 * Hkv * T);
+    pl.o_assign = carve(4 * Hkv * T);
+    pl.o_sim = carve(4 * Hkv * T);
+    pl.o_row_ptr = carve(4 * (Hkv * T + Hkv * (size_t)n_req));
+    pl.o_members = carve(4 * Hkv * T);
+    pl.o_sort_a = carve(8 * Hkv * T);
+    pl.o_sort_b = carve(8 * Hkv * T);
+    pl.total = o;
+    return LOOKM_OK;
+}
+
+int check_layout_ptrs(const lookm_layout* lay, const void* q, const void* k, const void* v) {
+    auto bad_ptr = [](const void* p) { return p && (reinterpret_cast<uintptr_t>(p) & 15u); };
+    if (bad_ptr(q) || bad_ptr(k) || bad_ptr(v)) return LOOKM_ERR_INVALID_ARG;
+    if (lay->q_stride_tok % 8 || lay->q_stride_head % 8 || lay->kv_stride_tok % 8 ||
+        lay->kv_stride_head % 8)
+        return LOOKM_ERR_INVALID_ARG;
+    if (lay->q_stride_tok <= 0 || lay->q_stride_head <= 0 || lay->kv_stride_tok <= 0 ||
+        lay->kv_stride_head <= 0)
+        return LOOKM_ERR_INVALID_ARG;
+    if (!(lay->softmax_scale >= 0.f) || !std::isfinite(lay->softmax_scale)) return LOOKM_ERR_INVALID_ARG;
+    return LOOKM_OK;
+}
+
+int check_workspace(const Plan& pl, void* ws, size_t bytes) {
+    if (!ws || (reinterpret_cast<uintptr_t>(ws) & 255u)) return LOOKM_ERR_INVALID_ARG;
+    if (bytes < pl.total) return LOOKM_ERR_WORKSPACE_TOO_SMALL;
+    return LOOKM_OK;
+}
+
+// ---- device facts and the tensor-map encoder ---------------------------------------------------
+struct DeviceInfo { int sms = 0; int cc_major = 0; bool ok = false; };
+
+int device_info(DeviceInfo& out) {
+    static std::mutex mu;
+    static DeviceInfo cache[64];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return LOOKM_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(mu);
+    if (!cache[dev].ok) {
+        if (cudaDeviceGetAttribute(&cache[dev].sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&cache[dev].cc_major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess)
+            return LOOKM_ERR_CUDA;
+        cache[dev].ok = true;
+    }
+    out = cache[dev];
+    return out.cc_major == 10 ? LOOKM_OK : LOOKM_ERR_UNSUPPORTED;
+}
+
+PFN_cuTensorMapEncodeTiled_v12000 tensor_map_encoder() {
+    static PFN_cuTensorMapEncodeTiled_v12000 fn = [] {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) != cudaSuccess ||
+            qres != cudaDriverEntryPointSuccess)
+            p = nullptr;
+        return reinterpret_cast<PFN_cuTensorMapEncodeTiled_v12000>(p);
+    }();
+    return fn;
+}
+
+// bf16 tensor [tokens, heads, 128] with element strides; box = 128 tokens x 1 head x 64 features
+// (128 bytes) with the 128-byte swizzle; out-of-range rows read as zero.
+int make_map_3d(CUtensorMap* map, const void* base, long long tokens, int heads,
+                long long stride_tok, long long stride_head) {
+    auto enc = tensor_map_encoder();
+    if (!enc) return LOOKM_ERR_CUDA;
+    cuuint64_t dims[3] = {(cuuint64_t)kHeadDim, (cuuint64_t)heads, (cuuint64_t)tokens};
+    cuuint64_t strides[2] = {(cuuint64_t)stride_head * 2, (cuuint64_t)stride_tok * 2};
+    cuuint32_t box[3] = {64, 1, (cuuint32_t)kTile};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides,
+                     box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                     CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? LOOKM_OK : LOOKM_ERR_CUDA;
+}
+
+int make_map_2d(CUtensorMap* map, const void* base, long long rows) {
+    auto enc = tensor_map_encoder();
+    if (!enc) return LOOKM_ERR_CUDA;
+    cuuint64_t dims[2] = {(cuuint64_t)kHeadDim, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)kHeadDim * 2};
+    cuuint32_t box[2] = {64, (cuuint32_t)kTile};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides,
+                     box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                     CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? LOOKM_OK : LOOKM_ERR_CUDA;
+}
+
+#define LOOKM_CUDA(expr)                                  \
+    do {                                                  \
+        if ((expr) != cudaSuccess) return LOOKM_ERR_CUDA; \
+    } while (0)
+#define LOOKM_TRY(expr)                   \
+    do {                                  \
+        int st_ = (expr);                 \
+        if (st_ != LOOKM_OK) return st_;  \
+    } while (0)
+
+template <class T>
+T* at(void* ws, size_t off) { return reinterpret_cast<T*>(static_cast<char*>(ws) + off); }
+
+// Clears the status word and writes the request table into the workspace.
+int begin_call(const Plan& pl, void* ws, cudaStream_t st) {
+    g_launches = 0;
+    LOOKM_CUDA(cudaMemsetAsync(at<int>(ws, pl.o_status), 0, 256, st));
+    for (int base = 0; base < pl.n_req; base += kReqChunk) {
+        ReqChunk chunk;
+        const int cnt = std::min(kReqChunk, pl.n_req - base);
+        std::memset(&chunk, 0, sizeof(chunk));
+        std::memcpy(chunk.r, pl.reqs.data() + base, sizeof(Req) * cnt);
+        LOOKM_CUDA(launch_write_table(chunk, cnt, at<Req>(ws, pl.o_reqs) + base, st));
+        ++g_launches;
+    }
+    return LOOKM_OK;
+}
+
+float scale_log2(const lookm_layout* lay) {
+    const float s = lay->softmax_scale > 0.f ? lay->softmax_scale : 1.0f / std::sqrt((float)lay->head_dim);
+    return s * 1.4426950408889634f;
+}
+
+TileParams tile_params(const Plan& pl, void* ws, const lookm_layout* lay) {
+    TileParams p;
+    std::memset(&p, 0, sizeof(p));
+    p.reqs = at<Req>(ws, pl.o_reqs);
+    p.n_req = pl.n_req;
+    p.n_q_heads = pl.n_q_heads;
+    p.n_kv_heads = pl.n_kv_heads;
+    p.group = pl.group;
+    p.T = pl.T;
+    p.scale_log2 = scale_log2(lay);
+    p.status = at<int>(ws, pl.o_status);
+    return p;
+}
+
+int run_score(const Plan& pl, const DeviceInfo& di, const lookm_layout* lay, const void* q,
+              const void* k, float* scores, float* lse, bool lse_is_input, void* ws, cudaStream_t st) {
+    CUtensorMap map_q, map_k;
+    LOOKM_TRY(make_map_3d(&map_q, q, pl.T, pl.n_q_heads, lay->q_stride_tok, lay->q_stride_head));
+    LOOKM_TRY(make_map_3d(&map_k, k, pl.T, pl.n_kv_heads, lay->kv_stride_tok, lay->kv_stride_head));
+    TileParams p = tile_params(pl, ws, lay);
+    p.lse = lse;
+    p.scores = scores;
+    if (!lse_is_input) {
+        p.n_items = pl.n_items[kSweep1];
+        LOOKM_CUDA(launch_tile_kernel(kSweep1, map_q, map_k, p, di.sms, st));
+        ++g_launches;
+    }
+    p.n_items = pl.n_items[kSweep2];
+    LOOKM_CUDA(launch_tile_kernel(kSweep2, map_k, map_q, p, di.sms, st));
+    ++g_launches;
+    return LOOKM_OK;
+}
+
+int run_match(const Plan& pl, const DeviceInfo& di, const lookm_layout* lay, const void* k,
+              const int* kept_idx, const int* rank, int* assign, float* sim, void* ws,
+              cudaStream_t st) {
+    if (pl.n_items[kMatch] == 0) return LOOKM_OK;
+    float* rnorm_all = at<float>(ws, pl.o_rnorm_all);
+    float* rnorm_kept = at<float>(ws, pl.o_rnorm_kept);
+    void* kept_keys = at<void>(ws, pl.o_kept_keys);
+    const Req* reqs = at<Req>(ws, pl.o_reqs);
+    LOOKM_CUDA(launch_key_norms(k, lay->kv_stride_tok, lay->kv_stride_head, pl.n_kv_heads, pl.T,
+                                rnorm_all, st));
+    ++g_launches;
+    LOOKM_CUDA(launch_gather_kept(k, lay->kv_stride_tok, lay->kv_stride_head, reqs, pl.n_req,
+                                  pl.n_kv_heads, pl.T, pl.total_slots, kept_idx, rnorm_all,
+                                  kept_keys, rnorm_kept, at<int>(ws, pl.o_status), st));
+    ++g_launches;
+    CUtensorMap map_k, map_c;
+    LOOKM_TRY(make_map_3d(&map_k, k, pl.T, pl.n_kv_heads, lay->kv_stride_tok, lay->kv_stride_head));
+    LOOKM_TRY(make_map_2d(&map_c, kept_keys, pl.total_slots));
+    TileParams p = tile_params(pl, ws, lay);
+    p.n_items = pl.n_items[kMatch];
+    p.rank = rank;
+    p.rnorm_all = rnorm_all;
+    p.rnorm_kept = rnorm_kept;
+    p.assign = assign;
+    p.sim = sim;
+    LOOKM_CUDA(launch_tile_kernel(kMatch, map_k, map_c, p, di.sms, st));
+    ++g_launches;
+    return LOOKM_OK;
+}
+
+int run_merge(const Plan& pl, const lookm_layout* lay, const void* k, const void* v,
+              const int* kept_idx, const int* evict_idx, const int* assign, const float* sim,
+              int varlen_output, void* out_k, void* out_v, void* ws, cudaStream_t st) {
+    const Req* reqs = at<Req>(ws, pl.o_reqs);
+    int* status = at<int>(ws, pl.o_status);
+    LOOKM_CUDA(launch_invert_assignment(assign, reqs, pl.n_req, pl.n_kv_heads,
+                                        at<int>(ws, pl.o_row_ptr), at<int>(ws, pl.o_members),
+                                        at<unsigned>(ws, pl.o_sort_a), at<unsigned>(ws, pl.o_sort_b),
+                                        status, st));
+    ++g_launches;
+    LOOKM_CUDA(launch_merge(k, v, lay->kv_stride_tok, lay->kv_stride_head, reqs, pl.n_req,
+                            pl.n_kv_heads, pl.T, pl.total_slots, kept_idx, evict_idx, sim,
+                            at<int>(ws, pl.o_row_ptr), at<int>(ws, pl.o_members), varlen_output,
+                            out_k, out_v, status, st));
+    ++g_launches;
+    return LOOKM_OK;
+}
+
+int compress_common(const void* q, const void* k, const void* v, const uint8_t* mask,
+                    const int* cu_seqlens, int n_req, const int* budgets, const int* windows,
+                    const int* modes, const lookm_layout* lay, int varlen_output, void* out_k,
+                    void* out_v, int* out_cu, void* ws, size_t ws_bytes, void* stream) {
+    if (!q || !k || !v || !mask || !out_k || !out_v || !budgets || !windows || !modes)
+        return LOOKM_ERR_INVALID_ARG;
+    Plan pl;
+    LOOKM_TRY(build_plan(pl, lay, n_req, cu_seqlens, nullptr, budgets, windows, modes));
+    LOOKM_TRY(check_layout_ptrs(lay, q, k, v));
+    LOOKM_TRY(check_workspace(pl, ws, ws_bytes));
+    DeviceInfo di;
+    LOOKM_TRY(device_info(di));
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (out_cu) {
+        out_cu[0] = 0;
+        for (int r = 0; r < n_req; ++r) out_cu[r + 1] = out_cu[r] + pl.out_len[r];
+    }
+    LOOKM_TRY(begin_call(pl, ws, st));
+    float* scores = at<float>(ws, pl.o_scores);
+    int* kept = at<int>(ws, pl.o_kept);
+    int* evict = at<int>(ws, pl.o_evict);
+    int* rank = at<int>(ws, pl.o_rank);
+    int* assign = at<int>(ws, pl.o_assign);
+    float* sim = at<float>(ws, pl.o_sim);
+    LOOKM_TRY(run_score(pl, di, lay, q, k, scores, at<float>(ws, pl.o_lse), false, ws, st));
+    LOOKM_CUDA(launch_select(scores, mask, at<Req>(ws, pl.o_reqs), pl.n_req, pl.n_kv_heads, pl.T,
+                             kept, evict, rank, st));
+    ++g_launches;
+    LOOKM_TRY(run_match(pl, di, lay, k, kept, rank, assign, sim, ws, st));
+    LOOKM_TRY(run_merge(pl, lay, k, v, kept, evict, assign, sim, varlen_output, out_k, out_v, ws, st));
+    return LOOKM_OK;
+}
+
+}  // namespace
+}  // namespace lookm
+
+using namespace lookm;
+
+extern "C" {
+
+size_t lookm_workspace_size(const lookm_layout* layout, int n_requests, const int* seq_lens_host,
+                            const int* budgets_host) {
+    Plan pl;
+    if (!seq_lens_host) return 0;
+    if (build_plan(pl, layout, n_requests, nullptr, seq_lens_host, budgets_host, nullptr, nullptr) != LOOKM_OK)
+        return 0;
+    return pl.total;
+}
+
+int lookm_compress_layer(const void* q, const void* k, const void* v, const uint8_t* modality_mask,
+                         int seq_len, int budget, int recent_window, int merge_mode,
+                         const lookm_layout* layout, void* out_k, void* out_v, int* out_len_host,
+                         void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    if (seq_len <= 0) return LOOKM_ERR_INVALID_ARG;
+    const int cu[2] = {0, seq_len};
+    int out_cu[2] = {0, 0};
+    const int st = compress_common(q, k, v, modality_mask, cu, 1, &budget, &recent_window, &merge_mode,
+                                   layout, 0, out_k, out_v, out_cu, workspace, workspace_bytes,
+                                   cuda_stream);
+    if (st == LOOKM_OK && out_len_host) *out_len_host = out_cu[1];
+    return st;
+}
+
+int lookm_compress_varlen(const void* q, const void* k, const void* v, const uint8_t* modality_mask,
+                          const int* cu_seqlens_host, int n_requests, const int* budgets_host,
+                          const int* windows_host, const int* merge_modes_host,
+                          const lookm_layout* layout, void* out_k, void* out_v,
+                          int* out_cu_seqlens_host, void* workspace, size_t workspace_bytes,
+                          void* cuda_stream) {
+    if (!cu_seqlens_host) return LOOKM_ERR_INVALID_ARG;
+    return compress_common(q, k, v, modality_mask, cu_seqlens_host, n_requests, budgets_host,
+                           windows_host, merge_modes_host, layout, 1, out_k, out_v,
+                           out_cu_seqlens_host, workspace, workspace_bytes, cuda_stream);
+}
+
+int lookm_score(const void* q, const void* k, const int* cu_seqlens_host, int n_requests,
+                const lookm_layout* layout, float* scores, float* lse, int lse_is_input,
+                void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    if (!q || !k || !cu_seqlens_host || !scores || (lse_is_input && !lse)) return LOOKM_ERR_INVALID_ARG;
+    Plan pl;
+    LOOKM_TRY(build_plan(pl, layout, n_requests, cu_seqlens_host, nullptr, nullptr, nullptr, nullptr));
+    LOOKM_TRY(check_layout_ptrs(layout, q, k, nullptr));
+    LOOKM_TRY(check_workspace(pl, workspace, workspace_bytes));
+    DeviceInfo di;
+    LOOKM_TRY(device_info(di));
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    LOOKM_TRY(begin_call(pl, workspace, st));
+    float* lse_buf = lse ? lse : at<float>(workspace, pl.o_lse);
+    return run_score(pl, di, layout, q, k, scores, lse_buf, lse_is_input != 0, workspace, st);
+}
+
+int lookm_select(const float* scores, const uint8_t* modality_mask, const int* cu_seqlens_host,
+                 int n_requests, const int* budgets_host, const int* windows_host, int n_kv_heads,
+                 int* kept_idx, int* evict_idx, int* rank, void* workspace, size_t workspace_bytes,
+                 void* cuda_stream) {
+    if (!scores || !modality_mask || !cu_seqlens_host || !budgets_host || !windows_host || !kept_idx ||
+        !evict_idx)
+        return LOOKM_ERR_INVALID_ARG;
+    lookm_layout lay;
+    std::memset(&lay, 0, sizeof(lay));
+    lay.n_q_heads = lay.n_kv_heads = n_kv_heads;
+    lay.head_dim = kHeadDim;
+    Plan pl;
+    LOOKM_TRY(build_plan(pl, &lay, n_requests, cu_seqlens_host, nullptr, budgets_host, windows_host, nullptr));
+    LOOKM_TRY(check_workspace(pl, workspace, workspace_bytes));
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    LOOKM_TRY(begin_call(pl, workspace, st));
+    LOOKM_CUDA(launch_select(scores, modality_mask, at<Req>(workspace, pl.o_reqs), pl.n_req,
+                             pl.n_kv_heads, pl.T, kept_idx, evict_idx, rank, st));
+    ++g_launches;
+    return LOOKM_OK;
+}
+
+int lookm_match(const void* k, const int* kept_idx, const int* evict_idx, const int* cu_seqlens_host,
+                int n_requests, const int* budgets_host, const lookm_layout* layout, int* assign,
+                float* sim, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    if (!k || !kept_idx || !evict_idx || !cu_seqlens_host || !budgets_host || !assign || !sim)
+        return LOOKM_ERR_INVALID_ARG;
+    Plan pl;
+    LOOKM_TRY(build_plan(pl, layout, n_requests, cu_seqlens_host, nullptr, budgets_host, nullptr, nullptr));
+    LOOKM_TRY(check_layout_ptrs(layout, nullptr, k, nullptr));
+    LOOKM_TRY(check_workspace(pl, workspace, workspace_bytes));
+    DeviceInfo di;
+    LOOKM_TRY(device_info(di));
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    LOOKM_TRY(begin_call(pl, workspace, st));
+    int* rank = at<int>(workspace, pl.o_rank);
+    LOOKM_CUDA(cudaMemsetAsync(rank, 0xFF, sizeof(int) * (size_t)pl.n_kv_heads * (size_t)pl.T, st));
+    LOOKM_CUDA(launch_rank_from_lists(at<Req>(workspace, pl.o_reqs), pl.n_req, pl.n_kv_heads, pl.T,
+                                      pl.max_L, kept_idx, evict_idx, rank,
+                                      at<int>(workspace, pl.o_status), st));
+    ++g_launches;
+    return run_match(pl, di, layout, k, kept_idx, rank, assign, sim, workspace, st);
+}
+
+int lookm_match_from_sim(const float* sim_matrix, const int* cu_seqlens_host, int n_requests,
+                         const int* budgets_host, int n_kv_heads, int* assign, float* sim,
+                         void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    if (!sim_matrix || !cu_seqlens_host || !budgets_host || !assign || !sim) return LOOKM_ERR_INVALID_ARG;
+    lookm_layout lay;
+    std::memset(&lay, 0, sizeof(lay));
+    lay.n_q_heads = lay.n_kv_heads = n_kv_heads;
+    lay.head_dim = kHeadDim;
+    Plan pl;
+    LOOKM_TRY(build_plan(pl, &lay, n_requests, cu_seqlens_host, nullptr, budgets_host, nullptr, nullptr));
+    LOOKM_TRY(check_workspace(pl, workspace, workspace_bytes));
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    LOOKM_TRY(begin_call(pl, workspace, st));
+    LOOKM_CUDA(launch_argmax_rows(sim_matrix, at<Req>(workspace, pl.o_reqs), pl.n_req, pl.n_kv_heads,
+                                  pl.max_E, assign, sim, st));
+    ++g_launches;
+    return LOOKM_OK;
+}
+
+int lookm_merge(const void* k, const void* v, const int* kept_idx, const int* evict_idx,
+                const int* assign, const float* sim, const int* cu_seqlens_host, int n_requests,
+                const int* budgets_host, const int* merge_modes_host, const lookm_layout* layout,
+                int varlen_output, void* out_k, void* out_v, void* workspace,
+                size_t workspace_bytes, void* cuda_stream) {
+    if (!k || !v || !kept_idx || !evict_idx || !assign || !sim || !cu_seqlens_host || !budgets_host ||
+        !merge_modes_host || !out_k || !out_v)
+        return LOOKM_ERR_INVALID_ARG;
+    if (!varlen_output && n_requests != 1) return LOOKM_ERR_INVALID_ARG;
+    Plan pl;
+    LOOKM_TRY(build_plan(pl, layout, n_requests, cu_seqlens_host, nullptr, budgets_host, nullptr,
+                         merge_modes_host));
+    LOOKM_TRY(check_layout_ptrs(layout, nullptr, k, v));
+    LOOKM_TRY(check_workspace(pl, workspace, workspace_bytes));
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    LOOKM_TRY(begin_call(pl, workspace, st));
+    return run_merge(pl, layout, k, v, kept_idx, evict_idx, assign, sim, varlen_output, out_k, out_v,
+                     workspace, st);
+}
+
+int lookm_device_status(void* workspace, void* cuda_stream) {
+    if (!workspace) return LOOKM_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    int word = 0;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return LOOKM_ERR_CUDA;
+    if (cudaMemcpy(&word, workspace, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return LOOKM_ERR_CUDA;
+    if (word != 0 && cudaMemset(workspace, 0, sizeof(int)) != cudaSuccess) return LOOKM_ERR_CUDA;
+    return word;
+}
+
+int lookm_last_launch_count(void) { return g_launches; }
+
+const char* lookm_strerror(int status) {
+    switch (status) {
+        case LOOKM_OK: return "ok";
+        case LOOKM_ERR_INVALID_ARG: return "invalid argument";
+        case LOOKM_ERR_UNSUPPORTED: return "unsupported configuration or device";
+        case LOOKM_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
+        case LOOKM_ERR_CUDA: return "a CUDA call failed";
+        case LOOKM_ERR_DEVICE_TIMEOUT: return "a bounded device-side wait expired";
+        case LOOKM_ERR_DEVICE_BAD_INDEX: return "an index list held an out-of-range entry";
+        default: return "unknown status";
+    }
+}
+
+}  // extern "C"

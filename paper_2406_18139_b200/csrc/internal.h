@@ -26,6 +26,8 @@ struct Req {
     long long kept_off;   // n_kv_heads * out_begin          (start of this request's kept lists)
     long long ev_off;     // n_kv_heads * sum of E before    (start of this request's evicted lists)
     long long sim_off;    // n_kv_heads * sum of E*B before  (start of its similarity blocks)
+    long long rp_off;     // kept_off + n_kv_heads * (caller index): start of its row_ptr blocks,
+                          // which hold B + 1 entries per head
     int item_begin[3];    // first work item of this request in sweep 1 / sweep 2 / match order
     int slot_begin;       // first (head, slot) row of this request in merge order (table order)
 };
@@ -67,7 +69,17 @@ cudaError_t launch_gather_kept(const void* k, long long stride_tok, long long st
                                int* status, cudaStream_t stream);
 
 cudaError_t launch_argmax_rows(const float* sim_matrix, const Req* reqs, int n_req, int n_kv_heads,
-                               int* assign, float* sim, cudaStream_t stream);
+                               int max_evicted, int* assign, float* sim, cudaStream_t stream);
+
+cudaError_t launch_rank_from_lists(const Req* reqs, int n_req, int n_kv_heads, long long T,
+                                   int max_len, const int* kept_idx, const int* evict_idx,
+                                   int* rank, int* status, cudaStream_t stream);
+
+// Copies up to kReqChunk table entries, passed by value as a kernel argument, into the workspace;
+// this keeps the host free of any synchronising copy.
+constexpr int kReqChunk = 40;
+struct ReqChunk { Req r[kReqChunk]; };
+cudaError_t launch_write_table(const ReqChunk& chunk, int count, Req* dst, cudaStream_t stream);
 
 cudaError_t launch_invert_assignment(const int* assign, const Req* reqs, int n_req, int n_kv_heads,
                                      int* row_ptr, int* members, unsigned* sort_a, unsigned* sort_b,

@@ -1,0 +1,432 @@
+// Bandwidth-bound kernels of the path: key norms, compaction of the kept keys (the B operand of
+// the matching), row arg-max of given similarity matrices, inversion of the evicted->kept
+// assignment into per-kept-row member lists, and the merge/compact kernel (Eq. 6-7, 10-12).
+//
+// A K or V row is 128 bf16 = 256 bytes = 16 lanes x 16 bytes, so a half-warp moves one row with
+// one 16-byte access per lane.
+#include <cuda_bf16.h>
+
+#include "internal.h"
+
+namespace lookm {
+namespace {
+
+struct Row8 { float v[8]; };
+
+__device__ __forceinline__ Row8 unpack8(const uint4& u) {
+    Row8 r;
+    const unsigned w[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        r.v[2 * i] = __uint_as_float(w[i] << 16);
+        r.v[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+    }
+    return r;
+}
+
+__device__ __forceinline__ uint4 pack8(const Row8& r) {
+    unsigned w[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const __nv_bfloat162 b = __floats2bfloat162_rn(r.v[2 * i], r.v[2 * i + 1]);
+        w[i] = *reinterpret_cast<const unsigned*>(&b);
+    }
+    return make_uint4(w[0], w[1], w[2], w[3]);
+}
+
+__device__ __forceinline__ const Req& find_req_by_slot(const Req* reqs, int n_req, long long g) {
+    int lo = 0, hi = n_req - 1;
+    while (lo < hi) {
+        const int mid = (lo + hi + 1) >> 1;
+        if ((long long)reqs[mid].slot_begin <= g) lo = mid; else hi = mid - 1;
+    }
+    return reqs[lo];
+}
+
+// ---------------------------------------------------------------------------------------------
+// 1 / |k| of every key row (0 for a zero row), the cosine denominators of Eq. 9.
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+key_norms_kernel(const __nv_bfloat16* __restrict__ k, long long stride_tok, long long stride_head,
+                 int n_kv_heads, long long T, float* __restrict__ rnorm_all) {
+    const int half = threadIdx.x >> 4, l16 = threadIdx.x & 15;
+    const long long n_rows = T * n_kv_heads;
+    for (long long r = (long long)blockIdx.x * 16 + half; r < n_rows; r += (long long)gridDim.x * 16) {
+        const long long tok = r / n_kv_heads;
+        const int h = (int)(r % n_kv_heads);
+        const uint4 u = *reinterpret_cast<const uint4*>(k + tok * stride_tok + h * stride_head + l16 * 8);
+        const Row8 x = unpack8(u);
+        float ss = 0.f;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) ss = fmaf(x.v[i], x.v[i], ss);
+#pragma unroll
+        for (int o = 8; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o, 16);
+        if (l16 == 0) rnorm_all[(long long)h * T + tok] = ss > 0.f ? 1.0f / sqrtf(ss) : 0.f;
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Kept keys of every (request, head) copied into one dense [rows, 128] matrix in kept-list
+// order, with their inverse norms.
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+gather_kept_kernel(const __nv_bfloat16* __restrict__ k, long long stride_tok, long long stride_head,
+                   const Req* __restrict__ reqs, int n_req, int n_kv_heads, long long T,
+                   long long total_rows, const int* __restrict__ kept_idx,
+                   const float* __restrict__ rnorm_all, __nv_bfloat16* __restrict__ kept_keys,
+                   float* __restrict__ rnorm_kept, int* status) {
+    const int half = threadIdx.x >> 4, l16 = threadIdx.x & 15;
+    const long long g = (long long)blockIdx.x * 16 + half;
+    if (g >= total_rows) return;
+    const Req& rq = find_req_by_slot(reqs, n_req, g);
+    const long long u = g - rq.slot_begin;
+    const int h = (int)(u / rq.B), slot = (int)(u % rq.B);
+    const long long dst = rq.kept_off + (long long)h * rq.B + slot;
+    int pos = kept_idx[dst];
+    if (pos < 0 || pos >= rq.L) { if (l16 == 0) atomicExch(status, (int)LOOKM_ERR_DEVICE_BAD_INDEX); pos = 0; }
+    const long long tok = rq.tok_begin + pos;
+    const uint4 u4 = *reinterpret_cast<const uint4*>(k + tok * stride_tok + h * stride_head + l16 * 8);
+    *reinterpret_cast<uint4*>(kept_keys + dst * kHeadDim + l16 * 8) = u4;
+    if (l16 == 0) rnorm_kept[dst] = rnorm_all[(long long)h * T + tok];
+}
+
+// ---------------------------------------------------------------------------------------------
+// Row arg-max of given similarity blocks (one warp per evicted row); lowest slot wins ties.
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+argmax_rows_kernel(const float* __restrict__ sim_matrix, const Req* __restrict__ reqs,
+                   int n_kv_heads, int* __restrict__ assign, float* __restrict__ sim) {
+    const Req rq = reqs[blockIdx.z];
+    const int h = blockIdx.y;
+    const int e = blockIdx.x * 8 + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
+    if (e >= rq.E) return;
+    const float* row = sim_matrix + rq.sim_off + ((long long)h * rq.E + e) * rq.B;
+    float best = -INFINITY;
+    int slot = 0x7fffffff;
+    for (int c = lane; c < rq.B; c += 32) {
+        const float v = row[c];
+        if (v > best) { best = v; slot = c; }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const float ob = __shfl_xor_sync(0xffffffffu, best, o);
+        const int os = __shfl_xor_sync(0xffffffffu, slot, o);
+        if (ob > best || (ob == best && os < slot)) { best = ob; slot = os; }
+    }
+    if (lane == 0) {
+        assign[rq.ev_off + (long long)h * rq.E + e] = slot;
+        sim[rq.ev_off + (long long)h * rq.E + e] = best;
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Inversion of the assignment: for each (request, head) a stable sort of the evicted ranks by
+// their kept slot gives, per kept row, its members in ascending position, as CSR
+// (row_ptr [B + 1 per (request, head)], members [E]).  One CTA per (request, head); stable LSD
+// radix sort with 8-bit digits: every warp owns a contiguous segment of the list, ranks equal
+// digits inside a 32-element step with match.any, and adds the counts of earlier steps and
+// earlier warps.  Keys are packed as (slot << 0) in one array and values in the other.
+// ---------------------------------------------------------------------------------------------
+constexpr int kInvThreads = 1024;
+
+__global__ void __launch_bounds__(kInvThreads)
+invert_assignment_kernel(const int* __restrict__ assign, const Req* __restrict__ reqs,
+                         int n_kv_heads, int* __restrict__ row_ptr, int* __restrict__ members,
+                         unsigned* __restrict__ sort_a, unsigned* __restrict__ sort_b, int* status) {
+    __shared__ int cnt[32][256];                         // [warp][digit]
+    __shared__ int digit_tot[256];
+    const Req rq = reqs[blockIdx.y];
+    const int h = blockIdx.x;
+    const int E = rq.E, B = rq.B;
+    const long long ev_base = rq.ev_off + (long long)h * E;
+    int* rp = row_ptr + rq.rp_off + (long long)h * (B + 1);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const unsigned lt_mask = (1u << lane) - 1u;
+
+    if (E == 0) {
+        for (int c = threadIdx.x; c <= B; c += kInvThreads) rp[c] = 0;
+        return;
+    }
+    // segment of the list owned by each warp: a multiple of 32 elements
+    const int seg = ((E + 32 * 32 - 1) / (32 * 32)) * 32;
+    const int s_begin = min(E, warp * seg), s_end = min(E, s_begin + seg);
+
+    int bits = 1;
+    while ((1 << bits) < B) ++bits;
+    const int n_pass = (bits + 7) / 8;
+
+    // pass p reads (key, value) from src and writes to dst; pass 0 reads assign directly
+    unsigned* key_buf[2] = {sort_a + 2 * ev_base, sort_b + 2 * ev_base};   // [E keys][E values] each
+    for (int pass = 0; pass < n_pass; ++pass) {
+        const int shift = pass * 8;
+        const unsigned* src_k = pass ? key_buf[(pass - 1) & 1] : nullptr;
+        const unsigned* src_v = pass ? key_buf[(pass - 1) & 1] + E : nullptr;
+        unsigned* dst_k = key_buf[pass & 1];
+        unsigned* dst_v = key_buf[pass & 1] + E;
+        for (int i = threadIdx.x; i < 32 * 256; i += kInvThreads) (&cnt[0][0])[i] = 0;
+        __syncthreads();
+        // count
+        for (int base = s_begin; base < s_end; base += 32) {
+            const int i = base + lane;
+            const bool valid = i < s_end;
+            unsigned key = 0;
+            if (valid) {
+                if (pass) key = src_k[i];
+                else {
+                    int a = assign[ev_base + i];
+                    if (a < 0 || a >= B) { atomicExch(status, (int)LOOKM_ERR_DEVICE_BAD_INDEX); a = 0; }
+                    key = (unsigned)a;
+                }
+            }
+            const unsigned d = valid ? ((key >> shift) & 255u) : 256u + lane;   // invalid lanes never match
+            const unsigned peers = __match_any_sync(0xffffffffu, d);
+            if (valid && (peers & lt_mask) == 0u) cnt[warp][d] += __popc(peers);
+            __syncwarp();
+        }
+        __syncthreads();
+        // exclusive scan over (digit major, warp minor)
+        if (threadIdx.x < 256) {
+            int tot = 0;
+            for (int w = 0; w < 32; ++w) { const int c = cnt[w][threadIdx.x]; cnt[w][threadIdx.x] = tot; tot += c; }
+            digit_tot[threadIdx.x] = tot;
+        }
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            int run = 0;
+            for (int d = 0; d < 256; ++d) { const int c = digit_tot[d]; digit_tot[d] = run; run += c; }
+        }
+        __syncthreads();
+        // scatter
+        for (int base = s_begin; base < s_end; base += 32) {
+            const int i = base + lane;
+            const bool valid = i < s_end;
+            unsigned key = 0, val = 0;
+            if (valid) {
+                if (pass) { key = src_k[i]; val = src_v[i]; }
+                else {
+                    int a = assign[ev_base + i];
+                    if (a < 0 || a >= B) a = 0;
+                    key = (unsigned)a;
+                    val = (unsigned)i;
+                }
+            }
+            const unsigned d = valid ? ((key >> shift) & 255u) : 256u + lane;
+            const unsigned peers = __match_any_sync(0xffffffffu, d);
+            int off = 0;
+            if (valid) off = digit_tot[d] + cnt[warp][d] + __popc(peers & lt_mask);
+            __syncwarp();
+            if (valid && (peers & lt_mask) == 0u) cnt[warp][d] += __popc(peers);
+            __syncwarp();
+            if (valid) { dst_k[off] = key; dst_v[off] = val; }
+        }
+        __syncthreads();
+    }
+    const unsigned* fin_k = key_buf[(n_pass - 1) & 1];
+    const unsigned* fin_v = fin_k + E;
+    // members and the row boundaries: row_ptr[c] = first sorted index whose slot is >= c
+    for (int i = threadIdx.x; i < E; i += kInvThreads) {
+        members[ev_base + i] = (int)fin_v[i];
+        const int cur = (int)fin_k[i];
+        const int prev = i ? (int)fin_k[i - 1] : -1;
+        for (int c = prev + 1; c <= cur; ++c) rp[c] = i;
+        if (i == E - 1) for (int c = cur + 1; c <= B; ++c) rp[c] = E;
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Merge + compact: one warp per kept row (lanes 0-15 the K row, 16-31 the V row).  Each warp
+// gathers its kept row and its members, accumulates in fp32 in member order and rounds once.
+//   averaged : (x_c + sum x_e) / (n + 1)                       (Eq. 10)
+//   pivotal  : (x_c + 1/2 sum (x_e + x_c)) / (n + 1)           (Eq. 11)
+//   weighted : (x_c + sum sim_e x_e) / (n + 1)                 (Eq. 12)
+// A row without members is copied bit for bit.
+// ---------------------------------------------------------------------------------------------
+constexpr int kMergeWarps = 8;
+
+__global__ void __launch_bounds__(kMergeWarps * 32)
+merge_kernel(const __nv_bfloat16* __restrict__ k, const __nv_bfloat16* __restrict__ v,
+             long long stride_tok, long long stride_head, const Req* __restrict__ reqs, int n_req,
+             int n_kv_heads, long long total_rows, const int* __restrict__ kept_idx,
+             const int* __restrict__ evict_idx, const float* __restrict__ sim,
+             const int* __restrict__ row_ptr, const int* __restrict__ members, int varlen_output,
+             __nv_bfloat16* __restrict__ out_k, __nv_bfloat16* __restrict__ out_v, int* status) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const long long g = (long long)blockIdx.x * kMergeWarps + warp;
+    if (g >= total_rows) return;
+    int ri;
+    {
+        int lo = 0, hi = n_req - 1;
+        while (lo < hi) {
+            const int mid = (lo + hi + 1) >> 1;
+            if ((long long)reqs[mid].slot_begin <= g) lo = mid; else hi = mid - 1;
+        }
+        ri = lo;
+    }
+    const Req& rq = reqs[ri];
+    const long long u = g - rq.slot_begin;
+    const int h = (int)(u / rq.B), slot = (int)(u % rq.B);
+    const int l16 = lane & 15;
+    const __nv_bfloat16* src = (lane < 16 ? k : v) + (long long)h * stride_head + l16 * 8;
+    const long long kept_base = rq.kept_off + (long long)h * rq.B;
+    const long long ev_base = rq.ev_off + (long long)h * rq.E;
+    const int* rp = row_ptr + rq.rp_off + (long long)h * (rq.B + 1);
+
+    int pos_c = kept_idx[kept_base + slot];
+    if (pos_c < 0 || pos_c >= rq.L) { if (lane == 0) atomicExch(status, (int)LOOKM_ERR_DEVICE_BAD_INDEX); pos_c = 0; }
+    const uint4 raw_c = *reinterpret_cast<const uint4*>(src + (rq.tok_begin + pos_c) * stride_tok);
+    const int m_begin = rp[slot], m_end = rp[slot + 1];
+    const int n = m_end - m_begin;
+    uint4 result = raw_c;
+    if (n > 0) {
+        const bool weighted = (rq.mode == LOOKM_MERGE_WEIGHTED);
+        float acc[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) acc[i] = 0.f;
+        int m = m_begin;
+        for (; m + 4 <= m_end; m += 4) {                 // four member rows in flight per lane
+            int e[4];
+            long long tok[4];
+            float w[4];
+            uint4 raw[4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) e[q] = members[ev_base + m + q];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                int pe = evict_idx[ev_base + e[q]];
+                if (pe < 0 || pe >= rq.L) { atomicExch(status, (int)LOOKM_ERR_DEVICE_BAD_INDEX); pe = 0; }
+                tok[q] = rq.tok_begin + pe;
+                w[q] = weighted ? sim[ev_base + e[q]] : 1.f;
+            }
+#pragma unroll
+            for (int q = 0; q < 4; ++q) raw[q] = *reinterpret_cast<const uint4*>(src + tok[q] * stride_tok);
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const Row8 x = unpack8(raw[q]);
+#pragma unroll
+                for (int i = 0; i < 8; ++i) acc[i] = fmaf(w[q], x.v[i], acc[i]);
+            }
+        }
+        for (; m < m_end; ++m) {
+            const int e = members[ev_base + m];
+            int pe = evict_idx[ev_base + e];
+            if (pe < 0 || pe >= rq.L) { atomicExch(status, (int)LOOKM_ERR_DEVICE_BAD_INDEX); pe = 0; }
+            const float w = weighted ? sim[ev_base + e] : 1.f;
+            const Row8 x = unpack8(*reinterpret_cast<const uint4*>(src + (rq.tok_begin + pe) * stride_tok));
+#pragma unroll
+            for (int i = 0; i < 8; ++i) acc[i] = fmaf(w, x.v[i], acc[i]);
+        }
+        const Row8 xc = unpack8(raw_c);
+        const float inv = 1.0f / (float)(n + 1);
+        // pivotal: each member contributes (x_e + x_c) / 2
+        const float wc = (rq.mode == LOOKM_MERGE_PIVOTAL) ? 1.f + 0.5f * (float)n : 1.f;
+        const float wm = (rq.mode == LOOKM_MERGE_PIVOTAL) ? 0.5f : 1.f;
+        Row8 o;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) o.v[i] = fmaf(wc, xc.v[i], wm * acc[i]) * inv;
+        result = pack8(o);
+    }
+    __nv_bfloat16* dst_base = lane < 16 ? out_k : out_v;
+    long long row;
+    if (varlen_output) row = ((long long)rq.out_begin + slot) * n_kv_heads + h;
+    else row = (long long)h * rq.B + slot;
+    *reinterpret_cast<uint4*>(dst_base + row * kHeadDim + l16 * 8) = result;
+}
+
+// Inverse map of given kept / evicted lists (used when the lists come from the caller).
+__global__ void __launch_bounds__(256)
+rank_from_lists_kernel(const Req* __restrict__ reqs, int n_kv_heads, long long T,
+                       const int* __restrict__ kept_idx, const int* __restrict__ evict_idx,
+                       int* __restrict__ rank, int* status) {
+    const Req rq = reqs[blockIdx.z];
+    const int h = blockIdx.y;
+    const int i = blockIdx.x * 256 + threadIdx.x;
+    if (i >= rq.L) return;
+    int pos, val;
+    if (i < rq.B) { pos = kept_idx[rq.kept_off + (long long)h * rq.B + i]; val = -1 - i; }
+    else { pos = evict_idx[rq.ev_off + (long long)h * rq.E + (i - rq.B)]; val = i - rq.B; }
+    if (pos < 0 || pos >= rq.L) { atomicExch(status, (int)LOOKM_ERR_DEVICE_BAD_INDEX); return; }
+    rank[(long long)h * T + rq.tok_begin + pos] = val;
+}
+
+__global__ void write_table_kernel(const __grid_constant__ ReqChunk chunk, int count, Req* dst) {
+    const int i = threadIdx.x;
+    if (i < count) dst[i] = chunk.r[i];
+}
+
+}  // namespace
+
+cudaError_t launch_rank_from_lists(const Req* reqs, int n_req, int n_kv_heads, long long T,
+                                   int max_len, const int* kept_idx, const int* evict_idx,
+                                   int* rank, int* status, cudaStream_t stream) {
+    if (max_len <= 0) return cudaSuccess;
+    dim3 grid((max_len + 255) / 256, n_kv_heads, n_req);
+    rank_from_lists_kernel<<<grid, 256, 0, stream>>>(reqs, n_kv_heads, T, kept_idx, evict_idx, rank,
+                                                     status);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_write_table(const ReqChunk& chunk, int count, Req* dst, cudaStream_t stream) {
+    write_table_kernel<<<1, 64, 0, stream>>>(chunk, count, dst);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_key_norms(const void* k, long long stride_tok, long long stride_head,
+                             int n_kv_heads, long long T, float* rnorm_all, cudaStream_t stream) {
+    const long long rows = T * n_kv_heads;
+    if (rows <= 0) return cudaSuccess;
+    long long blocks = (rows + 15) / 16;
+    if (blocks > 148 * 32) blocks = 148 * 32;
+    key_norms_kernel<<<(int)blocks, 256, 0, stream>>>((const __nv_bfloat16*)k, stride_tok, stride_head,
+                                                      n_kv_heads, T, rnorm_all);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_gather_kept(const void* k, long long stride_tok, long long stride_head,
+                               const Req* reqs, int n_req, int n_kv_heads, long long T,
+                               long long total_kept_rows, const int* kept_idx,
+                               const float* rnorm_all, void* kept_keys, float* rnorm_kept,
+                               int* status, cudaStream_t stream) {
+    if (total_kept_rows <= 0) return cudaSuccess;
+    const long long blocks = (total_kept_rows + 15) / 16;
+    gather_kept_kernel<<<(unsigned)blocks, 256, 0, stream>>>(
+        (const __nv_bfloat16*)k, stride_tok, stride_head, reqs, n_req, n_kv_heads, T,
+        total_kept_rows, kept_idx, rnorm_all, (__nv_bfloat16*)kept_keys, rnorm_kept, status);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_invert_assignment(const int* assign, const Req* reqs, int n_req, int n_kv_heads,
+                                     int* row_ptr, int* members, unsigned* sort_a, unsigned* sort_b,
+                                     int* status, cudaStream_t stream) {
+    dim3 grid(n_kv_heads, n_req);
+    invert_assignment_kernel<<<grid, kInvThreads, 0, stream>>>(assign, reqs, n_kv_heads, row_ptr,
+                                                               members, sort_a, sort_b, status);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_merge(const void* k, const void* v, long long stride_tok, long long stride_head,
+                         const Req* reqs, int n_req, int n_kv_heads, long long T,
+                         long long total_kept_rows, const int* kept_idx, const int* evict_idx,
+                         const float* sim, const int* row_ptr, const int* members,
+                         int varlen_output, void* out_k, void* out_v, int* status,
+                         cudaStream_t stream) {
+    (void)T;
+    if (total_kept_rows <= 0) return cudaSuccess;
+    const long long blocks = (total_kept_rows + kMergeWarps - 1) / kMergeWarps;
+    merge_kernel<<<(unsigned)blocks, kMergeWarps * 32, 0, stream>>>(
+        (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, stride_tok, stride_head, reqs, n_req,
+        n_kv_heads, total_kept_rows, kept_idx, evict_idx, sim, row_ptr, members, varlen_output,
+        (__nv_bfloat16*)out_k, (__nv_bfloat16*)out_v, status);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_argmax_rows(const float* sim_matrix, const Req* reqs, int n_req,
+                                    int n_kv_heads, int max_evicted, int* assign, float* sim,
+                                    cudaStream_t stream) {
+    if (max_evicted <= 0) return cudaSuccess;
+    dim3 grid((max_evicted + 7) / 8, n_kv_heads, n_req);
+    argmax_rows_kernel<<<grid, 256, 0, stream>>>(sim_matrix, reqs, n_kv_heads, assign, sim);
+    return cudaGetLastError();
+}
+
+}  // namespace lookm

@@ -1,0 +1,200 @@
+// Selection kernel: recent window, text prior and Top-N (Eq. 5-8), one CTA per (request, KV head).
+//
+// The text prior is applied as an ordering rule: adding T_p = max(A_s) to every text score makes
+// any text token outrank any image token (scores are positive), so candidates are ordered by
+// (is_text, score, lower position).  With n_text text candidates and N slots:
+//   n_text <= N : all text candidates are kept and the best N - n_text image candidates;
+//   n_text >  N : the best N text candidates are kept and no image candidate.
+// Either way one class is kept wholesale or not at all and the other needs an exact top-k, done
+// by a 4-pass radix select on an order-preserving 32-bit key; ties at the threshold go to the
+// lowest positions.  A final ordered pass writes the kept and evicted lists in ascending position.
+#include "internal.h"
+
+namespace lookm {
+namespace {
+
+constexpr int kSelThreads = 1024;
+constexpr int kPerThread = 4;
+
+__device__ __forceinline__ unsigned order_key(float s) {
+    unsigned b = __float_as_uint(s);
+    if (b == 0x80000000u) b = 0u;                        // -0 and +0 compare equal
+    return (b & 0x80000000u) ? ~b : (b | 0x80000000u);   // larger float <=> larger key
+}
+
+// Exclusive block scan of two ints per thread; returns the block totals through ta / tb.
+__device__ __forceinline__ void block_scan2(int a, int b, int& ea, int& eb, int& ta, int& tb,
+                                            int (*warp_tot)[2]) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    int ia = a, ib = b;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int xa = __shfl_up_sync(0xffffffffu, ia, o);
+        const int xb = __shfl_up_sync(0xffffffffu, ib, o);
+        if (lane >= o) { ia += xa; ib += xb; }
+    }
+    __syncthreads();                                     // protects warp_tot from the previous use
+    if (lane == 31) { warp_tot[warp][0] = ia; warp_tot[warp][1] = ib; }
+    __syncthreads();
+    if (warp == 0) {
+        int wa = warp_tot[lane][0], wb = warp_tot[lane][1];
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int xa = __shfl_up_sync(0xffffffffu, wa, o);
+            const int xb = __shfl_up_sync(0xffffffffu, wb, o);
+            if (lane >= o) { wa += xa; wb += xb; }
+        }
+        warp_tot[lane][0] = wa;
+        warp_tot[lane][1] = wb;
+    }
+    __syncthreads();
+    const int ba = warp ? warp_tot[warp - 1][0] : 0;
+    const int bb = warp ? warp_tot[warp - 1][1] : 0;
+    ea = ba + ia - a;
+    eb = bb + ib - b;
+    ta = warp_tot[31][0];
+    tb = warp_tot[31][1];
+}
+
+__global__ void __launch_bounds__(kSelThreads)
+select_kernel(const float* __restrict__ scores, const uint8_t* __restrict__ mask,
+              const Req* __restrict__ reqs, int n_kv_heads, long long T, int* __restrict__ kept_idx,
+              int* __restrict__ evict_idx, int* __restrict__ rank) {
+    __shared__ int hist[256];
+    __shared__ int warp_tot[32][2];
+    __shared__ int sh_val[4];
+
+    const Req rq = reqs[blockIdx.y];
+    const int h = blockIdx.x;
+    const float* s = scores + (long long)h * T + rq.tok_begin;
+    const uint8_t* msk = mask + rq.tok_begin;
+    const int L = rq.L, B = rq.B, M = rq.M;
+    const int N = B - M, nc = L - M;
+
+    // ---- count text candidates ---------------------------------------------------------------
+    int cnt = 0;
+    for (int j = threadIdx.x; j < nc; j += kSelThreads) cnt += (msk[j] == 0);
+    {
+        int e0, e1, t0, t1;
+        block_scan2(cnt, 0, e0, e1, t0, t1, warp_tot);
+        cnt = t0;
+    }
+    const int n_text = cnt;
+    // class whose members are ranked (1 = image); the other class is kept entirely or not at all
+    const int sel_cls = (n_text <= N) ? 1 : 0;
+    const bool other_kept = (n_text <= N);
+    int k = (n_text <= N) ? (N - n_text) : N;            // how many of sel_cls to keep
+    const int n_sel = sel_cls ? (nc - n_text) : n_text;
+
+    // ---- radix select: key of the k-th largest member of sel_cls -------------------------------
+    unsigned thr = 0u;          // threshold key
+    int need_ties = 0;          // members equal to thr to keep (lowest positions first)
+    bool take_all = (k >= n_sel), take_none = (k <= 0);
+    if (!take_all && !take_none) {
+        unsigned prefix = 0u, pmask = 0u;
+        int remaining = k;
+        for (int shift = 24; shift >= 0; shift -= 8) {
+            for (int i = threadIdx.x; i < 256; i += kSelThreads) hist[i] = 0;
+            __syncthreads();
+            for (int j = threadIdx.x; j < nc; j += kSelThreads) {
+                if ((msk[j] != 0) == (sel_cls != 0)) {
+                    const unsigned key = order_key(s[j]);
+                    if ((key & pmask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1);
+                }
+            }
+            __syncthreads();
+            if (threadIdx.x == 0) {
+                int acc = 0, d = 255;
+                for (; d > 0; --d) {
+                    if (acc + hist[d] >= remaining) break;
+                    acc += hist[d];
+                }
+                sh_val[0] = d;
+                sh_val[1] = remaining - acc;             // still to take inside digit d
+            }
+            __syncthreads();
+            prefix |= (unsigned)sh_val[0] << shift;
+            pmask |= 255u << shift;
+            remaining = sh_val[1];
+            __syncthreads();
+        }
+        thr = prefix;
+        need_ties = remaining;
+    }
+
+    // ---- ordered emission -----------------------------------------------------------------------
+    const long long kept_base = rq.kept_off + (long long)h * B;
+    const long long ev_base = rq.ev_off + (long long)h * rq.E;
+    int* rk = rank ? rank + (long long)h * T + rq.tok_begin : nullptr;
+    int kept_run = 0, tie_run = 0;
+    for (int base = 0; base < L; base += kSelThreads * kPerThread) {
+        const int j0 = base + threadIdx.x * kPerThread;
+        int keep[kPerThread], tie[kPerThread];
+        int nk = 0, nt = 0;
+#pragma unroll
+        for (int q = 0; q < kPerThread; ++q) {
+            const int j = j0 + q;
+            keep[q] = 0;
+            tie[q] = 0;
+            if (j < L) {
+                if (j >= nc) {
+                    keep[q] = 1;
+                } else {
+                    const int cls = (msk[j] != 0);
+                    if (cls != sel_cls) {
+                        keep[q] = other_kept;
+                    } else if (take_all) {
+                        keep[q] = 1;
+                    } else if (!take_none) {
+                        const unsigned key = order_key(s[j]);
+                        if (key > thr) keep[q] = 1;
+                        else if (key == thr) tie[q] = 1;
+                    }
+                }
+            }
+            nt += tie[q];
+        }
+        // ties first: a tie is kept while fewer than need_ties equal keys precede it
+        int e_tie, e_dummy, t_tie, t_dummy;
+        block_scan2(nt, 0, e_tie, e_dummy, t_tie, t_dummy, warp_tot);
+        int tr = tie_run + e_tie;
+#pragma unroll
+        for (int q = 0; q < kPerThread; ++q) {
+            if (tie[q]) { if (tr < need_ties) keep[q] = 1; ++tr; }
+            nk += keep[q];
+        }
+        int e_keep, t_keep;
+        block_scan2(nk, 0, e_keep, e_dummy, t_keep, t_dummy, warp_tot);
+        int slot = kept_run + e_keep;
+#pragma unroll
+        for (int q = 0; q < kPerThread; ++q) {
+            const int j = j0 + q;
+            if (j < L) {
+                if (keep[q]) {
+                    kept_idx[kept_base + slot] = j;
+                    if (rk) rk[j] = -1 - slot;
+                    ++slot;
+                } else {
+                    const int e = j - slot;              // evicted before j = j - kept before j
+                    evict_idx[ev_base + e] = j;
+                    if (rk) rk[j] = e;
+                }
+            }
+        }
+        kept_run += t_keep;
+        tie_run += t_tie;
+    }
+}
+
+}  // namespace
+
+cudaError_t launch_select(const float* scores, const uint8_t* mask, const Req* reqs, int n_req,
+                          int n_kv_heads, long long T, int* kept_idx, int* evict_idx, int* rank,
+                          cudaStream_t stream) {
+    dim3 grid(n_kv_heads, n_req);
+    select_kernel<<<grid, kSelThreads, 0, stream>>>(scores, mask, reqs, n_kv_heads, T, kept_idx,
+                                                    evict_idx, rank);
+    return cudaGetLastError();
+}
+
+}  // namespace lookm
