@@ -144,6 +144,25 @@ int lookm_merge(const void* k, const void* v, const int* kept_idx, const int* ev
                 int varlen_output, void* out_k, void* out_v, void* workspace,
                 size_t workspace_bytes, void* cuda_stream);
 
+/* Byte offsets, inside the workspace, of the intermediate results a whole-path call leaves behind
+ * (layouts as described at the top: scores [n_kv_heads, T] fp32, lse [n_q_heads, T] fp32,
+ * rank [n_kv_heads, T] i32, kept/evicted/assign lists i32, sim fp32).  They stay valid until
+ * the next call that uses the workspace and let a harness inspect every step of Eq. 4-9. */
+typedef struct {
+    size_t status, lse, scores, rank, kept_idx, evict_idx, assign, sim;
+} lookm_workspace_offsets;
+int lookm_workspace_layout(const lookm_layout* layout, int n_requests, const int* seq_lens_host,
+                           lookm_workspace_offsets* offsets_host);
+
+/* Optional per-stage timing.  While set (per host thread), every whole-path call records the
+ * caller's events (cudaEvent_t handles in a host array that must stay alive) on its stream at the
+ * step boundaries: [0] start, [1] after the first score sweep, [2] after the second (Eq. 4),
+ * [3] after the selection (Eq. 5-8), [4] after key norms and kept-key compaction, [5] after the
+ * matching (Eq. 9), [6] after the assignment inversion, [7] after merge + compaction (Eq. 10-12).
+ * n_events must be LOOKM_N_STAGE_EVENTS; pass NULL, 0 to stop.  Nothing is recorded otherwise. */
+#define LOOKM_N_STAGE_EVENTS 8
+int lookm_set_stage_events(void* const* events_host, int n_events);
+
 /* Synchronises `cuda_stream`, then returns and clears the device status word kept at the start
  * of `workspace` (LOOKM_OK if no kernel reported a problem since the last call that used this
  * workspace began). */

@@ -20,9 +20,16 @@ OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE_TOO_SMALL, ERR_CUDA, ERR_DEV
     ERR_DEVICE_BAD_INDEX = range(7)
 MERGE_AVERAGE, MERGE_PIVOTAL, MERGE_WEIGHTED = 0, 1, 2
 
-EXPORTS = ["lookm_workspace_size", "lookm_compress_layer", "lookm_compress_varlen", "lookm_score",
+EXPORTS = ["lookm_workspace_size", "lookm_workspace_layout", "lookm_compress_layer", "lookm_compress_varlen", "lookm_score",
            "lookm_select", "lookm_match", "lookm_match_from_sim", "lookm_merge",
-           "lookm_device_status", "lookm_last_launch_count", "lookm_strerror"]
+           "lookm_set_stage_events", "lookm_device_status", "lookm_last_launch_count", "lookm_strerror"]
+N_STAGE_EVENTS = 8
+STAGE_NAMES = ["score_sweep1", "score_sweep2", "select", "norms_gather", "match", "invert", "merge"]
+
+
+class WorkspaceOffsets(C.Structure):
+    _fields_ = [(n, C.c_size_t) for n in ("status", "lse", "scores", "rank", "kept_idx", "evict_idx",
+                                          "assign", "sim")]
 
 
 class Layout(C.Structure):
@@ -44,6 +51,8 @@ def lib():
         lp = C.POINTER(Layout)
         L.lookm_workspace_size.argtypes = [lp, C.c_int, ip, ip]
         L.lookm_workspace_size.restype = sz
+        L.lookm_workspace_layout.argtypes = [lp, C.c_int, ip, C.POINTER(WorkspaceOffsets)]
+        L.lookm_workspace_layout.restype = C.c_int
         L.lookm_compress_layer.argtypes = [vp, vp, vp, vp, C.c_int, C.c_int, C.c_int, C.c_int, lp,
                                            vp, vp, ip, vp, sz, vp]
         L.lookm_compress_varlen.argtypes = [vp, vp, vp, vp, ip, C.c_int, ip, ip, ip, lp, vp, vp, ip,
@@ -54,6 +63,8 @@ def lib():
         L.lookm_match_from_sim.argtypes = [vp, ip, C.c_int, ip, C.c_int, vp, vp, vp, sz, vp]
         L.lookm_merge.argtypes = [vp, vp, vp, vp, vp, vp, ip, C.c_int, ip, ip, lp, C.c_int, vp, vp,
                                   vp, sz, vp]
+        L.lookm_set_stage_events.argtypes = [C.POINTER(C.c_void_p), C.c_int]
+        L.lookm_set_stage_events.restype = C.c_int
         L.lookm_device_status.argtypes = [vp, vp]
         L.lookm_last_launch_count.argtypes = []
         L.lookm_strerror.argtypes = [C.c_int]
@@ -103,6 +114,47 @@ def make_layout(q, k, softmax_scale: float = 0.0) -> Layout:
 
 def lookm_workspace_size(layout: Layout, seq_lens: Sequence[int], budgets: Optional[Sequence[int]] = None) -> int:
     return int(lib().lookm_workspace_size(C.byref(layout), len(seq_lens), _ints(seq_lens), _ints(budgets)))
+
+
+def lookm_workspace_layout(layout: Layout, seq_lens: Sequence[int]) -> WorkspaceOffsets:
+    off = WorkspaceOffsets()
+    check(lib().lookm_workspace_layout(C.byref(layout), len(seq_lens), _ints(seq_lens), C.byref(off)))
+    return off
+
+
+def read_intermediates(workspace, layout: Layout, seq_lens: Sequence[int], budgets: Sequence[int]):
+    """Copies the intermediate results of the last whole-path call out of the workspace.
+
+    Returns (scores [Hkv, T] float32, per_request) where per_request[r][h] is the tuple
+    (kept positions, evicted positions, assign, sim) of request r and KV head h as numpy arrays.
+    """
+    import numpy as np
+    import torch
+    torch.cuda.synchronize()
+    off = lookm_workspace_layout(layout, seq_lens)
+    Hkv, T = layout.n_kv_heads, int(sum(seq_lens))
+    Bs = [min(int(b), int(L)) for b, L in zip(budgets, seq_lens)]
+    Es = [int(L) - b for b, L in zip(Bs, seq_lens)]
+
+    def view(byte_off, count, dtype):
+        nbytes = count * 4
+        return workspace[byte_off:byte_off + nbytes].view(dtype).cpu().numpy()
+
+    scores = view(off.scores, Hkv * T, torch.float32).reshape(Hkv, T)
+    kept = view(off.kept_idx, Hkv * sum(Bs), torch.int32)
+    ev = view(off.evict_idx, Hkv * sum(Es), torch.int32)
+    asg = view(off.assign, Hkv * sum(Es), torch.int32)
+    sim = view(off.sim, Hkv * sum(Es), torch.float32)
+    per_request, ko, eo = [], 0, 0
+    for b, e in zip(Bs, Es):
+        heads = []
+        for h in range(Hkv):
+            heads.append((kept[ko + h * b: ko + (h + 1) * b], ev[eo + h * e: eo + (h + 1) * e],
+                          asg[eo + h * e: eo + (h + 1) * e], sim[eo + h * e: eo + (h + 1) * e]))
+        per_request.append(heads)
+        ko += Hkv * b
+        eo += Hkv * e
+    return scores, per_request
 
 
 def lookm_compress_layer(q, k, v, modality_mask, seq_len, budget, recent_window, merge_mode, layout,
@@ -163,6 +215,21 @@ def lookm_merge(k, v, kept_idx, evict_idx, assign, sim, cu_seqlens, budgets, mer
                              C.byref(layout), int(bool(varlen_output)), _ptr(out_k), _ptr(out_v),
                              _ptr(workspace), workspace.numel() * workspace.element_size(),
                              _stream(stream))
+
+
+_stage_event_array = None
+
+
+def lookm_set_stage_events(events) -> int:
+    """events: 8 torch.cuda.Event (created with enable_timing=True and recorded once so that their
+    handles exist), or None to stop per-stage timing."""
+    global _stage_event_array
+    if events is None:
+        _stage_event_array = None
+        return lib().lookm_set_stage_events(None, 0)
+    arr = (C.c_void_p * len(events))(*[e.cuda_event for e in events])
+    _stage_event_array = arr                     # the library keeps the pointer: keep it alive
+    return lib().lookm_set_stage_events(arr, len(events))
 
 
 def lookm_device_status(workspace, stream=None) -> int:

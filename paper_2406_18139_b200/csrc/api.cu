@@ -14,6 +14,13 @@ namespace lookm {
 namespace {
 
 thread_local int g_launches = 0;
+thread_local void* const* g_stage_events = nullptr;
+
+// Records stage event i of the caller (if per-stage timing is on); errors are ignored on purpose:
+// timing must never change the result of a call.
+void mark_stage(int i, cudaStream_t st) {
+    if (g_stage_events && g_stage_events[i]) cudaEventRecord(static_cast<cudaEvent_t>(g_stage_events[i]), st);
+}
 
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
@@ -263,16 +270,18 @@ int run_score(const Plan& pl, const DeviceInfo& di, const lookm_layout* lay, con
         LOOKM_CUDA(launch_tile_kernel(kSweep1, map_q, map_k, p, di.sms, st));
         ++g_launches;
     }
+    mark_stage(1, st);
     p.n_items = pl.n_items[kSweep2];
     LOOKM_CUDA(launch_tile_kernel(kSweep2, map_k, map_q, p, di.sms, st));
     ++g_launches;
+    mark_stage(2, st);
     return LOOKM_OK;
 }
 
 int run_match(const Plan& pl, const DeviceInfo& di, const lookm_layout* lay, const void* k,
               const int* kept_idx, const int* rank, int* assign, float* sim, void* ws,
               cudaStream_t st) {
-    if (pl.n_items[kMatch] == 0) return LOOKM_OK;
+    if (pl.n_items[kMatch] == 0) { mark_stage(4, st); mark_stage(5, st); return LOOKM_OK; }
     float* rnorm_all = at<float>(ws, pl.o_rnorm_all);
     float* rnorm_kept = at<float>(ws, pl.o_rnorm_kept);
     void* kept_keys = at<void>(ws, pl.o_kept_keys);
@@ -284,6 +293,7 @@ int run_match(const Plan& pl, const DeviceInfo& di, const lookm_layout* lay, con
                                   pl.n_kv_heads, pl.T, pl.total_slots, kept_idx, rnorm_all,
                                   kept_keys, rnorm_kept, at<int>(ws, pl.o_status), st));
     ++g_launches;
+    mark_stage(4, st);
     CUtensorMap map_k, map_c;
     LOOKM_TRY(make_map_3d(&map_k, k, pl.T, pl.n_kv_heads, lay->kv_stride_tok, lay->kv_stride_head));
     LOOKM_TRY(make_map_2d(&map_c, kept_keys, pl.total_slots));
@@ -296,6 +306,7 @@ int run_match(const Plan& pl, const DeviceInfo& di, const lookm_layout* lay, con
     p.sim = sim;
     LOOKM_CUDA(launch_tile_kernel(kMatch, map_k, map_c, p, di.sms, st));
     ++g_launches;
+    mark_stage(5, st);
     return LOOKM_OK;
 }
 
@@ -309,11 +320,13 @@ int run_merge(const Plan& pl, const lookm_layout* lay, const void* k, const void
                                         at<unsigned>(ws, pl.o_sort_a), at<unsigned>(ws, pl.o_sort_b),
                                         status, st));
     ++g_launches;
+    mark_stage(6, st);
     LOOKM_CUDA(launch_merge(k, v, lay->kv_stride_tok, lay->kv_stride_head, reqs, pl.n_req,
                             pl.n_kv_heads, pl.T, pl.total_slots, kept_idx, evict_idx, sim,
                             at<int>(ws, pl.o_row_ptr), at<int>(ws, pl.o_members), varlen_output,
                             out_k, out_v, status, st));
     ++g_launches;
+    mark_stage(7, st);
     return LOOKM_OK;
 }
 
@@ -335,6 +348,7 @@ int compress_common(const void* q, const void* k, const void* v, const uint8_t* 
         for (int r = 0; r < n_req; ++r) out_cu[r + 1] = out_cu[r] + pl.out_len[r];
     }
     LOOKM_TRY(begin_call(pl, ws, st));
+    mark_stage(0, st);
     float* scores = at<float>(ws, pl.o_scores);
     int* kept = at<int>(ws, pl.o_kept);
     int* evict = at<int>(ws, pl.o_evict);
@@ -345,6 +359,7 @@ int compress_common(const void* q, const void* k, const void* v, const uint8_t* 
     LOOKM_CUDA(launch_select(scores, mask, at<Req>(ws, pl.o_reqs), pl.n_req, pl.n_kv_heads, pl.T,
                              kept, evict, rank, st));
     ++g_launches;
+    mark_stage(3, st);
     LOOKM_TRY(run_match(pl, di, lay, k, kept, rank, assign, sim, ws, st));
     LOOKM_TRY(run_merge(pl, lay, k, v, kept, evict, assign, sim, varlen_output, out_k, out_v, ws, st));
     return LOOKM_OK;
@@ -364,6 +379,22 @@ size_t lookm_workspace_size(const lookm_layout* layout, int n_requests, const in
     if (build_plan(pl, layout, n_requests, nullptr, seq_lens_host, budgets_host, nullptr, nullptr) != LOOKM_OK)
         return 0;
     return pl.total;
+}
+
+int lookm_workspace_layout(const lookm_layout* layout, int n_requests, const int* seq_lens_host,
+                           lookm_workspace_offsets* offsets_host) {
+    Plan pl;
+    if (!seq_lens_host || !offsets_host) return LOOKM_ERR_INVALID_ARG;
+    LOOKM_TRY(build_plan(pl, layout, n_requests, nullptr, seq_lens_host, nullptr, nullptr, nullptr));
+    offsets_host->status = pl.o_status;
+    offsets_host->lse = pl.o_lse;
+    offsets_host->scores = pl.o_scores;
+    offsets_host->rank = pl.o_rank;
+    offsets_host->kept_idx = pl.o_kept;
+    offsets_host->evict_idx = pl.o_evict;
+    offsets_host->assign = pl.o_assign;
+    offsets_host->sim = pl.o_sim;
+    return LOOKM_OK;
 }
 
 int lookm_compress_layer(const void* q, const void* k, const void* v, const uint8_t* modality_mask,
@@ -502,6 +533,13 @@ int lookm_device_status(void* workspace, void* cuda_stream) {
 }
 
 int lookm_last_launch_count(void) { return g_launches; }
+
+int lookm_set_stage_events(void* const* events_host, int n_events) {
+    if (!events_host || n_events == 0) { g_stage_events = nullptr; return LOOKM_OK; }
+    if (n_events != LOOKM_N_STAGE_EVENTS) return LOOKM_ERR_INVALID_ARG;
+    g_stage_events = events_host;
+    return LOOKM_OK;
+}
 
 const char* lookm_strerror(int status) {
     switch (status) {
