@@ -154,6 +154,39 @@ typedef struct {
 int lookm_workspace_layout(const lookm_layout* layout, int n_requests, const int* seq_lens_host,
                            lookm_workspace_offsets* offsets_host);
 
+/* The merging step for callers that must not allocate device memory.  (The paper has no
+ * counterpart to this entry point; it exists for deployment reasons only.)
+ *
+ * Some hosts of this library cannot call cudaMalloc at the point where they compress a cache: an
+ * inference server that has handed all device memory to its own pool and forbids driver
+ * allocations on the serving path (they serialise with other streams), or a plug-in that runs
+ * inside someone else's memory budget and has nowhere to put a workspace.  For them this variant
+ * of lookm_merge keeps its scratch (request table, member lists, sort buffers, status word) in a
+ * fixed array inside the library's device image, LOOKM_NOALLOC_SCRATCH_BYTES large, which every GPU
+ * that loads the library holds until the process exits.  Inputs and outputs are still the
+ * caller's, with the meaning and layouts of lookm_merge.
+ *
+ * Limits: the scratch needs 24 bytes per (KV head, token) plus a small table, so
+ * n_kv_heads * total_tokens may be at most about 349,000 (e.g. 32 heads x 8192 tokens uses
+ * 6.3 MB); larger batches return LOOKM_ERR_WORKSPACE_TOO_SMALL before anything is enqueued.
+ * The call performs no cudaMalloc/cudaFree and calls no allocating routine.
+ *
+ * The first call on each device looks up the array's device address (cudaGetSymbolAddress, with
+ * that device current) and caches it; make that first call outside any stream capture.
+ *
+ * All calls on a device share the one array, and it keeps what the previous call left in it.
+ * Each call clears the status word and rewrites everything it later reads, so back-to-back calls
+ * on one stream are safe; calls that can overlap on the GPU (different streams without an
+ * ordering between them) race on the array and must be serialised by the caller.
+ * lookm_noalloc_status() is lookm_device_status() for this scratch. */
+#define LOOKM_NOALLOC_SCRATCH_BYTES (8u << 20)
+int lookm_merge_noalloc(const void* k, const void* v, const int* kept_idx, const int* evict_idx,
+                        const int* assign, const float* sim, const int* cu_seqlens_host,
+                        int n_requests, const int* budgets_host, const int* merge_modes_host,
+                        const lookm_layout* layout, int varlen_output, void* out_k, void* out_v,
+                        void* cuda_stream);
+int lookm_noalloc_status(void* cuda_stream);
+
 /* Optional per-stage timing.  While set (per host thread), every whole-path call records the
  * caller's events (cudaEvent_t handles in a host array that must stay alive) on its stream at the
  * step boundaries: [0] start, [1] after the first score sweep, [2] after the second (Eq. 4),

@@ -22,7 +22,7 @@ MERGE_AVERAGE, MERGE_PIVOTAL, MERGE_WEIGHTED = 0, 1, 2
 
 EXPORTS = ["lookm_workspace_size", "lookm_workspace_layout", "lookm_compress_layer", "lookm_compress_varlen", "lookm_score",
            "lookm_select", "lookm_match", "lookm_match_from_sim", "lookm_merge",
-           "lookm_set_stage_events", "lookm_device_status", "lookm_last_launch_count", "lookm_strerror"]
+           "lookm_set_stage_events", "lookm_merge_noalloc", "lookm_noalloc_status", "lookm_device_status", "lookm_last_launch_count", "lookm_strerror"]
 N_STAGE_EVENTS = 8
 STAGE_NAMES = ["score_sweep1", "score_sweep2", "select", "norms_gather", "match", "invert", "merge"]
 
@@ -65,6 +65,10 @@ def lib():
                                   vp, sz, vp]
         L.lookm_set_stage_events.argtypes = [C.POINTER(C.c_void_p), C.c_int]
         L.lookm_set_stage_events.restype = C.c_int
+        L.lookm_merge_noalloc.argtypes = [vp, vp, vp, vp, vp, vp, ip, C.c_int, ip, ip, lp, C.c_int, vp, vp, vp]
+        L.lookm_merge_noalloc.restype = C.c_int
+        L.lookm_noalloc_status.argtypes = [vp]
+        L.lookm_noalloc_status.restype = C.c_int
         L.lookm_device_status.argtypes = [vp, vp]
         L.lookm_last_launch_count.argtypes = []
         L.lookm_strerror.argtypes = [C.c_int]
@@ -215,6 +219,20 @@ def lookm_merge(k, v, kept_idx, evict_idx, assign, sim, cu_seqlens, budgets, mer
                              C.byref(layout), int(bool(varlen_output)), _ptr(out_k), _ptr(out_v),
                              _ptr(workspace), workspace.numel() * workspace.element_size(),
                              _stream(stream))
+
+
+def lookm_merge_noalloc(k, v, kept_idx, evict_idx, assign, sim, cu_seqlens, budgets, merge_modes, layout,
+                        varlen_output, out_k, out_v, stream=None):
+    """lookm_merge without a workspace argument: the library's built-in scratch array is used, so
+    the call allocates nothing (for hosts that may not call cudaMalloc while serving)."""
+    return lib().lookm_merge_noalloc(_ptr(k), _ptr(v), _ptr(kept_idx), _ptr(evict_idx), _ptr(assign),
+                                     _ptr(sim), _ints(cu_seqlens), len(cu_seqlens) - 1, _ints(budgets),
+                                     _ints(merge_modes), C.byref(layout), int(bool(varlen_output)),
+                                     _ptr(out_k), _ptr(out_v), _stream(stream))
+
+
+def lookm_noalloc_status(stream=None) -> int:
+    return lib().lookm_noalloc_status(_stream(stream))
 
 
 _stage_event_array = None

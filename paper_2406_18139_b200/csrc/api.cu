@@ -555,3 +555,75 @@ const char* lookm_strerror(int status) {
 }
 
 }  // extern "C"
+
+// ------------------------------------------------------------------------------------------------
+// lookm_merge_noalloc: the merge step with its scratch in a static device array.
+// ------------------------------------------------------------------------------------------------
+namespace {
+
+// Scratch of the no-allocation merge: status word, request table, member lists (CSR) and the two
+// sort buffers.  Lives in the library's device image, so every GPU that loads the library holds
+// these bytes until the process exits.
+static __device__ __align__(256) unsigned char g_noalloc_scratch[LOOKM_NOALLOC_SCRATCH_BYTES];
+
+// Device address of the array on the current device.  The array's name is only a host-side
+// handle here; kernels must be given the address cudaGetSymbolAddress returns.  Looked up once
+// per device (with that device current) and cached.
+int noalloc_scratch_ptr(void** out) {
+    static std::mutex mu;
+    static void* cache[64] = {nullptr};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return LOOKM_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(mu);
+    if (!cache[dev]) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_noalloc_scratch) != cudaSuccess || !p) return LOOKM_ERR_CUDA;
+        cache[dev] = p;
+    }
+    *out = cache[dev];
+    return LOOKM_OK;
+}
+
+}  // namespace
+
+extern "C" int lookm_merge_noalloc(const void* k, const void* v, const int* kept_idx,
+                                   const int* evict_idx, const int* assign, const float* sim,
+                                   const int* cu_seqlens_host, int n_requests,
+                                   const int* budgets_host, const int* merge_modes_host,
+                                   const lookm_layout* layout, int varlen_output, void* out_k,
+                                   void* out_v, void* cuda_stream) {
+    if (!k || !v || !kept_idx || !evict_idx || !assign || !sim || !cu_seqlens_host || !budgets_host ||
+        !merge_modes_host || !out_k || !out_v)
+        return LOOKM_ERR_INVALID_ARG;
+    if (!varlen_output && n_requests != 1) return LOOKM_ERR_INVALID_ARG;
+    Plan pl;
+    LOOKM_TRY(build_plan(pl, layout, n_requests, cu_seqlens_host, nullptr, budgets_host, nullptr,
+                         merge_modes_host));
+    LOOKM_TRY(check_layout_ptrs(layout, nullptr, k, v));
+    // compact carving of just what the merge needs (24 bytes per (KV head, token) plus the table)
+    const size_t units = (size_t)pl.n_kv_heads * (size_t)pl.T;
+    size_t o = 0;
+    auto carve = [&](size_t bytes) { size_t at = o; o = align_up(o + bytes, 256); return at; };
+    pl.o_status = carve(256);
+    pl.o_reqs = carve(sizeof(Req) * (size_t)n_requests);
+    pl.o_row_ptr = carve(4 * (units + (size_t)pl.n_kv_heads * (size_t)n_requests));
+    pl.o_members = carve(4 * units);
+    pl.o_sort_a = carve(8 * units);
+    pl.o_sort_b = carve(8 * units);
+    pl.total = o;
+    if (pl.total > (size_t)LOOKM_NOALLOC_SCRATCH_BYTES) return LOOKM_ERR_WORKSPACE_TOO_SMALL;
+    void* scratch = nullptr;
+    LOOKM_TRY(noalloc_scratch_ptr(&scratch));
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    // begin_call clears the status word and rewrites the table; every list the kernels read is
+    // rewritten by the inversion kernel first, so nothing else of the last call's contents matters.
+    LOOKM_TRY(begin_call(pl, scratch, st));
+    return run_merge(pl, layout, k, v, kept_idx, evict_idx, assign, sim, varlen_output, out_k, out_v,
+                     scratch, st);
+}
+
+extern "C" int lookm_noalloc_status(void* cuda_stream) {
+    void* scratch = nullptr;
+    LOOKM_TRY(noalloc_scratch_ptr(&scratch));
+    return lookm_device_status(scratch, cuda_stream);
+}
