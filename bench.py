@@ -39,8 +39,19 @@ def measured_peaks():
     return {"hbm_gbs": 6650.0, "tflops": 1400.0, "source": "fallback"}
 
 
-def workload():
-    return synth.config2(seed=0)
+def workload(args=None):
+    """The 8K-prompt 7B-shape workload; --seq-len / --heads shrink it (profiling captures only)."""
+    w = synth.config2(seed=0)
+    if args is not None and (args.seq_len or args.heads):
+        L = args.seq_len or 8192
+        H = args.heads or 32
+        n_img = max(1, int(0.84 * L) // synth.IMAGE_TOKENS)
+        text = L - n_img * synth.IMAGE_TOKENS
+        seg = [text // (n_img + 1)] * (n_img + 1)
+        seg[-1] += text - sum(seg)
+        r = synth.Request(L, n_img, seg, int(0.2 * L), 32, 0, synth.interleave(n_img, seg))
+        w = synth.Workload("c2_shape_reduced_%dx%d" % (L, H), 2, 0, 32, H, H, 128, True, [r])
+    return w
 
 
 class ClockSampler(threading.Thread):
@@ -129,7 +140,7 @@ def run_reference(args):
     if rank != 0:
         return
     from oracle import lookm_oracle as orc
-    w = workload()
+    w = workload(args)
     cores = orc.default_threads()
     heads = list(range(min(cores, w.n_kv_heads)))
     qb, kb, vb = synth.layer_tensors(w, 0)
@@ -177,7 +188,7 @@ def run_ours(args):
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
     B.lib()
 
-    w = workload()
+    w = workload(args)
     req = w.requests[0]
     L, Hq, Hkv, budget, window = req.seq_len, w.n_q_heads, w.n_kv_heads, req.budget, req.window
     dev = lambda bits: torch.from_numpy(bits.view(np.int16)).cuda().view(torch.bfloat16)
@@ -329,6 +340,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=None)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--seq-len", type=int, default=0, help="reduced prompt length (profiling only)")
+    ap.add_argument("--heads", type=int, default=0, help="reduced head count (profiling only)")
     args = ap.parse_args()
     if args.steps is None:
         args.steps = 60 if args.impl == "ours" else 5
