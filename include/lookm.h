@@ -166,9 +166,9 @@ int lookm_workspace_layout(const lookm_layout* layout, int n_requests, const int
  * that loads the library holds until the process exits.  Inputs and outputs are still the
  * caller's, with the meaning and layouts of lookm_merge.
  *
- * Limits: the scratch needs 24 bytes per (KV head, token) plus a small table, so
- * n_kv_heads * total_tokens may be at most about 349,000 (e.g. 32 heads x 8192 tokens uses
- * 6.3 MB); larger batches return LOOKM_ERR_WORKSPACE_TOO_SMALL before anything is enqueued.
+ * Limits: the scratch needs 28 bytes per (KV head, token) plus a small table, so
+ * n_kv_heads * total_tokens may be at most about 299,000 (e.g. 32 heads x 8192 tokens uses
+ * 7.3 MB); larger batches return LOOKM_ERR_WORKSPACE_TOO_SMALL before anything is enqueued.
  * The call performs no cudaMalloc/cudaFree and calls no allocating routine.
  *
  * The first call on each device looks up the array's device address (cudaGetSymbolAddress, with

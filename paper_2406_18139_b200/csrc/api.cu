@@ -34,7 +34,7 @@ struct Plan {
     std::vector<int> out_len;               // caller order
     // workspace offsets (bytes)
     size_t o_status, o_reqs, o_lse, o_scores, o_rank, o_rnorm_all, o_kept, o_evict, o_kept_keys,
-        o_rnorm_kept, o_assign, o_sim, o_row_ptr, o_members, o_sort_a, o_sort_b, total;
+        o_rnorm_kept, o_assign, o_sim, o_row_ptr, o_members, o_member_w, o_sort_a, o_sort_b, total;
 };
 
 // Returns LOOKM_OK or the status describing the first bad argument.
@@ -125,6 +125,7 @@ int build_plan(Plan& pl, const lookm_layout* lay, int n_req, const int* cu_seqle
     pl.o_sim = carve(4 * Hkv * T);
     pl.o_row_ptr = carve(4 * (Hkv * T + Hkv * (size_t)n_req));
     pl.o_members = carve(4 * Hkv * T);
+    pl.o_member_w = carve(4 * Hkv * T);
     pl.o_sort_a = carve(8 * Hkv * T);
     pl.o_sort_b = carve(8 * Hkv * T);
     pl.total = o;
@@ -315,16 +316,16 @@ int run_merge(const Plan& pl, const lookm_layout* lay, const void* k, const void
               int varlen_output, void* out_k, void* out_v, void* ws, cudaStream_t st) {
     const Req* reqs = at<Req>(ws, pl.o_reqs);
     int* status = at<int>(ws, pl.o_status);
-    LOOKM_CUDA(launch_invert_assignment(assign, reqs, pl.n_req, pl.n_kv_heads,
+    LOOKM_CUDA(launch_invert_assignment(assign, evict_idx, sim, reqs, pl.n_req, pl.n_kv_heads,
                                         at<int>(ws, pl.o_row_ptr), at<int>(ws, pl.o_members),
-                                        at<unsigned>(ws, pl.o_sort_a), at<unsigned>(ws, pl.o_sort_b),
-                                        status, st));
+                                        at<float>(ws, pl.o_member_w), at<unsigned>(ws, pl.o_sort_a),
+                                        at<unsigned>(ws, pl.o_sort_b), status, st));
     ++g_launches;
     mark_stage(6, st);
     LOOKM_CUDA(launch_merge(k, v, lay->kv_stride_tok, lay->kv_stride_head, reqs, pl.n_req,
-                            pl.n_kv_heads, pl.T, pl.total_slots, kept_idx, evict_idx, sim,
-                            at<int>(ws, pl.o_row_ptr), at<int>(ws, pl.o_members), varlen_output,
-                            out_k, out_v, status, st));
+                            pl.n_kv_heads, pl.T, pl.total_slots, kept_idx,
+                            at<int>(ws, pl.o_row_ptr), at<int>(ws, pl.o_members),
+                            at<float>(ws, pl.o_member_w), varlen_output, out_k, out_v, status, st));
     ++g_launches;
     mark_stage(7, st);
     return LOOKM_OK;
@@ -600,7 +601,7 @@ extern "C" int lookm_merge_noalloc(const void* k, const void* v, const int* kept
     LOOKM_TRY(build_plan(pl, layout, n_requests, cu_seqlens_host, nullptr, budgets_host, nullptr,
                          merge_modes_host));
     LOOKM_TRY(check_layout_ptrs(layout, nullptr, k, v));
-    // compact carving of just what the merge needs (24 bytes per (KV head, token) plus the table)
+    // compact carving of just what the merge needs (28 bytes per (KV head, token) plus the table)
     const size_t units = (size_t)pl.n_kv_heads * (size_t)pl.T;
     size_t o = 0;
     auto carve = [&](size_t bytes) { size_t at = o; o = align_up(o + bytes, 256); return at; };
@@ -608,6 +609,7 @@ extern "C" int lookm_merge_noalloc(const void* k, const void* v, const int* kept
     pl.o_reqs = carve(sizeof(Req) * (size_t)n_requests);
     pl.o_row_ptr = carve(4 * (units + (size_t)pl.n_kv_heads * (size_t)n_requests));
     pl.o_members = carve(4 * units);
+    pl.o_member_w = carve(4 * units);
     pl.o_sort_a = carve(8 * units);
     pl.o_sort_b = carve(8 * units);
     pl.total = o;

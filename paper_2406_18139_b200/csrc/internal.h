@@ -81,15 +81,15 @@ constexpr int kReqChunk = 40;
 struct ReqChunk { Req r[kReqChunk]; };
 cudaError_t launch_write_table(const ReqChunk& chunk, int count, Req* dst, cudaStream_t stream);
 
-cudaError_t launch_invert_assignment(const int* assign, const Req* reqs, int n_req, int n_kv_heads,
-                                     int* row_ptr, int* members, unsigned* sort_a, unsigned* sort_b,
-                                     int* status, cudaStream_t stream);
+cudaError_t launch_invert_assignment(const int* assign, const int* evict_idx, const float* sim,
+                                     const Req* reqs, int n_req, int n_kv_heads, int* row_ptr,
+                                     int* member_pos, float* member_w, unsigned* sort_a,
+                                     unsigned* sort_b, int* status, cudaStream_t stream);
 
 cudaError_t launch_merge(const void* k, const void* v, long long stride_tok, long long stride_head,
                          const Req* reqs, int n_req, int n_kv_heads, long long T,
-                         long long total_kept_rows, const int* kept_idx, const int* evict_idx,
-                         const float* sim, const int* row_ptr, const int* members,
-                         int varlen_output, void* out_k, void* out_v, int* status,
-                         cudaStream_t stream);
+                         long long total_kept_rows, const int* kept_idx, const int* row_ptr,
+                         const int* member_pos, const float* member_w, int varlen_output,
+                         void* out_k, void* out_v, int* status, cudaStream_t stream);
 
 }  // namespace lookm

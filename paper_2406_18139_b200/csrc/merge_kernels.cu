@@ -123,7 +123,7 @@ argmax_rows_kernel(const float* __restrict__ sim_matrix, const Req* __restrict__
 // ---------------------------------------------------------------------------------------------
 // Inversion of the assignment: for each (request, head) a stable sort of the evicted ranks by
 // their kept slot gives, per kept row, its members in ascending position, as CSR
-// (row_ptr [B + 1 per (request, head)], members [E]).  One CTA per (request, head); stable LSD
+// (row_ptr [B + 1 per (request, head)], member positions and weights [E]).  One CTA per (request, head); stable LSD
 // radix sort with 8-bit digits: every warp owns a contiguous segment of the list, ranks equal
 // digits inside a 32-element step with match.any, and adds the counts of earlier steps and
 // earlier warps.  Keys are packed as (slot << 0) in one array and values in the other.
@@ -131,9 +131,11 @@ argmax_rows_kernel(const float* __restrict__ sim_matrix, const Req* __restrict__
 constexpr int kInvThreads = 1024;
 
 __global__ void __launch_bounds__(kInvThreads)
-invert_assignment_kernel(const int* __restrict__ assign, const Req* __restrict__ reqs,
-                         int n_kv_heads, int* __restrict__ row_ptr, int* __restrict__ members,
-                         unsigned* __restrict__ sort_a, unsigned* __restrict__ sort_b, int* status) {
+invert_assignment_kernel(const int* __restrict__ assign, const int* __restrict__ evict_idx,
+                         const float* __restrict__ sim, const Req* __restrict__ reqs,
+                         int n_kv_heads, int* __restrict__ row_ptr, int* __restrict__ member_pos,
+                         float* __restrict__ member_w, unsigned* __restrict__ sort_a,
+                         unsigned* __restrict__ sort_b, int* status) {
     __shared__ int cnt[32][256];                         // [warp][digit]
     __shared__ int digit_tot[256];
     const Req rq = reqs[blockIdx.y];
@@ -226,7 +228,11 @@ invert_assignment_kernel(const int* __restrict__ assign, const Req* __restrict__
     const unsigned* fin_v = fin_k + E;
     // members and the row boundaries: row_ptr[c] = first sorted index whose slot is >= c
     for (int i = threadIdx.x; i < E; i += kInvThreads) {
-        members[ev_base + i] = (int)fin_v[i];
+        const int e = (int)fin_v[i];
+        int pe = evict_idx[ev_base + e];
+        if (pe < 0 || pe >= rq.L) { atomicExch(status, (int)LOOKM_ERR_DEVICE_BAD_INDEX); pe = 0; }
+        member_pos[ev_base + i] = pe;                    // position of the i-th member in row order
+        member_w[ev_base + i] = sim[ev_base + e];        // its cosine with the kept row (Eq. 12 weight)
         const int cur = (int)fin_k[i];
         const int prev = i ? (int)fin_k[i - 1] : -1;
         for (int c = prev + 1; c <= cur; ++c) rp[c] = i;
@@ -235,8 +241,10 @@ invert_assignment_kernel(const int* __restrict__ assign, const Req* __restrict__
 }
 
 // ---------------------------------------------------------------------------------------------
-// Merge + compact: one warp per kept row (lanes 0-15 the K row, 16-31 the V row).  Each warp
-// gathers its kept row and its members, accumulates in fp32 in member order and rounds once.
+// Merge + compact: one warp per kept row (lanes 0-15 the K row, 16-31 the V row).  The lanes fetch
+// the row's metadata and up to 32 member positions / weights with one coalesced load each, then
+// the warp gathers the member rows eight at a time (eight 16-byte loads in flight per lane),
+// accumulates in fp32 in member order and rounds once.
 //   averaged : (x_c + sum x_e) / (n + 1)                       (Eq. 10)
 //   pivotal  : (x_c + 1/2 sum (x_e + x_c)) / (n + 1)           (Eq. 11)
 //   weighted : (x_c + sum sim_e x_e) / (n + 1)                 (Eq. 12)
@@ -244,83 +252,81 @@ invert_assignment_kernel(const int* __restrict__ assign, const Req* __restrict__
 // ---------------------------------------------------------------------------------------------
 constexpr int kMergeWarps = 8;
 
+__device__ __forceinline__ uint4 ld_stream(const __nv_bfloat16* p) {
+    uint4 r;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "l"(p));
+    return r;
+}
+
 __global__ void __launch_bounds__(kMergeWarps * 32)
 merge_kernel(const __nv_bfloat16* __restrict__ k, const __nv_bfloat16* __restrict__ v,
              long long stride_tok, long long stride_head, const Req* __restrict__ reqs, int n_req,
              int n_kv_heads, long long total_rows, const int* __restrict__ kept_idx,
-             const int* __restrict__ evict_idx, const float* __restrict__ sim,
-             const int* __restrict__ row_ptr, const int* __restrict__ members, int varlen_output,
+             const int* __restrict__ row_ptr, const int* __restrict__ member_pos,
+             const float* __restrict__ member_w, int varlen_output,
              __nv_bfloat16* __restrict__ out_k, __nv_bfloat16* __restrict__ out_v, int* status) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const long long g = (long long)blockIdx.x * kMergeWarps + warp;
     if (g >= total_rows) return;
-    int ri;
-    {
-        int lo = 0, hi = n_req - 1;
-        while (lo < hi) {
-            const int mid = (lo + hi + 1) >> 1;
-            if ((long long)reqs[mid].slot_begin <= g) lo = mid; else hi = mid - 1;
-        }
-        ri = lo;
-    }
-    const Req& rq = reqs[ri];
+    const Req& rq = find_req_by_slot(reqs, n_req, g);
     const long long u = g - rq.slot_begin;
-    const int h = (int)(u / rq.B), slot = (int)(u % rq.B);
+    const int B = rq.B, L = rq.L, mode = rq.mode;
+    const int h = (int)(u / B), slot = (int)(u % B);
     const int l16 = lane & 15;
-    const __nv_bfloat16* src = (lane < 16 ? k : v) + (long long)h * stride_head + l16 * 8;
-    const long long kept_base = rq.kept_off + (long long)h * rq.B;
+    const __nv_bfloat16* src = (lane < 16 ? k : v) + (long long)rq.tok_begin * stride_tok +
+                               (long long)h * stride_head + l16 * 8;
+    const long long kept_base = rq.kept_off + (long long)h * B;
     const long long ev_base = rq.ev_off + (long long)h * rq.E;
-    const int* rp = row_ptr + rq.rp_off + (long long)h * (rq.B + 1);
+    const int* rp = row_ptr + rq.rp_off + (long long)h * (B + 1);
 
-    int pos_c = kept_idx[kept_base + slot];
-    if (pos_c < 0 || pos_c >= rq.L) { if (lane == 0) atomicExch(status, (int)LOOKM_ERR_DEVICE_BAD_INDEX); pos_c = 0; }
-    const uint4 raw_c = *reinterpret_cast<const uint4*>(src + (rq.tok_begin + pos_c) * stride_tok);
-    const int m_begin = rp[slot], m_end = rp[slot + 1];
+    // lane 0: kept position, lane 1: first member, lane 2: one past the last member
+    int meta = 0;
+    if (lane == 0) meta = kept_idx[kept_base + slot];
+    else if (lane <= 2) meta = rp[slot + lane - 1];
+    int pos_c = __shfl_sync(0xffffffffu, meta, 0);
+    const int m_begin = __shfl_sync(0xffffffffu, meta, 1);
+    const int m_end = __shfl_sync(0xffffffffu, meta, 2);
+    if (pos_c < 0 || pos_c >= L) { if (lane == 0) atomicExch(status, (int)LOOKM_ERR_DEVICE_BAD_INDEX); pos_c = 0; }
+    const uint4 raw_c = ld_stream(src + (long long)pos_c * stride_tok);
     const int n = m_end - m_begin;
     uint4 result = raw_c;
     if (n > 0) {
-        const bool weighted = (rq.mode == LOOKM_MERGE_WEIGHTED);
+        const bool weighted = (mode == LOOKM_MERGE_WEIGHTED);
         float acc[8];
 #pragma unroll
         for (int i = 0; i < 8; ++i) acc[i] = 0.f;
-        int m = m_begin;
-        for (; m + 4 <= m_end; m += 4) {                 // four member rows in flight per lane
-            int e[4];
-            long long tok[4];
-            float w[4];
-            uint4 raw[4];
-#pragma unroll
-            for (int q = 0; q < 4; ++q) e[q] = members[ev_base + m + q];
-#pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                int pe = evict_idx[ev_base + e[q]];
-                if (pe < 0 || pe >= rq.L) { atomicExch(status, (int)LOOKM_ERR_DEVICE_BAD_INDEX); pe = 0; }
-                tok[q] = rq.tok_begin + pe;
-                w[q] = weighted ? sim[ev_base + e[q]] : 1.f;
+        for (int m0 = m_begin; m0 < m_end; m0 += 32) {
+            const int cnt = min(32, m_end - m0);
+            int my_pos = 0;
+            float my_w = 1.f;
+            if (lane < cnt) {
+                my_pos = member_pos[ev_base + m0 + lane];
+                if (weighted) my_w = member_w[ev_base + m0 + lane];
             }
+            for (int q0 = 0; q0 < cnt; q0 += 8) {
+                uint4 raw[8];
+                float w[8];
 #pragma unroll
-            for (int q = 0; q < 4; ++q) raw[q] = *reinterpret_cast<const uint4*>(src + tok[q] * stride_tok);
+                for (int q = 0; q < 8; ++q) {
+                    const int pe = __shfl_sync(0xffffffffu, my_pos, (q0 + q) & 31);
+                    w[q] = __shfl_sync(0xffffffffu, my_w, (q0 + q) & 31);
+                    if (q0 + q < cnt) raw[q] = ld_stream(src + (long long)pe * stride_tok);
+                    else { raw[q] = make_uint4(0u, 0u, 0u, 0u); w[q] = 0.f; }
+                }
 #pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                const Row8 x = unpack8(raw[q]);
+                for (int q = 0; q < 8; ++q) {
+                    const Row8 x = unpack8(raw[q]);
 #pragma unroll
-                for (int i = 0; i < 8; ++i) acc[i] = fmaf(w[q], x.v[i], acc[i]);
+                    for (int i = 0; i < 8; ++i) acc[i] = fmaf(w[q], x.v[i], acc[i]);
+                }
             }
-        }
-        for (; m < m_end; ++m) {
-            const int e = members[ev_base + m];
-            int pe = evict_idx[ev_base + e];
-            if (pe < 0 || pe >= rq.L) { atomicExch(status, (int)LOOKM_ERR_DEVICE_BAD_INDEX); pe = 0; }
-            const float w = weighted ? sim[ev_base + e] : 1.f;
-            const Row8 x = unpack8(*reinterpret_cast<const uint4*>(src + (rq.tok_begin + pe) * stride_tok));
-#pragma unroll
-            for (int i = 0; i < 8; ++i) acc[i] = fmaf(w, x.v[i], acc[i]);
         }
         const Row8 xc = unpack8(raw_c);
         const float inv = 1.0f / (float)(n + 1);
         // pivotal: each member contributes (x_e + x_c) / 2
-        const float wc = (rq.mode == LOOKM_MERGE_PIVOTAL) ? 1.f + 0.5f * (float)n : 1.f;
-        const float wm = (rq.mode == LOOKM_MERGE_PIVOTAL) ? 0.5f : 1.f;
+        const float wc = (mode == LOOKM_MERGE_PIVOTAL) ? 1.f + 0.5f * (float)n : 1.f;
+        const float wm = (mode == LOOKM_MERGE_PIVOTAL) ? 0.5f : 1.f;
         Row8 o;
 #pragma unroll
         for (int i = 0; i < 8; ++i) o.v[i] = fmaf(wc, xc.v[i], wm * acc[i]) * inv;
@@ -329,7 +335,7 @@ merge_kernel(const __nv_bfloat16* __restrict__ k, const __nv_bfloat16* __restric
     __nv_bfloat16* dst_base = lane < 16 ? out_k : out_v;
     long long row;
     if (varlen_output) row = ((long long)rq.out_begin + slot) * n_kv_heads + h;
-    else row = (long long)h * rq.B + slot;
+    else row = (long long)h * B + slot;
     *reinterpret_cast<uint4*>(dst_base + row * kHeadDim + l16 * 8) = result;
 }
 
@@ -395,27 +401,28 @@ cudaError_t launch_gather_kept(const void* k, long long stride_tok, long long st
     return cudaGetLastError();
 }
 
-cudaError_t launch_invert_assignment(const int* assign, const Req* reqs, int n_req, int n_kv_heads,
-                                     int* row_ptr, int* members, unsigned* sort_a, unsigned* sort_b,
-                                     int* status, cudaStream_t stream) {
+cudaError_t launch_invert_assignment(const int* assign, const int* evict_idx, const float* sim,
+                                     const Req* reqs, int n_req, int n_kv_heads, int* row_ptr,
+                                     int* member_pos, float* member_w, unsigned* sort_a,
+                                     unsigned* sort_b, int* status, cudaStream_t stream) {
     dim3 grid(n_kv_heads, n_req);
-    invert_assignment_kernel<<<grid, kInvThreads, 0, stream>>>(assign, reqs, n_kv_heads, row_ptr,
-                                                               members, sort_a, sort_b, status);
+    invert_assignment_kernel<<<grid, kInvThreads, 0, stream>>>(assign, evict_idx, sim, reqs, n_kv_heads,
+                                                               row_ptr, member_pos, member_w, sort_a,
+                                                               sort_b, status);
     return cudaGetLastError();
 }
 
 cudaError_t launch_merge(const void* k, const void* v, long long stride_tok, long long stride_head,
                          const Req* reqs, int n_req, int n_kv_heads, long long T,
-                         long long total_kept_rows, const int* kept_idx, const int* evict_idx,
-                         const float* sim, const int* row_ptr, const int* members,
-                         int varlen_output, void* out_k, void* out_v, int* status,
-                         cudaStream_t stream) {
+                         long long total_kept_rows, const int* kept_idx, const int* row_ptr,
+                         const int* member_pos, const float* member_w, int varlen_output,
+                         void* out_k, void* out_v, int* status, cudaStream_t stream) {
     (void)T;
     if (total_kept_rows <= 0) return cudaSuccess;
     const long long blocks = (total_kept_rows + kMergeWarps - 1) / kMergeWarps;
     merge_kernel<<<(unsigned)blocks, kMergeWarps * 32, 0, stream>>>(
         (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, stride_tok, stride_head, reqs, n_req,
-        n_kv_heads, total_kept_rows, kept_idx, evict_idx, sim, row_ptr, members, varlen_output,
+        n_kv_heads, total_kept_rows, kept_idx, row_ptr, member_pos, member_w, varlen_output,
         (__nv_bfloat16*)out_k, (__nv_bfloat16*)out_v, status);
     return cudaGetLastError();
 }

@@ -5,8 +5,9 @@
 //   - a work item owns one STATIONARY 128-row tile (the A operand, rows on the 128 TMEM lanes)
 //     and streams a sequence of 128-row tiles (the B operand) against it;
 //   - warp 0 (one thread) issues the TMA loads, warp 1 (one thread) issues tcgen05.mma into one of
-//     four 128-column TMEM accumulators, and two groups of four warps read the accumulators with
-//     tcgen05.ld and run the epilogue; group w takes the tiles whose running index is w mod 2;
+//     four 128-column TMEM accumulators, and four groups of four warps read the accumulators with
+//     tcgen05.ld and run the epilogue; group w owns accumulator w and takes the tiles whose running
+//     index is w mod 4, so each SM sub-partition always has four epilogue warps to switch between;
 //   - each epilogue thread owns one row of the stationary tile, so every reduction over the
 //     streamed axis (row maximum and sum, column-sum of probabilities for one key, running
 //     arg-max) stays in that thread's registers; the two groups are combined through shared
@@ -31,7 +32,8 @@ namespace {
 
 constexpr int kStages = 4;                       // ring of streamed tiles
 constexpr int kAccum = 4;                        // TMEM accumulators (128 fp32 columns each)
-constexpr int kThreads = 320;                    // producer warp, MMA warp, 2 x 4 epilogue warps
+constexpr int kGroups = 4;                       // epilogue groups (one per TMEM accumulator)
+constexpr int kThreads = 64 + kGroups * 128;     // producer warp, MMA warp, 4 x 4 epilogue warps
 constexpr int kHalfBytes = kTile * 64 * 2;       // one TMA box: 128 rows x 64 bf16 (128 B rows)
 constexpr int kTileBytes = 2 * kHalfBytes;       // 128 x 128 bf16
 constexpr float kLog2e = 1.4426950408889634f;
@@ -40,8 +42,8 @@ constexpr float kLn2 = 0.6931471805599453f;
 struct __align__(1024) Shared {
     uint8_t a[2][kTileBytes];                    // stationary tiles (double-buffered across items)
     uint8_t b[kStages][kTileBytes];              // streamed tiles
-    float side[2][2][kTile];                     // per epilogue group, double-buffered column data
-    float comb[2][4][kTile];                     // group-1 partial results, double-buffered
+    float side[kGroups][2][kTile];               // per epilogue group, double-buffered column data
+    float comb[2][kGroups - 1][2][kTile];        // partial results of groups 1.., double-buffered
     unsigned long long a_full[2], a_empty[2];
     unsigned long long b_full[kStages], b_empty[kStages];
     unsigned long long t_full[kAccum], t_empty[kAccum];
@@ -222,7 +224,7 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         }
     } else {
         // ------------------------------------------------------------ epilogue --------------
-        const int wg = (warp - 2) >> 2;                      // epilogue group 0 / 1
+        const int wg = (warp - 2) >> 2;                      // epilogue group 0..3
         const int quarter = warp & 3;                        // TMEM lane quarter this warp may read
         const int row = quarter * 32 + lane;                 // row of the stationary tile
         const uint32_t lane_addr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
@@ -241,8 +243,8 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
             int best_slot = 0x7fffffff;
 
             for (int t = 0; t < it.nt; ++t, ++gb) {
-                if ((int)(gb & 1u) != wg) continue;
-                const int buf = gb % kAccum;
+                if ((int)(gb % kGroups) != wg) continue;
+                const int buf = wg;
                 float* side = sh.side[wg][lt & 1];
                 bool diag = false;                           // tile crosses the causal diagonal
                 int col_limit = kTile;                       // match: valid kept slots in the tile
@@ -354,32 +356,41 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                 if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&sh.t_empty[buf]));
             }
 
-            // ---- combine the two groups and write this item's results ------------------------
-            float* cb0 = sh.comb[n & 1][0];
-            float* cb1 = sh.comb[n & 1][1];
-            if (wg == 1) {
+            // ---- combine the four groups and write this item's results -----------------------
+            if (wg > 0) {
+                float* cb0 = sh.comb[n & 1][wg - 1][0];
+                float* cb1 = sh.comb[n & 1][wg - 1][1];
                 if (KIND == kSweep1) { cb0[row] = m_run; cb1[row] = l_run; }
                 else if (KIND == kSweep2) { cb0[row] = (acc0 + acc1) + (acc2 + acc3); }
                 else { cb0[row] = best; cb1[row] = __int_as_float(best_slot); }
             }
-            ptx::named_barrier_sync(3, 256);
+            ptx::named_barrier_sync(1 + kGroups, kGroups * 128);
             if (wg == 0 && pos < it.L && !*abort_flag) {
                 if (KIND == kSweep1) {
-                    const float m1 = cb0[row], l1 = cb1[row];
-                    const float m = fmaxf(m_run, m1);
-                    const float l = l_run * ptx::ex2((m_run - m) * c2) + l1 * ptx::ex2((m1 - m) * c2);
+                    float m = m_run;
+#pragma unroll
+                    for (int g = 0; g < kGroups - 1; ++g) m = fmaxf(m, sh.comb[n & 1][g][0][row]);
+                    float l = l_run * ptx::ex2((m_run - m) * c2);
+#pragma unroll
+                    for (int g = 0; g < kGroups - 1; ++g)
+                        l += sh.comb[n & 1][g][1][row] * ptx::ex2((sh.comb[n & 1][g][0][row] - m) * c2);
                     // natural-log log-sum-exp of the scaled logits
                     p.lse[(long long)it.head * p.T + it.tok_begin + pos] = (m * c2 + ptx::lg2(l)) * kLn2;
                 } else if (KIND == kSweep2) {
-                    p.scores[(long long)it.head * p.T + it.tok_begin + pos] =
-                        ((acc0 + acc1) + (acc2 + acc3)) + cb0[row];
+                    float a = (acc0 + acc1) + (acc2 + acc3);
+#pragma unroll
+                    for (int g = 0; g < kGroups - 1; ++g) a += sh.comb[n & 1][g][0][row];
+                    p.scores[(long long)it.head * p.T + it.tok_begin + pos] = a;
                 } else {
                     const long long g = (long long)it.head * p.T + it.tok_begin + pos;
                     const int e = p.rank[g];
                     if (e >= 0) {
-                        const float b1 = cb0[row];
-                        const int s1 = __float_as_int(cb1[row]);
-                        if (b1 > best || (b1 == best && s1 < best_slot)) { best = b1; best_slot = s1; }
+#pragma unroll
+                        for (int gi = 0; gi < kGroups - 1; ++gi) {
+                            const float b1 = sh.comb[n & 1][gi][0][row];
+                            const int s1 = __float_as_int(sh.comb[n & 1][gi][1][row]);
+                            if (b1 > best || (b1 == best && s1 < best_slot)) { best = b1; best_slot = s1; }
+                        }
                         p.assign[it.ev0 + e] = best_slot;
                         p.sim[it.ev0 + e] = best * p.rnorm_all[g];
                     }
