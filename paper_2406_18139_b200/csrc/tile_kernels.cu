@@ -47,6 +47,7 @@ struct __align__(1024) Shared {
     unsigned long long a_full[2], a_empty[2];
     unsigned long long b_full[kStages], b_empty[kStages];
     unsigned long long t_full[kAccum], t_empty[kAccum];
+    unsigned long long mma_done;                 // every MMA of this CTA has completed
     uint32_t tmem_base;
     int abort_flag;
 };
@@ -120,6 +121,7 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
             ptx::mbar_init(ptx::smem_u32(&sh.t_full[i]), 1);
             ptx::mbar_init(ptx::smem_u32(&sh.t_empty[i]), 4);   // one arrival per epilogue warp
         }
+        ptx::mbar_init(ptx::smem_u32(&sh.mma_done), 1);
         sh.abort_flag = 0;
         ptx::fence_mbar_init();
     }
@@ -221,6 +223,11 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                     if (t == it.nt - 1) ptx::umma_commit(ptx::smem_u32(&sh.a_empty[ab]));
                 }
             }
+            // Nothing may release TMEM or leave the kernel while an MMA is still running, also
+            // after an abort: wait for all of them (own time limit, the abort flag is ignored).
+            int ignore = 0;
+            ptx::umma_commit(ptx::smem_u32(&sh.mma_done));
+            ptx::mbar_wait(ptx::smem_u32(&sh.mma_done), 0, &ignore, 1000000000ull);
         }
     } else {
         // ------------------------------------------------------------ epilogue --------------

@@ -17,6 +17,7 @@ are redundant, which is the structure the method's eviction and merging exploit.
 """
 from __future__ import annotations
 
+import os
 from dataclasses import dataclass, field
 from typing import List, Sequence, Tuple
 
@@ -67,28 +68,63 @@ def uniform_int(key: np.uint64, n: int, lo: int, hi: int, offset: int = 0) -> np
     return (uniform_u64(key, n, offset) >> np.uint64(11)) % span + np.uint64(lo)
 
 
+def _normal_chunk(key: np.uint64, s: int, m: int, out: np.ndarray) -> None:
+    x = uniform_u64(key, m, s)
+    u1 = ((x >> np.uint64(32)).astype(np.float64) + 0.5) * (1.0 / 4294967296.0)
+    u2 = ((x & np.uint64(0xFFFFFFFF)).astype(np.float64) + 0.5) * (1.0 / 4294967296.0)
+    r = np.sqrt(-2.0 * np.log(u1))
+    t = (2.0 * np.pi) * u2
+    out[2 * s:2 * (s + m):2] = r * np.cos(t)
+    out[2 * s + 1:2 * (s + m):2] = r * np.sin(t)
+
+
 def normal(key: np.uint64, n: int) -> np.ndarray:
-    """n standard normal draws (float64) from stream `key` by Box-Muller."""
+    """n standard normal draws (float64) from stream `key` by Box-Muller.
+
+    Counter c yields draws 2c and 2c+1, so the result does not depend on how the work is chunked;
+    large requests are spread over a thread pool (numpy releases the GIL inside each chunk).
+    """
     half = (n + 1) // 2
     out = np.empty(2 * half, dtype=np.float64)
-    chunk = 1 << 21
-    for s in range(0, half, chunk):
-        m = min(chunk, half - s)
-        x = uniform_u64(key, m, s)
-        u1 = ((x >> np.uint64(32)).astype(np.float64) + 0.5) * (1.0 / 4294967296.0)
-        u2 = ((x & np.uint64(0xFFFFFFFF)).astype(np.float64) + 0.5) * (1.0 / 4294967296.0)
-        r = np.sqrt(-2.0 * np.log(u1))
-        t = (2.0 * np.pi) * u2
-        out[2 * s:2 * (s + m):2] = r * np.cos(t)
-        out[2 * s + 1:2 * (s + m):2] = r * np.sin(t)
+    chunk = 1 << 20
+    starts = list(range(0, half, chunk))
+    if len(starts) <= 2:
+        for s in starts:
+            _normal_chunk(key, s, min(chunk, half - s), out)
+    else:
+        from concurrent.futures import ThreadPoolExecutor
+        with ThreadPoolExecutor(max_workers=_workers()) as ex:
+            list(ex.map(lambda s: _normal_chunk(key, s, min(chunk, half - s), out), starts))
     return out[:n]
+
+
+def _workers() -> int:
+    try:
+        return max(1, min(32, len(os.sched_getaffinity(0))))
+    except AttributeError:
+        return max(1, min(32, os.cpu_count() or 1))
 
 
 def f32_to_bf16_bits(x: np.ndarray) -> np.ndarray:
     """Round float32 to bf16 (nearest, ties to even); returns the uint16 bit patterns."""
-    b = np.ascontiguousarray(x, dtype=np.float32).view(np.uint32)
-    r = (b + np.uint32(0x7FFF) + ((b >> np.uint32(16)) & np.uint32(1))) >> np.uint32(16)
-    return r.astype(np.uint16)
+    x = np.ascontiguousarray(x, dtype=np.float32)
+    flat = x.reshape(-1).view(np.uint32)
+    out = np.empty(flat.shape[0], dtype=np.uint16)
+
+    def piece(s):
+        b = flat[s:s + (1 << 22)]
+        out[s:s + (1 << 22)] = ((b + np.uint32(0x7FFF) + ((b >> np.uint32(16)) & np.uint32(1)))
+                                >> np.uint32(16)).astype(np.uint16)
+
+    starts = list(range(0, flat.shape[0], 1 << 22))
+    if len(starts) <= 1:
+        for s0 in starts:
+            piece(s0)
+    else:
+        from concurrent.futures import ThreadPoolExecutor
+        with ThreadPoolExecutor(max_workers=_workers()) as ex:
+            list(ex.map(piece, starts))
+    return out.reshape(x.shape)
 
 
 def bf16_to_f32(bits: np.ndarray) -> np.ndarray:
