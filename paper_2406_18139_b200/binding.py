@@ -13,7 +13,7 @@ import os
 from typing import Optional, Sequence
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "liblookm.so")
+LIB_PATH = os.environ.get("LOOKM_LIB", os.path.join(_HERE, "liblookm.so"))   # LOOKM_LIB: another build of the same library
 _lib = None
 
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE_TOO_SMALL, ERR_CUDA, ERR_DEVICE_TIMEOUT, \

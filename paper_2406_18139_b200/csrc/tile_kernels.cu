@@ -2,22 +2,29 @@
 // the cosine matching with fused row argmax (Eq. 9).
 //
 // All three are the same persistent, warp-specialised pipeline over 128 x 128 x 128 bf16 tiles:
-//   - a work item owns one STATIONARY 128-row tile (the A operand, rows on the 128 TMEM lanes)
-//     and streams a sequence of 128-row tiles (the B operand) against it;
-//   - warp 0 (one thread) issues the TMA loads, warp 1 (one thread) issues tcgen05.mma into one of
-//     four 128-column TMEM accumulators, and four groups of four warps read the accumulators with
-//     tcgen05.ld and run the epilogue; group w owns accumulator w and takes the tiles whose running
-//     index is w mod 4, so each SM sub-partition always has four epilogue warps to switch between;
-//   - each epilogue thread owns one row of the stationary tile, so every reduction over the
+//   - a work item owns TWO stationary 128-row tiles (256 consecutive rows of the A operand; the
+//     rows of each tile sit on the 128 TMEM lanes) and streams a sequence of 128-row tiles (the B
+//     operand) against them, so every streamed tile feeds two MMAs (16 tcgen05.mma of
+//     128 x 128 x 16) and the L2 -> shared-memory traffic per flop is halved;
+//   - warp 0 (one thread) issues the TMA loads; warps 1 and 18 (one thread each) issue the MMAs
+//     of the even and of the odd streamed tiles into four 128-column TMEM accumulators (streamed
+//     tile parity x stationary tile).  Measured on B200: a thread that waits on an mbarrier,
+//     fences and commits between every 8 MMAs keeps the tensor pipe only about half busy (512
+//     clocks per 8 MMAs alone, about 900 with one wait and two commits in between), so the
+//     synchronisation is done once per streamed tile and two threads alternate;
+//   - four groups of four warps read the accumulators with tcgen05.ld and run the epilogue: group
+//     g owns accumulator g, i.e. stationary tile (g & 1) under the streamed tiles of parity
+//     (g >> 1);
+//   - each epilogue thread owns one row of its stationary tile, so every reduction over the
 //     streamed axis (row maximum and sum, column-sum of probabilities for one key, running
-//     arg-max) stays in that thread's registers; the two groups are combined through shared
-//     memory once per item.  No L x L matrix is ever stored.
+//     arg-max) stays in that thread's registers; the two groups that share a stationary tile are
+//     combined through shared memory once per item.  No L x L matrix is ever stored.
 //
-//   sweep 1: A = 128 queries of one query head, B = key tiles 0..diagonal.  Online softmax
+//   sweep 1: A = 256 queries of one query head, B = key tiles 0..diagonal.  Online softmax
 //            statistics per query row  ->  lse[i] = log sum_{j<=i} exp(s_ij).
-//   sweep 2: A = 128 keys of one KV head, B = query tiles diagonal..last of every query head in
+//   sweep 2: A = 256 keys of one KV head, B = query tiles diagonal..last of every query head in
 //            the group.  Thread of key j accumulates sum_i exp(s_ij - lse_i)  ->  A_s[j].
-//   match  : A = 128 key rows (all positions; kept rows are ignored at the end), B = tiles of the
+//   match  : A = 256 key rows (all positions; kept rows are ignored at the end), B = tiles of the
 //            compacted kept keys.  Thread keeps the largest s_ij / |k_j| and its slot.
 //
 // Work items are laid out heaviest first and dealt to the CTAs in serpentine order; every role
@@ -31,64 +38,81 @@ namespace lookm {
 namespace {
 
 constexpr int kStages = 4;                       // ring of streamed tiles
-constexpr int kAccum = 4;                        // TMEM accumulators (128 fp32 columns each)
 constexpr int kGroups = 4;                       // epilogue groups (one per TMEM accumulator)
-constexpr int kThreads = 64 + kGroups * 128;     // producer warp, MMA warp, 4 x 4 epilogue warps
+constexpr int kMmaWarp1 = 2 + kGroups * 4;       // the second MMA-issuing warp
+constexpr int kThreads = (kMmaWarp1 + 1) * 32;   // producer, MMA (even), 4 x 4 epilogue, MMA (odd)
 constexpr int kHalfBytes = kTile * 64 * 2;       // one TMA box: 128 rows x 64 bf16 (128 B rows)
 constexpr int kTileBytes = 2 * kHalfBytes;       // 128 x 128 bf16
+constexpr int kReqCache = 32;                    // request-table entries cached in shared memory
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 
 struct __align__(1024) Shared {
-    uint8_t a[2][kTileBytes];                    // stationary tiles (double-buffered across items)
+    uint8_t a[2][kTileBytes];                    // the item's two stationary tiles
     uint8_t b[kStages][kTileBytes];              // streamed tiles
     float side[kGroups][2][kTile];               // per epilogue group, double-buffered column data
-    float comb[2][kGroups - 1][2][kTile];        // partial results of groups 1.., double-buffered
-    unsigned long long a_full[2], a_empty[2];
+    float comb[2][2][2][kTile];                  // [item parity][stationary tile][array][row]
+    Req reqs[kReqCache];
+    unsigned long long a_full, a_empty;
     unsigned long long b_full[kStages], b_empty[kStages];
-    unsigned long long t_full[kAccum], t_empty[kAccum];
+    unsigned long long t_full[2], t_empty[2];    // per streamed-tile parity (two accumulators each)
     unsigned long long mma_done;                 // every MMA of this CTA has completed
     uint32_t tmem_base;
     int abort_flag;
 };
+static_assert(sizeof(Shared) + 1024 <= 232448, "shared storage exceeds what one CTA may use");
 
 struct Item {
-    int tok_begin, L, B, blk, head, nt;
+    int tok_begin, L, B, bp, head, nt, nblk;
     long long kept_row0;      // match: first row of this (request, head) in the kept-key matrix
     long long ev0;            // match: start of its evicted list
 };
 
+// Work item `item` of stage KIND.  An item covers block pair bp = stationary blocks 2bp, 2bp+1.
 template <int KIND>
-__device__ __forceinline__ Item decode_item(const TileParams& p, int item) {
+__device__ __forceinline__ Item decode_item(const TileParams& p, const Req* tbl, int item) {
     int lo = 0, hi = p.n_req - 1;
     while (lo < hi) {
         const int mid = (lo + hi + 1) >> 1;
-        if (p.reqs[mid].item_begin[KIND] <= item) lo = mid; else hi = mid - 1;
+        if (tbl[mid].item_begin[KIND] <= item) lo = mid; else hi = mid - 1;
     }
-    const Req& rq = p.reqs[lo];
+    const Req& rq = tbl[lo];
     const int u = item - rq.item_begin[KIND];
+    const int npair = (rq.nblk + 1) >> 1;
     Item it;
     it.tok_begin = rq.tok_begin;
     it.L = rq.L;
     it.B = rq.B;
+    it.nblk = rq.nblk;
     it.kept_row0 = 0;
     it.ev0 = 0;
-    if (KIND == kSweep1) {                       // heaviest first: last query block first
-        it.blk = rq.nblk - 1 - u / p.n_q_heads;
+    if (KIND == kSweep1) {                       // heaviest first: last query blocks first
+        it.bp = npair - 1 - u / p.n_q_heads;
         it.head = u % p.n_q_heads;
-        it.nt = it.blk + 1;
-    } else if (KIND == kSweep2) {                // heaviest first: first key block first
-        it.blk = u / p.n_kv_heads;
+        it.nt = min(rq.nblk, 2 * it.bp + 2);     // key tiles 0 .. the later block's diagonal
+    } else if (KIND == kSweep2) {                // heaviest first: first key blocks first
+        it.bp = u / p.n_kv_heads;
         it.head = u % p.n_kv_heads;
-        it.nt = (rq.nblk - it.blk) * p.group;
+        it.nt = (rq.nblk - 2 * it.bp) * p.group;
     } else {
-        it.blk = u / p.n_kv_heads;
+        it.bp = u / p.n_kv_heads;
         it.head = u % p.n_kv_heads;
         it.nt = (rq.B + kTile - 1) / kTile;
         it.kept_row0 = rq.kept_off + (long long)it.head * rq.B;
         it.ev0 = rq.ev_off + (long long)it.head * rq.E;
     }
     return it;
+}
+
+// Does streamed tile t contribute anything to stationary tile `sub` of the item?  (The block may
+// lie past the prompt end, or the whole tile may be on the wrong side of the causal diagonal.)
+template <int KIND>
+__device__ __forceinline__ bool unit_active(const TileParams& p, const Item& it, int t, int sub) {
+    const int blk = 2 * it.bp + sub;
+    if (blk >= it.nblk) return false;
+    if (KIND == kSweep1) return t <= blk;                          // keys up to the query block
+    if (KIND == kSweep2) return 2 * it.bp + t / p.group >= blk;    // queries from the key block on
+    return true;
 }
 
 // Serpentine deal of the item list: round k hands items k*G .. k*G+G-1 to the CTAs in forward
@@ -109,21 +133,25 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     volatile int* abort_flag = &sh.abort_flag;
 
     if (threadIdx.x == 0) {
-        for (int i = 0; i < 2; ++i) {
-            ptx::mbar_init(ptx::smem_u32(&sh.a_full[i]), 1);
-            ptx::mbar_init(ptx::smem_u32(&sh.a_empty[i]), 1);
-        }
+        ptx::mbar_init(ptx::smem_u32(&sh.a_full), 1);
+        ptx::mbar_init(ptx::smem_u32(&sh.a_empty), 2);         // one arrival per MMA thread
         for (int i = 0; i < kStages; ++i) {
             ptx::mbar_init(ptx::smem_u32(&sh.b_full[i]), 1);
             ptx::mbar_init(ptx::smem_u32(&sh.b_empty[i]), 1);
         }
-        for (int i = 0; i < kAccum; ++i) {
+        for (int i = 0; i < 2; ++i) {
             ptx::mbar_init(ptx::smem_u32(&sh.t_full[i]), 1);
-            ptx::mbar_init(ptx::smem_u32(&sh.t_empty[i]), 4);   // one arrival per epilogue warp
+            ptx::mbar_init(ptx::smem_u32(&sh.t_empty[i]), 8);  // one arrival per warp of two groups
         }
-        ptx::mbar_init(ptx::smem_u32(&sh.mma_done), 1);
+        ptx::mbar_init(ptx::smem_u32(&sh.mma_done), 2);
         sh.abort_flag = 0;
         ptx::fence_mbar_init();
+    }
+    const Req* tbl = p.reqs;
+    if (p.n_req <= kReqCache) {                  // the table is read once per item by every role
+        for (int i = threadIdx.x; i < p.n_req * (int)(sizeof(Req) / 4); i += kThreads)
+            reinterpret_cast<int*>(sh.reqs)[i] = reinterpret_cast<const int*>(p.reqs)[i];
+        tbl = sh.reqs;
     }
     if (warp == 0) {
         ptx::tmem_alloc(ptx::smem_u32(&sh.tmem_base), 512);
@@ -145,16 +173,18 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
             for (int round = 0;; ++round, ++n) {
                 const int item = item_of_round(round, blockIdx.x, n_cta);
                 if (item >= p.n_items) { if (round * n_cta >= p.n_items) break; --n; continue; }
-                const Item it = decode_item<KIND>(p, item);
-                const int ab = n & 1;
-                ptx::mbar_wait(ptx::smem_u32(&sh.a_empty[ab]), ((n >> 1) & 1) ^ 1, abort_flag);
-                const uint32_t abar = ptx::smem_u32(&sh.a_full[ab]);
-                ptx::mbar_arrive_expect_tx(abar, kTileBytes);
-                const uint32_t adst = ptx::smem_u32(&sh.a[ab][0]);
-                const int a_head = it.head;
-                const int a_row = it.tok_begin + it.blk * kTile;
-                ptx::tma_load_3d(adst, &map_a, 0, a_head, a_row, abar);
-                ptx::tma_load_3d(adst + kHalfBytes, &map_a, 64, a_head, a_row, abar);
+                const Item it = decode_item<KIND>(p, tbl, item);
+                // both stationary tiles; rows past the tensor end read as zero
+                ptx::mbar_wait(ptx::smem_u32(&sh.a_empty), (n & 1) ^ 1, abort_flag);
+                const uint32_t abar = ptx::smem_u32(&sh.a_full);
+                ptx::mbar_arrive_expect_tx(abar, 2 * kTileBytes);
+#pragma unroll
+                for (int sub = 0; sub < 2; ++sub) {
+                    const uint32_t adst = ptx::smem_u32(&sh.a[sub][0]);
+                    const int a_row = it.tok_begin + (2 * it.bp + sub) * kTile;
+                    ptx::tma_load_3d(adst, &map_a, 0, it.head, a_row, abar);
+                    ptx::tma_load_3d(adst + kHalfBytes, &map_a, 64, it.head, a_row, abar);
+                }
                 for (int t = 0; t < it.nt; ++t, ++gb) {
                     const int s = gb % kStages;
                     ptx::mbar_wait(ptx::smem_u32(&sh.b_empty[s]), ((gb / kStages) & 1) ^ 1, abort_flag);
@@ -167,7 +197,7 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                         ptx::tma_load_3d(bdst, &map_b, 0, h, row, bbar);
                         ptx::tma_load_3d(bdst + kHalfBytes, &map_b, 64, h, row, bbar);
                     } else if (KIND == kSweep2) {
-                        const int row = it.tok_begin + (it.blk + t / p.group) * kTile;
+                        const int row = it.tok_begin + (2 * it.bp + t / p.group) * kTile;
                         const int h = it.head * p.group + t % p.group;
                         ptx::tma_load_3d(bdst, &map_b, 0, h, row, bbar);
                         ptx::tma_load_3d(bdst + kHalfBytes, &map_b, 64, h, row, bbar);
@@ -178,7 +208,7 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                     }
                 }
             }
-            // Every load issued above is consumed by the MMA warp before it finishes, except
+            // Every load issued above is consumed by an MMA thread before it finishes, except
             // after an abort: then wait (bounded, ignoring the flag) until the last ring of
             // loads has landed so that no copy is in flight when the CTA exits.
             if (*abort_flag) {
@@ -189,38 +219,49 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                                    200000000ull);
             }
         }
-    } else if (warp == 1) {
-        // ------------------------------------------------------------ MMA issuer ------------
+    } else if (warp == 1 || warp == kMmaWarp1) {
+        // ------------------------------------------------------------ MMA issuers -----------
         if (lane == 0) {
             constexpr uint32_t idesc = ptx::umma_idesc_bf16(kTile, kTile);
+            const uint32_t mine = (warp == 1) ? 0u : 1u;     // parity of the streamed tiles I issue
             uint32_t gb = 0;
             int n = 0;
             for (int round = 0;; ++round, ++n) {
                 const int item = item_of_round(round, blockIdx.x, n_cta);
                 if (item >= p.n_items) { if (round * n_cta >= p.n_items) break; --n; continue; }
-                const Item it = decode_item<KIND>(p, item);
-                const int ab = n & 1;
-                ptx::mbar_wait(ptx::smem_u32(&sh.a_full[ab]), (n >> 1) & 1, abort_flag);
-                const uint32_t a_addr = ptx::smem_u32(&sh.a[ab][0]);
+                const Item it = decode_item<KIND>(p, tbl, item);
+                // my last streamed tile of this item (-1: its only tile has the other parity)
+                int last_t = it.nt - 1;
+                if (((gb + last_t) & 1u) != mine) --last_t;
+                // Always wait for this item's stationary tiles: their arrival also proves that the
+                // previous item's a_empty phase is over, so the arrival below cannot fall into it.
+                ptx::mbar_wait(ptx::smem_u32(&sh.a_full), n & 1, abort_flag);
+                if (last_t < 0) ptx::mbar_arrive(ptx::smem_u32(&sh.a_empty));
                 for (int t = 0; t < it.nt; ++t, ++gb) {
+                    if ((gb & 1u) != mine) continue;
                     const int s = gb % kStages;
-                    const int buf = gb % kAccum;
                     ptx::mbar_wait(ptx::smem_u32(&sh.b_full[s]), (gb / kStages) & 1, abort_flag);
-                    ptx::mbar_wait(ptx::smem_u32(&sh.t_empty[buf]), ((gb / kAccum) & 1) ^ 1, abort_flag);
+                    ptx::mbar_wait(ptx::smem_u32(&sh.t_empty[mine]), ((gb >> 1) & 1) ^ 1, abort_flag);
                     ptx::tc_fence_after_sync();
                     const uint32_t b_addr = ptx::smem_u32(&sh.b[s][0]);
-                    const uint32_t d_tmem = tmem_base + buf * kTile;
 #pragma unroll
-                    for (int kk = 0; kk < 8; ++kk) {
-                        // 16 bf16 (32 bytes) per MMA along the 128-byte swizzled row; the second
-                        // half of head_dim lives in the second TMA box.
-                        const uint32_t off = (kk >> 2) * kHalfBytes + (kk & 3) * 32;
-                        ptx::umma_bf16(d_tmem, ptx::umma_desc_sw128(a_addr + off),
-                                       ptx::umma_desc_sw128(b_addr + off), idesc, kk > 0);
+                    for (int sub = 0; sub < 2; ++sub) {
+                        if (unit_active<KIND>(p, it, t, sub)) {
+                            const uint32_t a_addr = ptx::smem_u32(&sh.a[sub][0]);
+                            const uint32_t d_tmem = tmem_base + (2 * mine + sub) * kTile;
+#pragma unroll
+                            for (int kk = 0; kk < 8; ++kk) {
+                                // 16 bf16 (32 bytes) per MMA along the 128-byte swizzled row; the
+                                // second half of head_dim lives in the second TMA box.
+                                const uint32_t off = (kk >> 2) * kHalfBytes + (kk & 3) * 32;
+                                ptx::umma_bf16(d_tmem, ptx::umma_desc_sw128(a_addr + off),
+                                               ptx::umma_desc_sw128(b_addr + off), idesc, kk > 0);
+                            }
+                        }
                     }
+                    ptx::umma_commit(ptx::smem_u32(&sh.t_full[mine]));
                     ptx::umma_commit(ptx::smem_u32(&sh.b_empty[s]));
-                    ptx::umma_commit(ptx::smem_u32(&sh.t_full[buf]));
-                    if (t == it.nt - 1) ptx::umma_commit(ptx::smem_u32(&sh.a_empty[ab]));
+                    if (t == last_t) ptx::umma_commit(ptx::smem_u32(&sh.a_empty));
                 }
             }
             // Nothing may release TMEM or leave the kernel while an MMA is still running, also
@@ -231,173 +272,175 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         }
     } else {
         // ------------------------------------------------------------ epilogue --------------
-        const int wg = (warp - 2) >> 2;                      // epilogue group 0..3
+        const int wg = (warp - 2) >> 2;                      // epilogue group 0..3 = its accumulator
+        const int sub = wg & 1;                              // stationary tile of this group
+        const int par = wg >> 1;                             // parity of the streamed tiles it takes
+        const int acc = wg;
         const int quarter = warp & 3;                        // TMEM lane quarter this warp may read
         const int row = quarter * 32 + lane;                 // row of the stationary tile
         const uint32_t lane_addr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
         const float c2 = p.scale_log2;
         uint32_t gb = 0;
-        uint32_t lt = 0;                                     // tiles taken by this group
+        uint32_t lt = 0;                                     // staged tiles of this group
         int n = 0;
         for (int round = 0;; ++round, ++n) {
             const int item = item_of_round(round, blockIdx.x, n_cta);
             if (item >= p.n_items) { if (round * n_cta >= p.n_items) break; --n; continue; }
-            const Item it = decode_item<KIND>(p, item);
-            const int pos = it.blk * kTile + row;            // position of this thread's row
+            const Item it = decode_item<KIND>(p, tbl, item);
+            const int blk = 2 * it.bp + sub;                 // this group's stationary block
+            const int pos = blk * kTile + row;               // position of this thread's row
             float m_run = -INFINITY, l_run = 0.f;            // sweep 1
             float acc0 = 0.f, acc1 = 0.f, acc2 = 0.f, acc3 = 0.f;   // sweep 2
             float best = -INFINITY;                          // match
             int best_slot = 0x7fffffff;
 
             for (int t = 0; t < it.nt; ++t, ++gb) {
-                if ((int)(gb % kGroups) != wg) continue;
-                const int buf = wg;
+                if ((int)(gb & 1u) != par) continue;
+                const bool active = unit_active<KIND>(p, it, t, sub);
                 float* side = sh.side[wg][lt & 1];
                 bool diag = false;                           // tile crosses the causal diagonal
                 int col_limit = kTile;                       // match: valid kept slots in the tile
                 if (KIND == kSweep1) {
-                    diag = (t == it.blk);
+                    diag = (t == blk);
                 } else if (KIND == kSweep2) {
-                    const int ib = it.blk + t / p.group;
-                    const int qh = it.head * p.group + t % p.group;
-                    const int i = ib * kTile + row;          // query column staged by this thread
-                    float v = INFINITY;                      // +inf turns the probability into 0
-                    if (i < it.L) v = p.lse[(long long)qh * p.T + it.tok_begin + i] * kLog2e;
-                    side[row] = v;
-                    diag = (ib == it.blk);
-                    ptx::named_barrier_sync(1 + wg, 128);
+                    const int ib = 2 * it.bp + t / p.group;
+                    diag = (ib == blk);
+                    if (active) {
+                        const int qh = it.head * p.group + t % p.group;
+                        const int i = ib * kTile + row;      // query column staged by this thread
+                        float v = INFINITY;                  // +inf turns the probability into 0
+                        if (i < it.L) v = p.lse[(long long)qh * p.T + it.tok_begin + i] * kLog2e;
+                        side[row] = v;
+                        ptx::named_barrier_sync(1 + wg, 128);
+                        ++lt;
+                    }
                 } else {
-                    const int slot = t * kTile + row;
-                    side[row] = (slot < it.B) ? p.rnorm_kept[it.kept_row0 + slot] : 0.f;
                     col_limit = min(kTile, it.B - t * kTile);
-                    ptx::named_barrier_sync(1 + wg, 128);
+                    if (active) {
+                        const int slot = t * kTile + row;
+                        side[row] = (slot < it.B) ? p.rnorm_kept[it.kept_row0 + slot] : 0.f;
+                        ptx::named_barrier_sync(1 + wg, 128);
+                        ++lt;
+                    }
                 }
-                ++lt;
-                ptx::mbar_wait(ptx::smem_u32(&sh.t_full[buf]), (gb / kAccum) & 1, abort_flag);
+                ptx::mbar_wait(ptx::smem_u32(&sh.t_full[par]), (gb >> 1) & 1, abort_flag);
                 ptx::tc_fence_after_sync();
+                if (active) {
 #pragma unroll 1
-                for (int ch = 0; ch < 4; ++ch) {
-                    uint32_t raw[32];
-                    ptx::tmem_ld_32x32(lane_addr + buf * kTile + ch * 32, raw);
-                    ptx::tmem_ld_wait();
-                    const int c0 = ch * 32;
-                    if (KIND == kSweep1) {
-                        // online softmax statistics of row `pos` over key columns c0..c0+31
-                        float mx = m_run;
-                        if (diag) {
-#pragma unroll
-                            for (int c = 0; c < 32; ++c)
-                                if (c0 + c <= row) mx = fmaxf(mx, __uint_as_float(raw[c]));
-                        } else {
-#pragma unroll
-                            for (int c = 0; c < 32; ++c) mx = fmaxf(mx, __uint_as_float(raw[c]));
-                        }
-                        if (mx != -INFINITY) {               // false only above the diagonal
-                            const float mc = mx * c2;
-                            float s0 = 0.f, s1 = 0.f;
+                    for (int ch = 0; ch < 4; ++ch) {
+                        uint32_t raw[32];
+                        ptx::tmem_ld_32x32(lane_addr + acc * kTile + ch * 32, raw);
+                        ptx::tmem_ld_wait();
+                        const int c0 = ch * 32;
+                        if (KIND == kSweep1) {
+                            // online softmax statistics of row `pos` over key columns c0..c0+31
+                            float mx = m_run;
                             if (diag) {
 #pragma unroll
-                                for (int c = 0; c < 32; c += 2) {
-                                    const float e0 = ptx::ex2(fmaf(__uint_as_float(raw[c]), c2, -mc));
-                                    const float e1 = ptx::ex2(fmaf(__uint_as_float(raw[c + 1]), c2, -mc));
-                                    s0 += (c0 + c <= row) ? e0 : 0.f;
-                                    s1 += (c0 + c + 1 <= row) ? e1 : 0.f;
+                                for (int c = 0; c < 32; ++c)
+                                    if (c0 + c <= row) mx = fmaxf(mx, __uint_as_float(raw[c]));
+                            } else {
+#pragma unroll
+                                for (int c = 0; c < 32; ++c) mx = fmaxf(mx, __uint_as_float(raw[c]));
+                            }
+                            if (mx != -INFINITY) {               // false only above the diagonal
+                                const float mc = mx * c2;
+                                float s0 = 0.f, s1 = 0.f;
+                                if (diag) {
+#pragma unroll
+                                    for (int c = 0; c < 32; c += 2) {
+                                        const float e0 = ptx::ex2(fmaf(__uint_as_float(raw[c]), c2, -mc));
+                                        const float e1 = ptx::ex2(fmaf(__uint_as_float(raw[c + 1]), c2, -mc));
+                                        s0 += (c0 + c <= row) ? e0 : 0.f;
+                                        s1 += (c0 + c + 1 <= row) ? e1 : 0.f;
+                                    }
+                                } else {
+#pragma unroll
+                                    for (int c = 0; c < 32; c += 2) {
+                                        s0 += ptx::ex2(fmaf(__uint_as_float(raw[c]), c2, -mc));
+                                        s1 += ptx::ex2(fmaf(__uint_as_float(raw[c + 1]), c2, -mc));
+                                    }
+                                }
+                                l_run = l_run * ptx::ex2(m_run * c2 - mc) + (s0 + s1);
+                                m_run = mx;
+                            }
+                        } else if (KIND == kSweep2) {
+                            // probabilities of key `pos` under query columns c0..c0+31
+                            const float4* sd = reinterpret_cast<const float4*>(side + c0);
+                            if (diag) {
+#pragma unroll
+                                for (int c4 = 0; c4 < 8; ++c4) {
+                                    const float4 l4 = sd[c4];
+                                    const int c = c0 + c4 * 4;
+                                    const float e0 = ptx::ex2(fmaf(__uint_as_float(raw[c4 * 4 + 0]), c2, -l4.x));
+                                    const float e1 = ptx::ex2(fmaf(__uint_as_float(raw[c4 * 4 + 1]), c2, -l4.y));
+                                    const float e2 = ptx::ex2(fmaf(__uint_as_float(raw[c4 * 4 + 2]), c2, -l4.z));
+                                    const float e3 = ptx::ex2(fmaf(__uint_as_float(raw[c4 * 4 + 3]), c2, -l4.w));
+                                    acc0 += (c + 0 >= row) ? e0 : 0.f;
+                                    acc1 += (c + 1 >= row) ? e1 : 0.f;
+                                    acc2 += (c + 2 >= row) ? e2 : 0.f;
+                                    acc3 += (c + 3 >= row) ? e3 : 0.f;
                                 }
                             } else {
 #pragma unroll
-                                for (int c = 0; c < 32; c += 2) {
-                                    s0 += ptx::ex2(fmaf(__uint_as_float(raw[c]), c2, -mc));
-                                    s1 += ptx::ex2(fmaf(__uint_as_float(raw[c + 1]), c2, -mc));
+                                for (int c4 = 0; c4 < 8; ++c4) {
+                                    const float4 l4 = sd[c4];
+                                    acc0 += ptx::ex2(fmaf(__uint_as_float(raw[c4 * 4 + 0]), c2, -l4.x));
+                                    acc1 += ptx::ex2(fmaf(__uint_as_float(raw[c4 * 4 + 1]), c2, -l4.y));
+                                    acc2 += ptx::ex2(fmaf(__uint_as_float(raw[c4 * 4 + 2]), c2, -l4.z));
+                                    acc3 += ptx::ex2(fmaf(__uint_as_float(raw[c4 * 4 + 3]), c2, -l4.w));
                                 }
                             }
-                            l_run = l_run * ptx::ex2(m_run * c2 - mc) + (s0 + s1);
-                            m_run = mx;
-                        }
-                    } else if (KIND == kSweep2) {
-                        // probabilities of key `pos` under query columns c0..c0+31
-                        const float4* sd = reinterpret_cast<const float4*>(side + c0);
-                        if (diag) {
-#pragma unroll
-                            for (int c4 = 0; c4 < 8; ++c4) {
-                                const float4 l4 = sd[c4];
-                                const int c = c0 + c4 * 4;
-                                const float e0 = ptx::ex2(fmaf(__uint_as_float(raw[c4 * 4 + 0]), c2, -l4.x));
-                                const float e1 = ptx::ex2(fmaf(__uint_as_float(raw[c4 * 4 + 1]), c2, -l4.y));
-                                const float e2 = ptx::ex2(fmaf(__uint_as_float(raw[c4 * 4 + 2]), c2, -l4.z));
-                                const float e3 = ptx::ex2(fmaf(__uint_as_float(raw[c4 * 4 + 3]), c2, -l4.w));
-                                acc0 += (c + 0 >= row) ? e0 : 0.f;
-                                acc1 += (c + 1 >= row) ? e1 : 0.f;
-                                acc2 += (c + 2 >= row) ? e2 : 0.f;
-                                acc3 += (c + 3 >= row) ? e3 : 0.f;
-                            }
                         } else {
+                            // running arg-max of dot / |kept key| over kept slots; ascending slot order
+                            // with a strict comparison keeps the lowest slot on ties
+                            const float4* sd = reinterpret_cast<const float4*>(side + c0);
+                            const int slot0 = t * kTile + c0;
 #pragma unroll
                             for (int c4 = 0; c4 < 8; ++c4) {
-                                const float4 l4 = sd[c4];
-                                acc0 += ptx::ex2(fmaf(__uint_as_float(raw[c4 * 4 + 0]), c2, -l4.x));
-                                acc1 += ptx::ex2(fmaf(__uint_as_float(raw[c4 * 4 + 1]), c2, -l4.y));
-                                acc2 += ptx::ex2(fmaf(__uint_as_float(raw[c4 * 4 + 2]), c2, -l4.z));
-                                acc3 += ptx::ex2(fmaf(__uint_as_float(raw[c4 * 4 + 3]), c2, -l4.w));
-                            }
-                        }
-                    } else {
-                        // running arg-max of dot / |kept key| over kept slots; ascending slot order
-                        // with a strict comparison keeps the lowest slot on ties
-                        const float4* sd = reinterpret_cast<const float4*>(side + c0);
-                        const int slot0 = t * kTile + c0;
+                                const float4 r4 = sd[c4];
+                                const float rn[4] = {r4.x, r4.y, r4.z, r4.w};
 #pragma unroll
-                        for (int c4 = 0; c4 < 8; ++c4) {
-                            const float4 r4 = sd[c4];
-                            const float rn[4] = {r4.x, r4.y, r4.z, r4.w};
-#pragma unroll
-                            for (int q = 0; q < 4; ++q) {
-                                const int c = c4 * 4 + q;
-                                const float v = __uint_as_float(raw[c]) * rn[q];
-                                if (c0 + c < col_limit && v > best) { best = v; best_slot = slot0 + c; }
+                                for (int q = 0; q < 4; ++q) {
+                                    const int c = c4 * 4 + q;
+                                    const float v = __uint_as_float(raw[c]) * rn[q];
+                                    if (c0 + c < col_limit && v > best) { best = v; best_slot = slot0 + c; }
+                                }
                             }
                         }
                     }
                 }
                 ptx::tc_fence_before_sync();
                 __syncwarp();
-                if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&sh.t_empty[buf]));
+                if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&sh.t_empty[par]));
             }
 
-            // ---- combine the four groups and write this item's results -----------------------
-            if (wg > 0) {
-                float* cb0 = sh.comb[n & 1][wg - 1][0];
-                float* cb1 = sh.comb[n & 1][wg - 1][1];
+            // ---- combine the two groups of each stationary tile and write the item's results ---
+            float* cb0 = sh.comb[n & 1][sub][0];
+            float* cb1 = sh.comb[n & 1][sub][1];
+            if (par == 1) {
                 if (KIND == kSweep1) { cb0[row] = m_run; cb1[row] = l_run; }
                 else if (KIND == kSweep2) { cb0[row] = (acc0 + acc1) + (acc2 + acc3); }
                 else { cb0[row] = best; cb1[row] = __int_as_float(best_slot); }
             }
             ptx::named_barrier_sync(1 + kGroups, kGroups * 128);
-            if (wg == 0 && pos < it.L && !*abort_flag) {
+            if (par == 0 && pos < it.L && !*abort_flag) {
                 if (KIND == kSweep1) {
-                    float m = m_run;
-#pragma unroll
-                    for (int g = 0; g < kGroups - 1; ++g) m = fmaxf(m, sh.comb[n & 1][g][0][row]);
-                    float l = l_run * ptx::ex2((m_run - m) * c2);
-#pragma unroll
-                    for (int g = 0; g < kGroups - 1; ++g)
-                        l += sh.comb[n & 1][g][1][row] * ptx::ex2((sh.comb[n & 1][g][0][row] - m) * c2);
+                    const float m1 = cb0[row], l1 = cb1[row];
+                    const float m = fmaxf(m_run, m1);
+                    const float l = l_run * ptx::ex2((m_run - m) * c2) + l1 * ptx::ex2((m1 - m) * c2);
                     // natural-log log-sum-exp of the scaled logits
                     p.lse[(long long)it.head * p.T + it.tok_begin + pos] = (m * c2 + ptx::lg2(l)) * kLn2;
                 } else if (KIND == kSweep2) {
-                    float a = (acc0 + acc1) + (acc2 + acc3);
-#pragma unroll
-                    for (int g = 0; g < kGroups - 1; ++g) a += sh.comb[n & 1][g][0][row];
-                    p.scores[(long long)it.head * p.T + it.tok_begin + pos] = a;
+                    p.scores[(long long)it.head * p.T + it.tok_begin + pos] =
+                        ((acc0 + acc1) + (acc2 + acc3)) + cb0[row];
                 } else {
                     const long long g = (long long)it.head * p.T + it.tok_begin + pos;
                     const int e = p.rank[g];
                     if (e >= 0) {
-#pragma unroll
-                        for (int gi = 0; gi < kGroups - 1; ++gi) {
-                            const float b1 = sh.comb[n & 1][gi][0][row];
-                            const int s1 = __float_as_int(sh.comb[n & 1][gi][1][row]);
-                            if (b1 > best || (b1 == best && s1 < best_slot)) { best = b1; best_slot = s1; }
-                        }
+                        const float b1 = cb0[row];
+                        const int s1 = __float_as_int(cb1[row]);
+                        if (b1 > best || (b1 == best && s1 < best_slot)) { best = b1; best_slot = s1; }
                         p.assign[it.ev0 + e] = best_slot;
                         p.sim[it.ev0 + e] = best * p.rnorm_all[g];
                     }
