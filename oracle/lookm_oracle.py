@@ -16,6 +16,7 @@ import ctypes as C
 import math
 import os
 import subprocess
+import threading
 from concurrent.futures import ThreadPoolExecutor
 from typing import Optional, Sequence
 
@@ -25,6 +26,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "lookm_oracle.c")
 _SO = os.path.join(_HERE, "_lookm_oracle.so")
 _lib = None
+_lock = threading.Lock()
 
 MERGE_AVERAGE, MERGE_PIVOTAL, MERGE_WEIGHTED = 0, 1, 2
 
@@ -39,6 +41,12 @@ def build(force: bool = False) -> str:
 
 
 def lib():
+    global _lib
+    with _lock:                      # the heads of a layer call in from a thread pool
+        return _lib_locked()
+
+
+def _lib_locked():
     global _lib
     if _lib is None:
         L = C.CDLL(build())
