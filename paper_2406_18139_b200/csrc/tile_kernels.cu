@@ -12,13 +12,14 @@
 //     fences and commits between every 8 MMAs keeps the tensor pipe only about half busy (512
 //     clocks per 8 MMAs alone, about 900 with one wait and two commits in between), so the
 //     synchronisation is done once per streamed tile and two threads alternate;
-//   - four groups of four warps read the accumulators with tcgen05.ld and run the epilogue: group
-//     g owns accumulator g, i.e. stationary tile (g & 1) under the streamed tiles of parity
-//     (g >> 1);
-//   - each epilogue thread owns one row of its stationary tile, so every reduction over the
-//     streamed axis (row maximum and sum, column-sum of probabilities for one key, running
-//     arg-max) stays in that thread's registers; the two groups that share a stationary tile are
-//     combined through shared memory once per item.  No L x L matrix is ever stored.
+//   - two groups of four warps run the epilogue, one group per stationary tile, alternating
+//     between that tile's two accumulators (so the MMA of the next streamed tile runs meanwhile).
+//     A thread reads its whole accumulator row (128 columns, four tcgen05.ld.x32 in flight, one
+//     wait) before it computes: the TMEM load latency of several hundred clocks is then paid once
+//     per tile, which is what lets two warps per SM sub-partition keep the exp unit busy;
+//   - each epilogue thread owns one row of its stationary tile for the whole item, so every
+//     reduction over the streamed axis (row maximum and sum, column-sum of probabilities for one
+//     key, running arg-max) stays in that thread's registers.  No L x L matrix is ever stored.
 //
 //   sweep 1: A = 256 queries of one query head, B = key tiles 0..diagonal.  Online softmax
 //            statistics per query row  ->  lse[i] = log sum_{j<=i} exp(s_ij).
@@ -38,9 +39,9 @@ namespace lookm {
 namespace {
 
 constexpr int kStages = 4;                       // ring of streamed tiles
-constexpr int kGroups = 4;                       // epilogue groups (one per TMEM accumulator)
+constexpr int kGroups = 2;                       // epilogue groups (one per stationary tile)
 constexpr int kMmaWarp1 = 2 + kGroups * 4;       // the second MMA-issuing warp
-constexpr int kThreads = (kMmaWarp1 + 1) * 32;   // producer, MMA (even), 4 x 4 epilogue, MMA (odd)
+constexpr int kThreads = (kMmaWarp1 + 1) * 32;   // producer, MMA (even), 2 x 4 epilogue, MMA (odd)
 constexpr int kHalfBytes = kTile * 64 * 2;       // one TMA box: 128 rows x 64 bf16 (128 B rows)
 constexpr int kTileBytes = 2 * kHalfBytes;       // 128 x 128 bf16
 constexpr int kReqCache = 32;                    // request-table entries cached in shared memory
@@ -50,8 +51,7 @@ constexpr float kLn2 = 0.6931471805599453f;
 struct __align__(1024) Shared {
     uint8_t a[2][kTileBytes];                    // the item's two stationary tiles
     uint8_t b[kStages][kTileBytes];              // streamed tiles
-    float side[kGroups][2][kTile];               // per epilogue group, double-buffered column data
-    float comb[2][2][2][kTile];                  // [item parity][stationary tile][array][row]
+    alignas(16) float side[kGroups][2][kTile];   // per epilogue group, double-buffered column data
     Req reqs[kReqCache];
     unsigned long long a_full, a_empty;
     unsigned long long b_full[kStages], b_empty[kStages];
@@ -272,20 +272,16 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         }
     } else {
         // ------------------------------------------------------------ epilogue --------------
-        const int wg = (warp - 2) >> 2;                      // epilogue group 0..3 = its accumulator
-        const int sub = wg & 1;                              // stationary tile of this group
-        const int par = wg >> 1;                             // parity of the streamed tiles it takes
-        const int acc = wg;
+        const int sub = (warp - 2) >> 2;                     // epilogue group = stationary tile
         const int quarter = warp & 3;                        // TMEM lane quarter this warp may read
         const int row = quarter * 32 + lane;                 // row of the stationary tile
         const uint32_t lane_addr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
         const float c2 = p.scale_log2;
         uint32_t gb = 0;
         uint32_t lt = 0;                                     // staged tiles of this group
-        int n = 0;
-        for (int round = 0;; ++round, ++n) {
+        for (int round = 0;; ++round) {
             const int item = item_of_round(round, blockIdx.x, n_cta);
-            if (item >= p.n_items) { if (round * n_cta >= p.n_items) break; --n; continue; }
+            if (item >= p.n_items) { if (round * n_cta >= p.n_items) break; continue; }
             const Item it = decode_item<KIND>(p, tbl, item);
             const int blk = 2 * it.bp + sub;                 // this group's stationary block
             const int pos = blk * kTile + row;               // position of this thread's row
@@ -294,118 +290,142 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
             float best = -INFINITY;                          // match
             int best_slot = 0x7fffffff;
 
+            // per-column data of streamed tile t, for the column this thread stages:
+            // sweep 2: log2-sum-exp of the query (+inf past the prompt end: probability 0);
+            // match  : inverse norm of the kept key (0 past the last kept slot)
+            auto side_value = [&](int t) -> float {
+                if (KIND == kSweep2) {
+                    const int i = (2 * it.bp + t / p.group) * kTile + row;
+                    const int qh = it.head * p.group + t % p.group;
+                    return (i < it.L) ? p.lse[(long long)qh * p.T + it.tok_begin + i] * kLog2e : INFINITY;
+                } else if (KIND == kMatch) {
+                    const int slot = t * kTile + row;
+                    return (slot < it.B) ? p.rnorm_kept[it.kept_row0 + slot] : 0.f;
+                }
+                return 0.f;
+            };
+            // first active tile of this group, so that its column data can be fetched ahead
+            int t_next = 0;
+            while (t_next < it.nt && !unit_active<KIND>(p, it, t_next, sub)) ++t_next;
+            float side_next = (KIND != kSweep1 && t_next < it.nt) ? side_value(t_next) : 0.f;
+
             for (int t = 0; t < it.nt; ++t, ++gb) {
-                if ((int)(gb & 1u) != par) continue;
+                const int par = gb & 1;
+                const int acc = 2 * par + sub;
                 const bool active = unit_active<KIND>(p, it, t, sub);
-                float* side = sh.side[wg][lt & 1];
-                bool diag = false;                           // tile crosses the causal diagonal
-                int col_limit = kTile;                       // match: valid kept slots in the tile
-                if (KIND == kSweep1) {
-                    diag = (t == blk);
-                } else if (KIND == kSweep2) {
-                    const int ib = 2 * it.bp + t / p.group;
-                    diag = (ib == blk);
-                    if (active) {
-                        const int qh = it.head * p.group + t % p.group;
-                        const int i = ib * kTile + row;      // query column staged by this thread
-                        float v = INFINITY;                  // +inf turns the probability into 0
-                        if (i < it.L) v = p.lse[(long long)qh * p.T + it.tok_begin + i] * kLog2e;
-                        side[row] = v;
-                        ptx::named_barrier_sync(1 + wg, 128);
-                        ++lt;
-                    }
-                } else {
-                    col_limit = min(kTile, it.B - t * kTile);
-                    if (active) {
-                        const int slot = t * kTile + row;
-                        side[row] = (slot < it.B) ? p.rnorm_kept[it.kept_row0 + slot] : 0.f;
-                        ptx::named_barrier_sync(1 + wg, 128);
-                        ++lt;
-                    }
+                float* side = sh.side[sub][lt & 1];
+                if (KIND != kSweep1 && active) {
+                    side[row] = side_next;                   // fetched during the previous tile
+                    ptx::named_barrier_sync(1 + sub, 128);
+                    ++lt;
+                    t_next = t + 1;                          // later tiles of an item are all active
+                    if (t_next < it.nt) side_next = side_value(t_next);
                 }
                 ptx::mbar_wait(ptx::smem_u32(&sh.t_full[par]), (gb >> 1) & 1, abort_flag);
                 ptx::tc_fence_after_sync();
                 if (active) {
-#pragma unroll 1
-                    for (int ch = 0; ch < 4; ++ch) {
-                        uint32_t raw[32];
-                        ptx::tmem_ld_32x32(lane_addr + acc * kTile + ch * 32, raw);
-                        ptx::tmem_ld_wait();
-                        const int c0 = ch * 32;
-                        if (KIND == kSweep1) {
-                            // online softmax statistics of row `pos` over key columns c0..c0+31
-                            float mx = m_run;
-                            if (diag) {
+                    uint32_t raw[kTile];
 #pragma unroll
-                                for (int c = 0; c < 32; ++c)
-                                    if (c0 + c <= row) mx = fmaxf(mx, __uint_as_float(raw[c]));
-                            } else {
+                    for (int ch = 0; ch < 4; ++ch)
+                        ptx::tmem_ld_32x32(lane_addr + acc * kTile + ch * 32,
+                                           *reinterpret_cast<uint32_t(*)[32]>(&raw[ch * 32]));
+                    ptx::tmem_ld_wait128(raw);
+                    if (KIND == kSweep1) {
+                        // online softmax statistics of row `pos` over the tile's 128 key columns
+                        const bool diag = (t == blk);        // keys j <= i only
+                        float m0 = m_run, m1 = -INFINITY, m2 = -INFINITY, m3 = -INFINITY;
 #pragma unroll
-                                for (int c = 0; c < 32; ++c) mx = fmaxf(mx, __uint_as_float(raw[c]));
-                            }
-                            if (mx != -INFINITY) {               // false only above the diagonal
-                                const float mc = mx * c2;
-                                float s0 = 0.f, s1 = 0.f;
-                                if (diag) {
+                        for (int c = 0; c < kTile; c += 4) {
+                            if (!diag || c + 0 <= row) m0 = fmaxf(m0, __uint_as_float(raw[c + 0]));
+                            if (!diag || c + 1 <= row) m1 = fmaxf(m1, __uint_as_float(raw[c + 1]));
+                            if (!diag || c + 2 <= row) m2 = fmaxf(m2, __uint_as_float(raw[c + 2]));
+                            if (!diag || c + 3 <= row) m3 = fmaxf(m3, __uint_as_float(raw[c + 3]));
+                        }
+                        const float mx = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));   // finite: column 0 is valid
+                        const float mc = mx * c2;
+                        float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+                        if (diag) {
 #pragma unroll
-                                    for (int c = 0; c < 32; c += 2) {
-                                        const float e0 = ptx::ex2(fmaf(__uint_as_float(raw[c]), c2, -mc));
-                                        const float e1 = ptx::ex2(fmaf(__uint_as_float(raw[c + 1]), c2, -mc));
-                                        s0 += (c0 + c <= row) ? e0 : 0.f;
-                                        s1 += (c0 + c + 1 <= row) ? e1 : 0.f;
-                                    }
-                                } else {
-#pragma unroll
-                                    for (int c = 0; c < 32; c += 2) {
-                                        s0 += ptx::ex2(fmaf(__uint_as_float(raw[c]), c2, -mc));
-                                        s1 += ptx::ex2(fmaf(__uint_as_float(raw[c + 1]), c2, -mc));
-                                    }
-                                }
-                                l_run = l_run * ptx::ex2(m_run * c2 - mc) + (s0 + s1);
-                                m_run = mx;
-                            }
-                        } else if (KIND == kSweep2) {
-                            // probabilities of key `pos` under query columns c0..c0+31
-                            const float4* sd = reinterpret_cast<const float4*>(side + c0);
-                            if (diag) {
-#pragma unroll
-                                for (int c4 = 0; c4 < 8; ++c4) {
-                                    const float4 l4 = sd[c4];
-                                    const int c = c0 + c4 * 4;
-                                    const float e0 = ptx::ex2(fmaf(__uint_as_float(raw[c4 * 4 + 0]), c2, -l4.x));
-                                    const float e1 = ptx::ex2(fmaf(__uint_as_float(raw[c4 * 4 + 1]), c2, -l4.y));
-                                    const float e2 = ptx::ex2(fmaf(__uint_as_float(raw[c4 * 4 + 2]), c2, -l4.z));
-                                    const float e3 = ptx::ex2(fmaf(__uint_as_float(raw[c4 * 4 + 3]), c2, -l4.w));
-                                    acc0 += (c + 0 >= row) ? e0 : 0.f;
-                                    acc1 += (c + 1 >= row) ? e1 : 0.f;
-                                    acc2 += (c + 2 >= row) ? e2 : 0.f;
-                                    acc3 += (c + 3 >= row) ? e3 : 0.f;
-                                }
-                            } else {
-#pragma unroll
-                                for (int c4 = 0; c4 < 8; ++c4) {
-                                    const float4 l4 = sd[c4];
-                                    acc0 += ptx::ex2(fmaf(__uint_as_float(raw[c4 * 4 + 0]), c2, -l4.x));
-                                    acc1 += ptx::ex2(fmaf(__uint_as_float(raw[c4 * 4 + 1]), c2, -l4.y));
-                                    acc2 += ptx::ex2(fmaf(__uint_as_float(raw[c4 * 4 + 2]), c2, -l4.z));
-                                    acc3 += ptx::ex2(fmaf(__uint_as_float(raw[c4 * 4 + 3]), c2, -l4.w));
-                                }
+                            for (int c = 0; c < kTile; c += 4) {
+                                const float e0 = ptx::ex2(fmaf(__uint_as_float(raw[c + 0]), c2, -mc));
+                                const float e1 = ptx::ex2(fmaf(__uint_as_float(raw[c + 1]), c2, -mc));
+                                const float e2 = ptx::ex2(fmaf(__uint_as_float(raw[c + 2]), c2, -mc));
+                                const float e3 = ptx::ex2(fmaf(__uint_as_float(raw[c + 3]), c2, -mc));
+                                s0 += (c + 0 <= row) ? e0 : 0.f;
+                                s1 += (c + 1 <= row) ? e1 : 0.f;
+                                s2 += (c + 2 <= row) ? e2 : 0.f;
+                                s3 += (c + 3 <= row) ? e3 : 0.f;
                             }
                         } else {
-                            // running arg-max of dot / |kept key| over kept slots; ascending slot order
-                            // with a strict comparison keeps the lowest slot on ties
-                            const float4* sd = reinterpret_cast<const float4*>(side + c0);
-                            const int slot0 = t * kTile + c0;
 #pragma unroll
-                            for (int c4 = 0; c4 < 8; ++c4) {
-                                const float4 r4 = sd[c4];
-                                const float rn[4] = {r4.x, r4.y, r4.z, r4.w};
+                            for (int c = 0; c < kTile; c += 4) {
+                                s0 += ptx::ex2(fmaf(__uint_as_float(raw[c + 0]), c2, -mc));
+                                s1 += ptx::ex2(fmaf(__uint_as_float(raw[c + 1]), c2, -mc));
+                                s2 += ptx::ex2(fmaf(__uint_as_float(raw[c + 2]), c2, -mc));
+                                s3 += ptx::ex2(fmaf(__uint_as_float(raw[c + 3]), c2, -mc));
+                            }
+                        }
+                        l_run = l_run * ptx::ex2(m_run * c2 - mc) + ((s0 + s1) + (s2 + s3));
+                        m_run = mx;
+                    } else if (KIND == kSweep2) {
+                        // probabilities of key `pos` under the tile's 128 query columns
+                        const bool diag = (2 * it.bp + t / p.group == blk);   // queries i >= j only
+                        const float4* sd = reinterpret_cast<const float4*>(side);
+                        if (diag) {
 #pragma unroll
-                                for (int q = 0; q < 4; ++q) {
-                                    const int c = c4 * 4 + q;
-                                    const float v = __uint_as_float(raw[c]) * rn[q];
-                                    if (c0 + c < col_limit && v > best) { best = v; best_slot = slot0 + c; }
-                                }
+                            for (int c4 = 0; c4 < kTile / 4; ++c4) {
+                                const float4 l4 = sd[c4];
+                                const int c = c4 * 4;
+                                const float e0 = ptx::ex2(fmaf(__uint_as_float(raw[c + 0]), c2, -l4.x));
+                                const float e1 = ptx::ex2(fmaf(__uint_as_float(raw[c + 1]), c2, -l4.y));
+                                const float e2 = ptx::ex2(fmaf(__uint_as_float(raw[c + 2]), c2, -l4.z));
+                                const float e3 = ptx::ex2(fmaf(__uint_as_float(raw[c + 3]), c2, -l4.w));
+                                acc0 += (c + 0 >= row) ? e0 : 0.f;
+                                acc1 += (c + 1 >= row) ? e1 : 0.f;
+                                acc2 += (c + 2 >= row) ? e2 : 0.f;
+                                acc3 += (c + 3 >= row) ? e3 : 0.f;
+                            }
+                        } else {
+#pragma unroll
+                            for (int c4 = 0; c4 < kTile / 4; ++c4) {
+                                const float4 l4 = sd[c4];
+                                const int c = c4 * 4;
+                                acc0 += ptx::ex2(fmaf(__uint_as_float(raw[c + 0]), c2, -l4.x));
+                                acc1 += ptx::ex2(fmaf(__uint_as_float(raw[c + 1]), c2, -l4.y));
+                                acc2 += ptx::ex2(fmaf(__uint_as_float(raw[c + 2]), c2, -l4.z));
+                                acc3 += ptx::ex2(fmaf(__uint_as_float(raw[c + 3]), c2, -l4.w));
+                            }
+                        }
+                    } else {
+                        // running arg-max of dot / |kept key| over kept slots: per 16 columns the
+                        // maximum first; only a new maximum is searched for its (lowest) column
+                        const int col_limit = it.B - t * kTile;      // valid kept slots in the tile
+                        const float4* sd = reinterpret_cast<const float4*>(side);
+#pragma unroll
+                        for (int g16 = 0; g16 < kTile / 16; ++g16) {
+                            float v[16];
+#pragma unroll
+                            for (int c4 = 0; c4 < 4; ++c4) {
+                                const float4 r4 = sd[g16 * 4 + c4];
+                                const int c = g16 * 16 + c4 * 4;
+                                v[c4 * 4 + 0] = __uint_as_float(raw[c + 0]) * r4.x;
+                                v[c4 * 4 + 1] = __uint_as_float(raw[c + 1]) * r4.y;
+                                v[c4 * 4 + 2] = __uint_as_float(raw[c + 2]) * r4.z;
+                                v[c4 * 4 + 3] = __uint_as_float(raw[c + 3]) * r4.w;
+                            }
+                            if (col_limit < kTile) {
+#pragma unroll
+                                for (int c = 0; c < 16; ++c) if (g16 * 16 + c >= col_limit) v[c] = -INFINITY;
+                            }
+                            float mx = v[0];
+#pragma unroll
+                            for (int c = 1; c < 16; ++c) mx = fmaxf(mx, v[c]);
+                            if (mx > best) {                  // strict: an equal value keeps the lower slot
+                                best = mx;
+                                int idx = 15;
+#pragma unroll
+                                for (int c = 14; c >= 0; --c) if (v[c] == mx) idx = c;
+                                best_slot = t * kTile + g16 * 16 + idx;
                             }
                         }
                     }
@@ -415,32 +435,17 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                 if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&sh.t_empty[par]));
             }
 
-            // ---- combine the two groups of each stationary tile and write the item's results ---
-            float* cb0 = sh.comb[n & 1][sub][0];
-            float* cb1 = sh.comb[n & 1][sub][1];
-            if (par == 1) {
-                if (KIND == kSweep1) { cb0[row] = m_run; cb1[row] = l_run; }
-                else if (KIND == kSweep2) { cb0[row] = (acc0 + acc1) + (acc2 + acc3); }
-                else { cb0[row] = best; cb1[row] = __int_as_float(best_slot); }
-            }
-            ptx::named_barrier_sync(1 + kGroups, kGroups * 128);
-            if (par == 0 && pos < it.L && !*abort_flag) {
+            // ---- this thread's row is complete: write the item's result --------------------------
+            if (pos < it.L && !*abort_flag) {
                 if (KIND == kSweep1) {
-                    const float m1 = cb0[row], l1 = cb1[row];
-                    const float m = fmaxf(m_run, m1);
-                    const float l = l_run * ptx::ex2((m_run - m) * c2) + l1 * ptx::ex2((m1 - m) * c2);
                     // natural-log log-sum-exp of the scaled logits
-                    p.lse[(long long)it.head * p.T + it.tok_begin + pos] = (m * c2 + ptx::lg2(l)) * kLn2;
+                    p.lse[(long long)it.head * p.T + it.tok_begin + pos] = (m_run * c2 + ptx::lg2(l_run)) * kLn2;
                 } else if (KIND == kSweep2) {
-                    p.scores[(long long)it.head * p.T + it.tok_begin + pos] =
-                        ((acc0 + acc1) + (acc2 + acc3)) + cb0[row];
+                    p.scores[(long long)it.head * p.T + it.tok_begin + pos] = (acc0 + acc1) + (acc2 + acc3);
                 } else {
                     const long long g = (long long)it.head * p.T + it.tok_begin + pos;
                     const int e = p.rank[g];
                     if (e >= 0) {
-                        const float b1 = cb0[row];
-                        const int s1 = __float_as_int(cb1[row]);
-                        if (b1 > best || (b1 == best && s1 < best_slot)) { best = b1; best_slot = s1; }
                         p.assign[it.ev0 + e] = best_slot;
                         p.sim[it.ev0 + e] = best * p.rnorm_all[g];
                     }
