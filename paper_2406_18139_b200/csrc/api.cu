@@ -97,10 +97,9 @@ int build_plan(Plan& pl, const lookm_layout* lay, int n_req, const int* cu_seqle
         q.item_begin[kSweep2] = (int)it1;
         q.item_begin[kMatch] = (int)it2;
         q.slot_begin = (int)slots;
-        const long long npair = (q.nblk + 1) / 2;        // a work item covers two 128-row blocks
-        it0 += npair * pl.n_q_heads;
-        it1 += npair * pl.n_kv_heads;
-        it2 += q.E > 0 ? npair * pl.n_kv_heads : 0;
+        it0 += (long long)q.nblk * pl.n_q_heads;
+        it1 += (long long)q.nblk * pl.n_kv_heads;
+        it2 += q.E > 0 ? (long long)q.nblk * pl.n_kv_heads : 0;
         slots += (long long)q.B * pl.n_kv_heads;
     }
     pl.n_items[kSweep1] = (int)it0;

@@ -157,19 +157,6 @@ __device__ __forceinline__ void tmem_ld_wait() {
     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
 
-// Waits for every outstanding tcgen05.ld of this thread.  The 128 destination registers are
-// named as in/out operands (in groups, an asm statement takes at most 30 operands) so that no
-// use of them can be scheduled before the wait.
-__device__ __forceinline__ void tmem_ld_wait128(uint32_t (&r)[128]) {
-    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-#pragma unroll
-    for (int g = 0; g < 128; g += 16)
-        asm volatile("" : "+r"(r[g + 0]), "+r"(r[g + 1]), "+r"(r[g + 2]), "+r"(r[g + 3]), "+r"(r[g + 4]),
-                          "+r"(r[g + 5]), "+r"(r[g + 6]), "+r"(r[g + 7]), "+r"(r[g + 8]), "+r"(r[g + 9]),
-                          "+r"(r[g + 10]), "+r"(r[g + 11]), "+r"(r[g + 12]), "+r"(r[g + 13]),
-                          "+r"(r[g + 14]), "+r"(r[g + 15]) :: "memory");
-}
-
 __device__ __forceinline__ float ex2(float x) {
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));

@@ -2,30 +2,22 @@
 // the cosine matching with fused row argmax (Eq. 9).
 //
 // All three are the same persistent, warp-specialised pipeline over 128 x 128 x 128 bf16 tiles:
-//   - a work item owns TWO stationary 128-row tiles (256 consecutive rows of the A operand; the
-//     rows of each tile sit on the 128 TMEM lanes) and streams a sequence of 128-row tiles (the B
-//     operand) against them, so every streamed tile feeds two MMAs (16 tcgen05.mma of
-//     128 x 128 x 16) and the L2 -> shared-memory traffic per flop is halved;
-//   - warp 0 (one thread) issues the TMA loads; warps 1 and 18 (one thread each) issue the MMAs
-//     of the even and of the odd streamed tiles into four 128-column TMEM accumulators (streamed
-//     tile parity x stationary tile).  Measured on B200: a thread that waits on an mbarrier,
-//     fences and commits between every 8 MMAs keeps the tensor pipe only about half busy (512
-//     clocks per 8 MMAs alone, about 900 with one wait and two commits in between), so the
-//     synchronisation is done once per streamed tile and two threads alternate;
-//   - two groups of four warps run the epilogue, one group per stationary tile, alternating
-//     between that tile's two accumulators (so the MMA of the next streamed tile runs meanwhile).
-//     A thread reads its whole accumulator row (128 columns, four tcgen05.ld.x32 in flight, one
-//     wait) before it computes: the TMEM load latency of several hundred clocks is then paid once
-//     per tile, which is what lets two warps per SM sub-partition keep the exp unit busy;
-//   - each epilogue thread owns one row of its stationary tile for the whole item, so every
-//     reduction over the streamed axis (row maximum and sum, column-sum of probabilities for one
-//     key, running arg-max) stays in that thread's registers.  No L x L matrix is ever stored.
+//   - a work item owns one STATIONARY 128-row tile (the A operand, rows on the 128 TMEM lanes)
+//     and streams a sequence of 128-row tiles (the B operand) against it;
+//   - warp 0 (one thread) issues the TMA loads, warp 1 (one thread) issues tcgen05.mma into one of
+//     four 128-column TMEM accumulators, and four groups of four warps read the accumulators with
+//     tcgen05.ld and run the epilogue; group w owns accumulator w and takes the tiles whose running
+//     index is w mod 4, so each SM sub-partition always has four epilogue warps to switch between;
+//   - each epilogue thread owns one row of the stationary tile, so every reduction over the
+//     streamed axis (row maximum and sum, column-sum of probabilities for one key, running
+//     arg-max) stays in that thread's registers; the two groups are combined through shared
+//     memory once per item.  No L x L matrix is ever stored.
 //
-//   sweep 1: A = 256 queries of one query head, B = key tiles 0..diagonal.  Online softmax
+//   sweep 1: A = 128 queries of one query head, B = key tiles 0..diagonal.  Online softmax
 //            statistics per query row  ->  lse[i] = log sum_{j<=i} exp(s_ij).
-//   sweep 2: A = 256 keys of one KV head, B = query tiles diagonal..last of every query head in
+//   sweep 2: A = 128 keys of one KV head, B = query tiles diagonal..last of every query head in
 //            the group.  Thread of key j accumulates sum_i exp(s_ij - lse_i)  ->  A_s[j].
-//   match  : A = 256 key rows (all positions; kept rows are ignored at the end), B = tiles of the
+//   match  : A = 128 key rows (all positions; kept rows are ignored at the end), B = tiles of the
 //            compacted kept keys.  Thread keeps the largest s_ij / |k_j| and its slot.
 //
 // Work items are laid out heaviest first and dealt to the CTAs in serpentine order; every role
@@ -39,9 +31,9 @@ namespace lookm {
 namespace {
 
 constexpr int kStages = 4;                       // ring of streamed tiles
-constexpr int kGroups = 2;                       // epilogue groups (one per stationary tile)
-constexpr int kMmaWarp1 = 2 + kGroups * 4;       // the second MMA-issuing warp
-constexpr int kThreads = (kMmaWarp1 + 1) * 32;   // producer, MMA (even), 2 x 4 epilogue, MMA (odd)
+constexpr int kAccum = 4;                        // TMEM accumulators (128 fp32 columns each)
+constexpr int kGroups = 4;                       // epilogue groups (one per TMEM accumulator)
+constexpr int kThreads = 64 + kGroups * 128;     // producer warp, MMA warp, 4 x 4 epilogue warps
 constexpr int kHalfBytes = kTile * 64 * 2;       // one TMA box: 128 rows x 64 bf16 (128 B rows)
 constexpr int kTileBytes = 2 * kHalfBytes;       // 128 x 128 bf16
 constexpr int kReqCache = 32;                    // request-table entries cached in shared memory
@@ -49,26 +41,25 @@ constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 
 struct __align__(1024) Shared {
-    uint8_t a[2][kTileBytes];                    // the item's two stationary tiles
+    uint8_t a[2][kTileBytes];                    // stationary tiles (double-buffered across items)
     uint8_t b[kStages][kTileBytes];              // streamed tiles
-    alignas(16) float side[kGroups][2][kTile];   // per epilogue group, double-buffered column data
-    Req reqs[kReqCache];
-    unsigned long long a_full, a_empty;
+    float side[kGroups][2][kTile];               // per epilogue group, double-buffered column data
+    float comb[2][kGroups - 1][2][kTile];        // partial results of groups 1.., double-buffered
+    Req reqs[kReqCache];                         // copy of the request table (when it fits)
+    unsigned long long a_full[2], a_empty[2];
     unsigned long long b_full[kStages], b_empty[kStages];
-    unsigned long long t_full[2], t_empty[2];    // per streamed-tile parity (two accumulators each)
+    unsigned long long t_full[kAccum], t_empty[kAccum];
     unsigned long long mma_done;                 // every MMA of this CTA has completed
     uint32_t tmem_base;
     int abort_flag;
 };
-static_assert(sizeof(Shared) + 1024 <= 232448, "shared storage exceeds what one CTA may use");
 
 struct Item {
-    int tok_begin, L, B, bp, head, nt, nblk;
+    int tok_begin, L, B, blk, head, nt;
     long long kept_row0;      // match: first row of this (request, head) in the kept-key matrix
     long long ev0;            // match: start of its evicted list
 };
 
-// Work item `item` of stage KIND.  An item covers block pair bp = stationary blocks 2bp, 2bp+1.
 template <int KIND>
 __device__ __forceinline__ Item decode_item(const TileParams& p, const Req* tbl, int item) {
     int lo = 0, hi = p.n_req - 1;
@@ -78,41 +69,28 @@ __device__ __forceinline__ Item decode_item(const TileParams& p, const Req* tbl,
     }
     const Req& rq = tbl[lo];
     const int u = item - rq.item_begin[KIND];
-    const int npair = (rq.nblk + 1) >> 1;
     Item it;
     it.tok_begin = rq.tok_begin;
     it.L = rq.L;
     it.B = rq.B;
-    it.nblk = rq.nblk;
     it.kept_row0 = 0;
     it.ev0 = 0;
-    if (KIND == kSweep1) {                       // heaviest first: last query blocks first
-        it.bp = npair - 1 - u / p.n_q_heads;
+    if (KIND == kSweep1) {                       // heaviest first: last query block first
+        it.blk = rq.nblk - 1 - u / p.n_q_heads;
         it.head = u % p.n_q_heads;
-        it.nt = min(rq.nblk, 2 * it.bp + 2);     // key tiles 0 .. the later block's diagonal
-    } else if (KIND == kSweep2) {                // heaviest first: first key blocks first
-        it.bp = u / p.n_kv_heads;
+        it.nt = it.blk + 1;
+    } else if (KIND == kSweep2) {                // heaviest first: first key block first
+        it.blk = u / p.n_kv_heads;
         it.head = u % p.n_kv_heads;
-        it.nt = (rq.nblk - 2 * it.bp) * p.group;
+        it.nt = (rq.nblk - it.blk) * p.group;
     } else {
-        it.bp = u / p.n_kv_heads;
+        it.blk = u / p.n_kv_heads;
         it.head = u % p.n_kv_heads;
         it.nt = (rq.B + kTile - 1) / kTile;
         it.kept_row0 = rq.kept_off + (long long)it.head * rq.B;
         it.ev0 = rq.ev_off + (long long)it.head * rq.E;
     }
     return it;
-}
-
-// Does streamed tile t contribute anything to stationary tile `sub` of the item?  (The block may
-// lie past the prompt end, or the whole tile may be on the wrong side of the causal diagonal.)
-template <int KIND>
-__device__ __forceinline__ bool unit_active(const TileParams& p, const Item& it, int t, int sub) {
-    const int blk = 2 * it.bp + sub;
-    if (blk >= it.nblk) return false;
-    if (KIND == kSweep1) return t <= blk;                          // keys up to the query block
-    if (KIND == kSweep2) return 2 * it.bp + t / p.group >= blk;    // queries from the key block on
-    return true;
 }
 
 // Serpentine deal of the item list: round k hands items k*G .. k*G+G-1 to the CTAs in forward
@@ -133,17 +111,19 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     volatile int* abort_flag = &sh.abort_flag;
 
     if (threadIdx.x == 0) {
-        ptx::mbar_init(ptx::smem_u32(&sh.a_full), 1);
-        ptx::mbar_init(ptx::smem_u32(&sh.a_empty), 2);         // one arrival per MMA thread
+        for (int i = 0; i < 2; ++i) {
+            ptx::mbar_init(ptx::smem_u32(&sh.a_full[i]), 1);
+            ptx::mbar_init(ptx::smem_u32(&sh.a_empty[i]), 1);
+        }
         for (int i = 0; i < kStages; ++i) {
             ptx::mbar_init(ptx::smem_u32(&sh.b_full[i]), 1);
             ptx::mbar_init(ptx::smem_u32(&sh.b_empty[i]), 1);
         }
-        for (int i = 0; i < 2; ++i) {
+        for (int i = 0; i < kAccum; ++i) {
             ptx::mbar_init(ptx::smem_u32(&sh.t_full[i]), 1);
-            ptx::mbar_init(ptx::smem_u32(&sh.t_empty[i]), 8);  // one arrival per warp of two groups
+            ptx::mbar_init(ptx::smem_u32(&sh.t_empty[i]), 4);   // one arrival per epilogue warp
         }
-        ptx::mbar_init(ptx::smem_u32(&sh.mma_done), 2);
+        ptx::mbar_init(ptx::smem_u32(&sh.mma_done), 1);
         sh.abort_flag = 0;
         ptx::fence_mbar_init();
     }
@@ -174,17 +154,15 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                 const int item = item_of_round(round, blockIdx.x, n_cta);
                 if (item >= p.n_items) { if (round * n_cta >= p.n_items) break; --n; continue; }
                 const Item it = decode_item<KIND>(p, tbl, item);
-                // both stationary tiles; rows past the tensor end read as zero
-                ptx::mbar_wait(ptx::smem_u32(&sh.a_empty), (n & 1) ^ 1, abort_flag);
-                const uint32_t abar = ptx::smem_u32(&sh.a_full);
-                ptx::mbar_arrive_expect_tx(abar, 2 * kTileBytes);
-#pragma unroll
-                for (int sub = 0; sub < 2; ++sub) {
-                    const uint32_t adst = ptx::smem_u32(&sh.a[sub][0]);
-                    const int a_row = it.tok_begin + (2 * it.bp + sub) * kTile;
-                    ptx::tma_load_3d(adst, &map_a, 0, it.head, a_row, abar);
-                    ptx::tma_load_3d(adst + kHalfBytes, &map_a, 64, it.head, a_row, abar);
-                }
+                const int ab = n & 1;
+                ptx::mbar_wait(ptx::smem_u32(&sh.a_empty[ab]), ((n >> 1) & 1) ^ 1, abort_flag);
+                const uint32_t abar = ptx::smem_u32(&sh.a_full[ab]);
+                ptx::mbar_arrive_expect_tx(abar, kTileBytes);
+                const uint32_t adst = ptx::smem_u32(&sh.a[ab][0]);
+                const int a_head = it.head;
+                const int a_row = it.tok_begin + it.blk * kTile;
+                ptx::tma_load_3d(adst, &map_a, 0, a_head, a_row, abar);
+                ptx::tma_load_3d(adst + kHalfBytes, &map_a, 64, a_head, a_row, abar);
                 for (int t = 0; t < it.nt; ++t, ++gb) {
                     const int s = gb % kStages;
                     ptx::mbar_wait(ptx::smem_u32(&sh.b_empty[s]), ((gb / kStages) & 1) ^ 1, abort_flag);
@@ -197,7 +175,7 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                         ptx::tma_load_3d(bdst, &map_b, 0, h, row, bbar);
                         ptx::tma_load_3d(bdst + kHalfBytes, &map_b, 64, h, row, bbar);
                     } else if (KIND == kSweep2) {
-                        const int row = it.tok_begin + (2 * it.bp + t / p.group) * kTile;
+                        const int row = it.tok_begin + (it.blk + t / p.group) * kTile;
                         const int h = it.head * p.group + t % p.group;
                         ptx::tma_load_3d(bdst, &map_b, 0, h, row, bbar);
                         ptx::tma_load_3d(bdst + kHalfBytes, &map_b, 64, h, row, bbar);
@@ -208,7 +186,7 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                     }
                 }
             }
-            // Every load issued above is consumed by an MMA thread before it finishes, except
+            // Every load issued above is consumed by the MMA warp before it finishes, except
             // after an abort: then wait (bounded, ignoring the flag) until the last ring of
             // loads has landed so that no copy is in flight when the CTA exits.
             if (*abort_flag) {
@@ -219,49 +197,38 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                                    200000000ull);
             }
         }
-    } else if (warp == 1 || warp == kMmaWarp1) {
-        // ------------------------------------------------------------ MMA issuers -----------
+    } else if (warp == 1) {
+        // ------------------------------------------------------------ MMA issuer ------------
         if (lane == 0) {
             constexpr uint32_t idesc = ptx::umma_idesc_bf16(kTile, kTile);
-            const uint32_t mine = (warp == 1) ? 0u : 1u;     // parity of the streamed tiles I issue
             uint32_t gb = 0;
             int n = 0;
             for (int round = 0;; ++round, ++n) {
                 const int item = item_of_round(round, blockIdx.x, n_cta);
                 if (item >= p.n_items) { if (round * n_cta >= p.n_items) break; --n; continue; }
                 const Item it = decode_item<KIND>(p, tbl, item);
-                // my last streamed tile of this item (-1: its only tile has the other parity)
-                int last_t = it.nt - 1;
-                if (((gb + last_t) & 1u) != mine) --last_t;
-                // Always wait for this item's stationary tiles: their arrival also proves that the
-                // previous item's a_empty phase is over, so the arrival below cannot fall into it.
-                ptx::mbar_wait(ptx::smem_u32(&sh.a_full), n & 1, abort_flag);
-                if (last_t < 0) ptx::mbar_arrive(ptx::smem_u32(&sh.a_empty));
+                const int ab = n & 1;
+                ptx::mbar_wait(ptx::smem_u32(&sh.a_full[ab]), (n >> 1) & 1, abort_flag);
+                const uint32_t a_addr = ptx::smem_u32(&sh.a[ab][0]);
                 for (int t = 0; t < it.nt; ++t, ++gb) {
-                    if ((gb & 1u) != mine) continue;
                     const int s = gb % kStages;
+                    const int buf = gb % kAccum;
                     ptx::mbar_wait(ptx::smem_u32(&sh.b_full[s]), (gb / kStages) & 1, abort_flag);
-                    ptx::mbar_wait(ptx::smem_u32(&sh.t_empty[mine]), ((gb >> 1) & 1) ^ 1, abort_flag);
+                    ptx::mbar_wait(ptx::smem_u32(&sh.t_empty[buf]), ((gb / kAccum) & 1) ^ 1, abort_flag);
                     ptx::tc_fence_after_sync();
                     const uint32_t b_addr = ptx::smem_u32(&sh.b[s][0]);
+                    const uint32_t d_tmem = tmem_base + buf * kTile;
 #pragma unroll
-                    for (int sub = 0; sub < 2; ++sub) {
-                        if (unit_active<KIND>(p, it, t, sub)) {
-                            const uint32_t a_addr = ptx::smem_u32(&sh.a[sub][0]);
-                            const uint32_t d_tmem = tmem_base + (2 * mine + sub) * kTile;
-#pragma unroll
-                            for (int kk = 0; kk < 8; ++kk) {
-                                // 16 bf16 (32 bytes) per MMA along the 128-byte swizzled row; the
-                                // second half of head_dim lives in the second TMA box.
-                                const uint32_t off = (kk >> 2) * kHalfBytes + (kk & 3) * 32;
-                                ptx::umma_bf16(d_tmem, ptx::umma_desc_sw128(a_addr + off),
-                                               ptx::umma_desc_sw128(b_addr + off), idesc, kk > 0);
-                            }
-                        }
+                    for (int kk = 0; kk < 8; ++kk) {
+                        // 16 bf16 (32 bytes) per MMA along the 128-byte swizzled row; the second
+                        // half of head_dim lives in the second TMA box.
+                        const uint32_t off = (kk >> 2) * kHalfBytes + (kk & 3) * 32;
+                        ptx::umma_bf16(d_tmem, ptx::umma_desc_sw128(a_addr + off),
+                                       ptx::umma_desc_sw128(b_addr + off), idesc, kk > 0);
                     }
-                    ptx::umma_commit(ptx::smem_u32(&sh.t_full[mine]));
                     ptx::umma_commit(ptx::smem_u32(&sh.b_empty[s]));
-                    if (t == last_t) ptx::umma_commit(ptx::smem_u32(&sh.a_empty));
+                    ptx::umma_commit(ptx::smem_u32(&sh.t_full[buf]));
+                    if (t == it.nt - 1) ptx::umma_commit(ptx::smem_u32(&sh.a_empty[ab]));
                 }
             }
             // Nothing may release TMEM or leave the kernel while an MMA is still running, also
@@ -272,114 +239,100 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         }
     } else {
         // ------------------------------------------------------------ epilogue --------------
-        const int sub = (warp - 2) >> 2;                     // epilogue group = stationary tile
+        const int wg = (warp - 2) >> 2;                      // epilogue group 0..3
         const int quarter = warp & 3;                        // TMEM lane quarter this warp may read
         const int row = quarter * 32 + lane;                 // row of the stationary tile
         const uint32_t lane_addr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
         const float c2 = p.scale_log2;
         uint32_t gb = 0;
-        uint32_t lt = 0;                                     // staged tiles of this group
-        for (int round = 0;; ++round) {
+        uint32_t lt = 0;                                     // tiles taken by this group
+        int n = 0;
+        for (int round = 0;; ++round, ++n) {
             const int item = item_of_round(round, blockIdx.x, n_cta);
-            if (item >= p.n_items) { if (round * n_cta >= p.n_items) break; continue; }
+            if (item >= p.n_items) { if (round * n_cta >= p.n_items) break; --n; continue; }
             const Item it = decode_item<KIND>(p, tbl, item);
-            const int blk = 2 * it.bp + sub;                 // this group's stationary block
-            const int pos = blk * kTile + row;               // position of this thread's row
+            const int pos = it.blk * kTile + row;            // position of this thread's row
             float m_run = -INFINITY, l_run = 0.f;            // sweep 1
             float acc0 = 0.f, acc1 = 0.f, acc2 = 0.f, acc3 = 0.f;   // sweep 2
             float best = -INFINITY;                          // match
             int best_slot = 0x7fffffff;
 
-            // per-column data of streamed tile t, for the column this thread stages:
-            // sweep 2: log2-sum-exp of the query (+inf past the prompt end: probability 0);
-            // match  : inverse norm of the kept key (0 past the last kept slot)
-            auto side_value = [&](int t) -> float {
-                if (KIND == kSweep2) {
-                    const int i = (2 * it.bp + t / p.group) * kTile + row;
-                    const int qh = it.head * p.group + t % p.group;
-                    return (i < it.L) ? p.lse[(long long)qh * p.T + it.tok_begin + i] * kLog2e : INFINITY;
-                } else if (KIND == kMatch) {
-                    const int slot = t * kTile + row;
-                    return (slot < it.B) ? p.rnorm_kept[it.kept_row0 + slot] : 0.f;
-                }
-                return 0.f;
-            };
-            // first active tile of this group, so that its column data can be fetched ahead
-            int t_next = 0;
-            while (t_next < it.nt && !unit_active<KIND>(p, it, t_next, sub)) ++t_next;
-            float side_next = (KIND != kSweep1 && t_next < it.nt) ? side_value(t_next) : 0.f;
-
             for (int t = 0; t < it.nt; ++t, ++gb) {
-                const int par = gb & 1;
-                const int acc = 2 * par + sub;
-                const bool active = unit_active<KIND>(p, it, t, sub);
-                float* side = sh.side[sub][lt & 1];
-                if (KIND != kSweep1 && active) {
-                    side[row] = side_next;                   // fetched during the previous tile
-                    ptx::named_barrier_sync(1 + sub, 128);
-                    ++lt;
-                    t_next = t + 1;                          // later tiles of an item are all active
-                    if (t_next < it.nt) side_next = side_value(t_next);
+                if ((int)(gb % kGroups) != wg) continue;
+                const int buf = wg;
+                float* side = sh.side[wg][lt & 1];
+                bool diag = false;                           // tile crosses the causal diagonal
+                int col_limit = kTile;                       // match: valid kept slots in the tile
+                if (KIND == kSweep1) {
+                    diag = (t == it.blk);
+                } else if (KIND == kSweep2) {
+                    const int ib = it.blk + t / p.group;
+                    const int qh = it.head * p.group + t % p.group;
+                    const int i = ib * kTile + row;          // query column staged by this thread
+                    float v = INFINITY;                      // +inf turns the probability into 0
+                    if (i < it.L) v = p.lse[(long long)qh * p.T + it.tok_begin + i] * kLog2e;
+                    side[row] = v;
+                    diag = (ib == it.blk);
+                    ptx::named_barrier_sync(1 + wg, 128);
+                } else {
+                    const int slot = t * kTile + row;
+                    side[row] = (slot < it.B) ? p.rnorm_kept[it.kept_row0 + slot] : 0.f;
+                    col_limit = min(kTile, it.B - t * kTile);
+                    ptx::named_barrier_sync(1 + wg, 128);
                 }
-                ptx::mbar_wait(ptx::smem_u32(&sh.t_full[par]), (gb >> 1) & 1, abort_flag);
+                ++lt;
+                ptx::mbar_wait(ptx::smem_u32(&sh.t_full[buf]), (gb / kAccum) & 1, abort_flag);
                 ptx::tc_fence_after_sync();
-                if (active) {
-                    uint32_t raw[kTile];
-#pragma unroll
-                    for (int ch = 0; ch < 4; ++ch)
-                        ptx::tmem_ld_32x32(lane_addr + acc * kTile + ch * 32,
-                                           *reinterpret_cast<uint32_t(*)[32]>(&raw[ch * 32]));
-                    ptx::tmem_ld_wait128(raw);
+#pragma unroll 1
+                for (int ch = 0; ch < 4; ++ch) {
+                    uint32_t raw[32];
+                    ptx::tmem_ld_32x32(lane_addr + buf * kTile + ch * 32, raw);
+                    ptx::tmem_ld_wait();
+                    const int c0 = ch * 32;
                     if (KIND == kSweep1) {
-                        // online softmax statistics of row `pos` over the tile's 128 key columns
-                        const bool diag = (t == blk);        // keys j <= i only
-                        float m0 = m_run, m1 = -INFINITY, m2 = -INFINITY, m3 = -INFINITY;
-#pragma unroll
-                        for (int c = 0; c < kTile; c += 4) {
-                            if (!diag || c + 0 <= row) m0 = fmaxf(m0, __uint_as_float(raw[c + 0]));
-                            if (!diag || c + 1 <= row) m1 = fmaxf(m1, __uint_as_float(raw[c + 1]));
-                            if (!diag || c + 2 <= row) m2 = fmaxf(m2, __uint_as_float(raw[c + 2]));
-                            if (!diag || c + 3 <= row) m3 = fmaxf(m3, __uint_as_float(raw[c + 3]));
-                        }
-                        const float mx = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));   // finite: column 0 is valid
-                        const float mc = mx * c2;
-                        float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+                        // online softmax statistics of row `pos` over key columns c0..c0+31
+                        float mx = m_run;
                         if (diag) {
 #pragma unroll
-                            for (int c = 0; c < kTile; c += 4) {
-                                const float e0 = ptx::ex2(fmaf(__uint_as_float(raw[c + 0]), c2, -mc));
-                                const float e1 = ptx::ex2(fmaf(__uint_as_float(raw[c + 1]), c2, -mc));
-                                const float e2 = ptx::ex2(fmaf(__uint_as_float(raw[c + 2]), c2, -mc));
-                                const float e3 = ptx::ex2(fmaf(__uint_as_float(raw[c + 3]), c2, -mc));
-                                s0 += (c + 0 <= row) ? e0 : 0.f;
-                                s1 += (c + 1 <= row) ? e1 : 0.f;
-                                s2 += (c + 2 <= row) ? e2 : 0.f;
-                                s3 += (c + 3 <= row) ? e3 : 0.f;
-                            }
+                            for (int c = 0; c < 32; ++c)
+                                if (c0 + c <= row) mx = fmaxf(mx, __uint_as_float(raw[c]));
                         } else {
 #pragma unroll
-                            for (int c = 0; c < kTile; c += 4) {
-                                s0 += ptx::ex2(fmaf(__uint_as_float(raw[c + 0]), c2, -mc));
-                                s1 += ptx::ex2(fmaf(__uint_as_float(raw[c + 1]), c2, -mc));
-                                s2 += ptx::ex2(fmaf(__uint_as_float(raw[c + 2]), c2, -mc));
-                                s3 += ptx::ex2(fmaf(__uint_as_float(raw[c + 3]), c2, -mc));
-                            }
+                            for (int c = 0; c < 32; ++c) mx = fmaxf(mx, __uint_as_float(raw[c]));
                         }
-                        l_run = l_run * ptx::ex2(m_run * c2 - mc) + ((s0 + s1) + (s2 + s3));
-                        m_run = mx;
+                        if (mx != -INFINITY) {               // false only above the diagonal
+                            const float mc = mx * c2;
+                            float s0 = 0.f, s1 = 0.f;
+                            if (diag) {
+#pragma unroll
+                                for (int c = 0; c < 32; c += 2) {
+                                    const float e0 = ptx::ex2(fmaf(__uint_as_float(raw[c]), c2, -mc));
+                                    const float e1 = ptx::ex2(fmaf(__uint_as_float(raw[c + 1]), c2, -mc));
+                                    s0 += (c0 + c <= row) ? e0 : 0.f;
+                                    s1 += (c0 + c + 1 <= row) ? e1 : 0.f;
+                                }
+                            } else {
+#pragma unroll
+                                for (int c = 0; c < 32; c += 2) {
+                                    s0 += ptx::ex2(fmaf(__uint_as_float(raw[c]), c2, -mc));
+                                    s1 += ptx::ex2(fmaf(__uint_as_float(raw[c + 1]), c2, -mc));
+                                }
+                            }
+                            l_run = l_run * ptx::ex2(m_run * c2 - mc) + (s0 + s1);
+                            m_run = mx;
+                        }
                     } else if (KIND == kSweep2) {
-                        // probabilities of key `pos` under the tile's 128 query columns
-                        const bool diag = (2 * it.bp + t / p.group == blk);   // queries i >= j only
-                        const float4* sd = reinterpret_cast<const float4*>(side);
+                        // probabilities of key `pos` under query columns c0..c0+31
+                        const float4* sd = reinterpret_cast<const float4*>(side + c0);
                         if (diag) {
 #pragma unroll
-                            for (int c4 = 0; c4 < kTile / 4; ++c4) {
+                            for (int c4 = 0; c4 < 8; ++c4) {
                                 const float4 l4 = sd[c4];
-                                const int c = c4 * 4;
-                                const float e0 = ptx::ex2(fmaf(__uint_as_float(raw[c + 0]), c2, -l4.x));
-                                const float e1 = ptx::ex2(fmaf(__uint_as_float(raw[c + 1]), c2, -l4.y));
-                                const float e2 = ptx::ex2(fmaf(__uint_as_float(raw[c + 2]), c2, -l4.z));
-                                const float e3 = ptx::ex2(fmaf(__uint_as_float(raw[c + 3]), c2, -l4.w));
+                                const int c = c0 + c4 * 4;
+                                const float e0 = ptx::ex2(fmaf(__uint_as_float(raw[c4 * 4 + 0]), c2, -l4.x));
+                                const float e1 = ptx::ex2(fmaf(__uint_as_float(raw[c4 * 4 + 1]), c2, -l4.y));
+                                const float e2 = ptx::ex2(fmaf(__uint_as_float(raw[c4 * 4 + 2]), c2, -l4.z));
+                                const float e3 = ptx::ex2(fmaf(__uint_as_float(raw[c4 * 4 + 3]), c2, -l4.w));
                                 acc0 += (c + 0 >= row) ? e0 : 0.f;
                                 acc1 += (c + 1 >= row) ? e1 : 0.f;
                                 acc2 += (c + 2 >= row) ? e2 : 0.f;
@@ -387,65 +340,72 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                             }
                         } else {
 #pragma unroll
-                            for (int c4 = 0; c4 < kTile / 4; ++c4) {
+                            for (int c4 = 0; c4 < 8; ++c4) {
                                 const float4 l4 = sd[c4];
-                                const int c = c4 * 4;
-                                acc0 += ptx::ex2(fmaf(__uint_as_float(raw[c + 0]), c2, -l4.x));
-                                acc1 += ptx::ex2(fmaf(__uint_as_float(raw[c + 1]), c2, -l4.y));
-                                acc2 += ptx::ex2(fmaf(__uint_as_float(raw[c + 2]), c2, -l4.z));
-                                acc3 += ptx::ex2(fmaf(__uint_as_float(raw[c + 3]), c2, -l4.w));
+                                acc0 += ptx::ex2(fmaf(__uint_as_float(raw[c4 * 4 + 0]), c2, -l4.x));
+                                acc1 += ptx::ex2(fmaf(__uint_as_float(raw[c4 * 4 + 1]), c2, -l4.y));
+                                acc2 += ptx::ex2(fmaf(__uint_as_float(raw[c4 * 4 + 2]), c2, -l4.z));
+                                acc3 += ptx::ex2(fmaf(__uint_as_float(raw[c4 * 4 + 3]), c2, -l4.w));
                             }
                         }
                     } else {
-                        // running arg-max of dot / |kept key| over kept slots: per 16 columns the
-                        // maximum first; only a new maximum is searched for its (lowest) column
-                        const int col_limit = it.B - t * kTile;      // valid kept slots in the tile
-                        const float4* sd = reinterpret_cast<const float4*>(side);
+                        // running arg-max of dot / |kept key| over kept slots; ascending slot order
+                        // with a strict comparison keeps the lowest slot on ties
+                        const float4* sd = reinterpret_cast<const float4*>(side + c0);
+                        const int slot0 = t * kTile + c0;
 #pragma unroll
-                        for (int g16 = 0; g16 < kTile / 16; ++g16) {
-                            float v[16];
+                        for (int c4 = 0; c4 < 8; ++c4) {
+                            const float4 r4 = sd[c4];
+                            const float rn[4] = {r4.x, r4.y, r4.z, r4.w};
 #pragma unroll
-                            for (int c4 = 0; c4 < 4; ++c4) {
-                                const float4 r4 = sd[g16 * 4 + c4];
-                                const int c = g16 * 16 + c4 * 4;
-                                v[c4 * 4 + 0] = __uint_as_float(raw[c + 0]) * r4.x;
-                                v[c4 * 4 + 1] = __uint_as_float(raw[c + 1]) * r4.y;
-                                v[c4 * 4 + 2] = __uint_as_float(raw[c + 2]) * r4.z;
-                                v[c4 * 4 + 3] = __uint_as_float(raw[c + 3]) * r4.w;
-                            }
-                            if (col_limit < kTile) {
-#pragma unroll
-                                for (int c = 0; c < 16; ++c) if (g16 * 16 + c >= col_limit) v[c] = -INFINITY;
-                            }
-                            float mx = v[0];
-#pragma unroll
-                            for (int c = 1; c < 16; ++c) mx = fmaxf(mx, v[c]);
-                            if (mx > best) {                  // strict: an equal value keeps the lower slot
-                                best = mx;
-                                int idx = 15;
-#pragma unroll
-                                for (int c = 14; c >= 0; --c) if (v[c] == mx) idx = c;
-                                best_slot = t * kTile + g16 * 16 + idx;
+                            for (int q = 0; q < 4; ++q) {
+                                const int c = c4 * 4 + q;
+                                const float v = __uint_as_float(raw[c]) * rn[q];
+                                if (c0 + c < col_limit && v > best) { best = v; best_slot = slot0 + c; }
                             }
                         }
                     }
                 }
                 ptx::tc_fence_before_sync();
                 __syncwarp();
-                if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&sh.t_empty[par]));
+                if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&sh.t_empty[buf]));
             }
 
-            // ---- this thread's row is complete: write the item's result --------------------------
-            if (pos < it.L && !*abort_flag) {
+            // ---- combine the four groups and write this item's results -----------------------
+            if (wg > 0) {
+                float* cb0 = sh.comb[n & 1][wg - 1][0];
+                float* cb1 = sh.comb[n & 1][wg - 1][1];
+                if (KIND == kSweep1) { cb0[row] = m_run; cb1[row] = l_run; }
+                else if (KIND == kSweep2) { cb0[row] = (acc0 + acc1) + (acc2 + acc3); }
+                else { cb0[row] = best; cb1[row] = __int_as_float(best_slot); }
+            }
+            ptx::named_barrier_sync(1 + kGroups, kGroups * 128);
+            if (wg == 0 && pos < it.L && !*abort_flag) {
                 if (KIND == kSweep1) {
+                    float m = m_run;
+#pragma unroll
+                    for (int g = 0; g < kGroups - 1; ++g) m = fmaxf(m, sh.comb[n & 1][g][0][row]);
+                    float l = l_run * ptx::ex2((m_run - m) * c2);
+#pragma unroll
+                    for (int g = 0; g < kGroups - 1; ++g)
+                        l += sh.comb[n & 1][g][1][row] * ptx::ex2((sh.comb[n & 1][g][0][row] - m) * c2);
                     // natural-log log-sum-exp of the scaled logits
-                    p.lse[(long long)it.head * p.T + it.tok_begin + pos] = (m_run * c2 + ptx::lg2(l_run)) * kLn2;
+                    p.lse[(long long)it.head * p.T + it.tok_begin + pos] = (m * c2 + ptx::lg2(l)) * kLn2;
                 } else if (KIND == kSweep2) {
-                    p.scores[(long long)it.head * p.T + it.tok_begin + pos] = (acc0 + acc1) + (acc2 + acc3);
+                    float a = (acc0 + acc1) + (acc2 + acc3);
+#pragma unroll
+                    for (int g = 0; g < kGroups - 1; ++g) a += sh.comb[n & 1][g][0][row];
+                    p.scores[(long long)it.head * p.T + it.tok_begin + pos] = a;
                 } else {
                     const long long g = (long long)it.head * p.T + it.tok_begin + pos;
                     const int e = p.rank[g];
                     if (e >= 0) {
+#pragma unroll
+                        for (int gi = 0; gi < kGroups - 1; ++gi) {
+                            const float b1 = sh.comb[n & 1][gi][0][row];
+                            const int s1 = __float_as_int(sh.comb[n & 1][gi][1][row]);
+                            if (b1 > best || (b1 == best && s1 < best_slot)) { best = b1; best_slot = s1; }
+                        }
                         p.assign[it.ev0 + e] = best_slot;
                         p.sim[it.ev0 + e] = best * p.rnorm_all[g];
                     }
