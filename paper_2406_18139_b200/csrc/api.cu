@@ -30,11 +30,12 @@ struct Plan {
     int max_L = 0, max_E = 0;
     int n_items[3] = {0, 0, 0};
     long long total_slots = 0;              // n_kv_heads * sum_B
+    long long total_units = 0, unit_ints = 0;  // merge work units; ints in their boundary arrays
     std::vector<Req> reqs;                  // table order (longest first)
     std::vector<int> out_len;               // caller order
     // workspace offsets (bytes)
     size_t o_status, o_reqs, o_lse, o_scores, o_rank, o_rnorm_all, o_kept, o_evict, o_kept_keys,
-        o_rnorm_kept, o_assign, o_sim, o_row_ptr, o_members, o_member_w, o_sort_a, o_sort_b, total;
+        o_rnorm_kept, o_assign, o_sim, o_row_ptr, o_members, o_member_w, o_units, o_sort_a, o_sort_b, total;
 };
 
 // Returns LOOKM_OK or the status describing the first bad argument.
@@ -91,17 +92,23 @@ int build_plan(Plan& pl, const lookm_layout* lay, int n_req, const int* cu_seqle
         return LOOKM_ERR_UNSUPPORTED;
     // table order: longest request first
     std::stable_sort(pl.reqs.begin(), pl.reqs.end(), [](const Req& a, const Req& b) { return a.L > b.L; });
-    long long it0 = 0, it1 = 0, it2 = 0, slots = 0;
+    long long it0 = 0, it1 = 0, it2 = 0, slots = 0, units = 0, unit_ints = 0;
     for (Req& q : pl.reqs) {
         q.item_begin[kSweep1] = (int)it0;
         q.item_begin[kSweep2] = (int)it1;
         q.item_begin[kMatch] = (int)it2;
         q.slot_begin = (int)slots;
+        q.unit_begin = (int)units;
+        q.unit_store = unit_ints;
+        units += (long long)pl.n_kv_heads * ((q.L + 63) / 64);
+        unit_ints += (long long)pl.n_kv_heads * ((q.L + 63) / 64 + 1);
         it0 += (long long)q.nblk * pl.n_q_heads;
         it1 += (long long)q.nblk * pl.n_kv_heads;
         it2 += q.E > 0 ? (long long)q.nblk * pl.n_kv_heads : 0;
         slots += (long long)q.B * pl.n_kv_heads;
     }
+    pl.total_units = units;
+    pl.unit_ints = unit_ints;
     pl.n_items[kSweep1] = (int)it0;
     pl.n_items[kSweep2] = (int)it1;
     pl.n_items[kMatch] = (int)it2;
@@ -126,6 +133,7 @@ int build_plan(Plan& pl, const lookm_layout* lay, int n_req, const int* cu_seqle
     pl.o_row_ptr = carve(4 * (Hkv * T + Hkv * (size_t)n_req));
     pl.o_members = carve(4 * Hkv * T);
     pl.o_member_w = carve(4 * Hkv * T);
+    pl.o_units = carve(4 * Hkv * (T / 64 + 2 * (size_t)n_req));
     pl.o_sort_a = carve(8 * Hkv * T);
     pl.o_sort_b = carve(8 * Hkv * T);
     pl.total = o;
@@ -316,16 +324,19 @@ int run_merge(const Plan& pl, const lookm_layout* lay, const void* k, const void
               int varlen_output, void* out_k, void* out_v, void* ws, cudaStream_t st) {
     const Req* reqs = at<Req>(ws, pl.o_reqs);
     int* status = at<int>(ws, pl.o_status);
-    LOOKM_CUDA(launch_invert_assignment(assign, evict_idx, sim, reqs, pl.n_req, pl.n_kv_heads,
-                                        at<int>(ws, pl.o_row_ptr), at<int>(ws, pl.o_members),
-                                        at<float>(ws, pl.o_member_w), at<unsigned>(ws, pl.o_sort_a),
-                                        at<unsigned>(ws, pl.o_sort_b), status, st));
+    LOOKM_CUDA(launch_invert_assignment(assign, kept_idx, evict_idx, sim, reqs, pl.n_req, pl.n_kv_heads,
+                                        pl.T, at<int>(ws, pl.o_row_ptr), at<int>(ws, pl.o_members),
+                                        at<float>(ws, pl.o_member_w), at<int>(ws, pl.o_units),
+                                        at<unsigned>(ws, pl.o_sort_a), at<unsigned>(ws, pl.o_sort_b),
+                                        status, st));
     ++g_launches;
     mark_stage(6, st);
+    DeviceInfo di;
+    LOOKM_TRY(device_info(di));
     LOOKM_CUDA(launch_merge(k, v, lay->kv_stride_tok, lay->kv_stride_head, reqs, pl.n_req,
-                            pl.n_kv_heads, pl.T, pl.total_slots, kept_idx,
-                            at<int>(ws, pl.o_row_ptr), at<int>(ws, pl.o_members),
-                            at<float>(ws, pl.o_member_w), varlen_output, out_k, out_v, status, st));
+                            pl.n_kv_heads, pl.T, pl.total_units, at<int>(ws, pl.o_row_ptr),
+                            at<int>(ws, pl.o_members), at<float>(ws, pl.o_member_w),
+                            at<int>(ws, pl.o_units), varlen_output, out_k, out_v, status, di.sms, st));
     ++g_launches;
     mark_stage(7, st);
     return LOOKM_OK;
@@ -610,6 +621,7 @@ extern "C" int lookm_merge_noalloc(const void* k, const void* v, const int* kept
     pl.o_row_ptr = carve(4 * (units + (size_t)pl.n_kv_heads * (size_t)n_requests));
     pl.o_members = carve(4 * units);
     pl.o_member_w = carve(4 * units);
+    pl.o_units = carve(4 * ((size_t)pl.n_kv_heads * ((size_t)pl.T / 64 + 2 * (size_t)n_requests)));
     pl.o_sort_a = carve(8 * units);
     pl.o_sort_b = carve(8 * units);
     pl.total = o;

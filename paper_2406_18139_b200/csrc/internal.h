@@ -30,6 +30,9 @@ struct Req {
                           // which hold B + 1 entries per head
     int item_begin[3];    // first work item of this request in sweep 1 / sweep 2 / match order
     int slot_begin;       // first (head, slot) row of this request in merge order (table order)
+    int unit_begin;       // first merge work unit of this request (table order); a unit is
+                          // about kUnitEntries = 64 rows to read, n_kv_heads * ceil(L / 64) per request
+    long long unit_store; // start of its unit-boundary arrays (ceil(L / 64) + 1 ints per head)
 };
 
 enum TileKind { kSweep1 = 0, kSweep2 = 1, kMatch = 2 };
@@ -81,15 +84,16 @@ constexpr int kReqChunk = 40;
 struct ReqChunk { Req r[kReqChunk]; };
 cudaError_t launch_write_table(const ReqChunk& chunk, int count, Req* dst, cudaStream_t stream);
 
-cudaError_t launch_invert_assignment(const int* assign, const int* evict_idx, const float* sim,
-                                     const Req* reqs, int n_req, int n_kv_heads, int* row_ptr,
-                                     int* member_pos, float* member_w, unsigned* sort_a,
-                                     unsigned* sort_b, int* status, cudaStream_t stream);
+cudaError_t launch_invert_assignment(const int* assign, const int* kept_idx, const int* evict_idx,
+                                     const float* sim, const Req* reqs, int n_req, int n_kv_heads,
+                                     long long T, int* row_ptr, int* ent_pos, float* ent_w,
+                                     int* unit_slot, unsigned* sort_a, unsigned* sort_b, int* status,
+                                     cudaStream_t stream);
 
 cudaError_t launch_merge(const void* k, const void* v, long long stride_tok, long long stride_head,
                          const Req* reqs, int n_req, int n_kv_heads, long long T,
-                         long long total_kept_rows, const int* kept_idx, const int* row_ptr,
-                         const int* member_pos, const float* member_w, int varlen_output,
-                         void* out_k, void* out_v, int* status, cudaStream_t stream);
+                         long long total_units, const int* row_ptr, const int* ent_pos,
+                         const float* ent_w, const int* unit_slot, int varlen_output, void* out_k,
+                         void* out_v, int* status, int num_sms, cudaStream_t stream);
 
 }  // namespace lookm

@@ -129,12 +129,36 @@ argmax_rows_kernel(const float* __restrict__ sim_matrix, const Req* __restrict__
 // earlier warps.  Keys are packed as (slot << 0) in one array and values in the other.
 // ---------------------------------------------------------------------------------------------
 constexpr int kInvThreads = 1024;
+constexpr int kUnitEntries = 64;     // entries (rows to read) per work unit of the merge kernel
+
+// Second half of the entry list: the kept rows (flagged with the sign bit, weight = member count)
+// and the work-unit boundaries: unit u covers the slots [units[u], units[u+1]), where units[u] is
+// the first slot whose entry index c + row_ptr[c] is >= u * kUnitEntries.
+__device__ __forceinline__ void write_kept_entries(const Req& rq, int h, int B, int E, const int* rp,
+                                                   const int* kept_idx_head, int* ent, float* entw,
+                                                   int* units, int* status) {
+    const int n_units = (rq.L + kUnitEntries - 1) / kUnitEntries;
+    for (int c = threadIdx.x; c < B; c += blockDim.x) {
+        int pc = kept_idx_head[c];
+        if (pc < 0 || pc >= rq.L) { atomicExch(status, (int)LOOKM_ERR_DEVICE_BAD_INDEX); pc = 0; }
+        const int s_c = c + rp[c];
+        ent[s_c] = pc | (int)0x80000000;
+        entw[s_c] = (float)(rp[c + 1] - rp[c]);
+        const int s_prev = c ? (c - 1) + rp[c - 1] : -1;
+        for (int u = s_prev / kUnitEntries + (s_prev >= 0 ? 1 : 0); u * kUnitEntries <= s_c; ++u) units[u] = c;
+        if (c == B - 1)
+            for (int u = s_c / kUnitEntries + 1; u <= n_units; ++u) units[u] = B;
+    }
+    (void)h; (void)E;
+}
 
 __global__ void __launch_bounds__(kInvThreads)
-invert_assignment_kernel(const int* __restrict__ assign, const int* __restrict__ evict_idx,
+invert_assignment_kernel(const int* __restrict__ assign, const int* __restrict__ kept_idx,
+                         const int* __restrict__ evict_idx,
                          const float* __restrict__ sim, const Req* __restrict__ reqs,
-                         int n_kv_heads, int* __restrict__ row_ptr, int* __restrict__ member_pos,
-                         float* __restrict__ member_w, unsigned* __restrict__ sort_a,
+                         int n_kv_heads, long long T, int* __restrict__ row_ptr,
+                         int* __restrict__ ent_pos, float* __restrict__ ent_w,
+                         int* __restrict__ unit_slot, unsigned* __restrict__ sort_a,
                          unsigned* __restrict__ sort_b, int* status) {
     __shared__ int cnt[32][256];                         // [warp][digit]
     __shared__ int digit_tot[256];
@@ -146,8 +170,17 @@ invert_assignment_kernel(const int* __restrict__ assign, const int* __restrict__
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const unsigned lt_mask = (1u << lane) - 1u;
 
+    // entry list of this (request, head): for every kept slot its kept row, then its members
+    int* ent = ent_pos + (long long)h * T + rq.tok_begin;
+    float* entw = ent_w + (long long)h * T + rq.tok_begin;
+    const int n_units = (rq.L + kUnitEntries - 1) / kUnitEntries;
+    int* units = unit_slot + rq.unit_store + (long long)h * (n_units + 1);
+    const int* kept_idx_head = kept_idx + rq.kept_off + (long long)h * B;
+    const bool weighted = (rq.mode == LOOKM_MERGE_WEIGHTED);
     if (E == 0) {
         for (int c = threadIdx.x; c <= B; c += kInvThreads) rp[c] = 0;
+        __syncthreads();
+        write_kept_entries(rq, h, B, E, rp, kept_idx_head, ent, entw, units, status);
         return;
     }
     // segment of the list owned by each warp: a multiple of 32 elements
@@ -226,117 +259,212 @@ invert_assignment_kernel(const int* __restrict__ assign, const int* __restrict__
     }
     const unsigned* fin_k = key_buf[(n_pass - 1) & 1];
     const unsigned* fin_v = fin_k + E;
-    // members and the row boundaries: row_ptr[c] = first sorted index whose slot is >= c
+    // member entries and the row boundaries: row_ptr[c] = first sorted index whose slot is >= c
     for (int i = threadIdx.x; i < E; i += kInvThreads) {
         const int e = (int)fin_v[i];
         int pe = evict_idx[ev_base + e];
         if (pe < 0 || pe >= rq.L) { atomicExch(status, (int)LOOKM_ERR_DEVICE_BAD_INDEX); pe = 0; }
-        member_pos[ev_base + i] = pe;                    // position of the i-th member in row order
-        member_w[ev_base + i] = sim[ev_base + e];        // its cosine with the kept row (Eq. 12 weight)
         const int cur = (int)fin_k[i];
+        ent[i + cur + 1] = pe;                           // i-th member sits after cur + 1 kept rows
+        entw[i + cur + 1] = weighted ? sim[ev_base + e] : 1.0f;
         const int prev = i ? (int)fin_k[i - 1] : -1;
         for (int c = prev + 1; c <= cur; ++c) rp[c] = i;
         if (i == E - 1) for (int c = cur + 1; c <= B; ++c) rp[c] = E;
     }
+    __syncthreads();
+    write_kept_entries(rq, h, B, E, rp, kept_idx_head, ent, entw, units, status);
 }
 
 // ---------------------------------------------------------------------------------------------
-// Merge + compact: one warp per kept row (lanes 0-15 the K row, 16-31 the V row).  The lanes fetch
-// the row's metadata and up to 32 member positions / weights with one coalesced load each, then
-// the warp gathers the member rows eight at a time (eight 16-byte loads in flight per lane),
-// accumulates in fp32 in member order and rounds once.
+// Merge + compact (Eq. 6-7, 10-12).  Every K and V row of the prompt is read exactly once: the
+// entry list of a (request, head) names, slot by slot, the kept row and then its members.  A warp
+// takes a work unit of about 64 consecutive entries (whole slots), fetches the rows 16 entries at
+// a time with bulk async copies into its own shared-memory ring (256 bytes per row and tensor, two
+// buffers, completion on an mbarrier), and walks the staged rows in order: lanes 0-15 hold the K
+// row, lanes 16-31 the V row, 16 bytes per lane, fp32 accumulation in member order, one rounding.
 //   averaged : (x_c + sum x_e) / (n + 1)                       (Eq. 10)
 //   pivotal  : (x_c + 1/2 sum (x_e + x_c)) / (n + 1)           (Eq. 11)
 //   weighted : (x_c + sum sim_e x_e) / (n + 1)                 (Eq. 12)
-// A row without members is copied bit for bit.
+// A row without members is copied bit for bit.  With 8 KB of copies in flight per warp the kernel
+// is bound by HBM, not by the latency of the dependent index loads.
 // ---------------------------------------------------------------------------------------------
 constexpr int kMergeWarps = 8;
+constexpr int kChunk = 16;                           // entries staged per buffer
+constexpr int kRowBytes = kHeadDim * 2;              // one bf16 row of K or V
 
-__device__ __forceinline__ uint4 ld_stream(const __nv_bfloat16* p) {
-    uint4 r;
-    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0, %1, %2, %3}, [%4];"
-                 : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "l"(p));
-    return r;
+struct MergeShared {
+    alignas(128) uint8_t rows[kMergeWarps][2][kChunk][2 * kRowBytes];   // [warp][buffer][entry][K|V]
+    unsigned long long bar[kMergeWarps][2];
+};
+
+__device__ __forceinline__ const Req& find_req_by_unit(const Req* reqs, int n_req, long long g) {
+    int lo = 0, hi = n_req - 1;
+    while (lo < hi) {
+        const int mid = (lo + hi + 1) >> 1;
+        if ((long long)reqs[mid].unit_begin <= g) lo = mid; else hi = mid - 1;
+    }
+    return reqs[lo];
 }
 
 __global__ void __launch_bounds__(kMergeWarps * 32)
 merge_kernel(const __nv_bfloat16* __restrict__ k, const __nv_bfloat16* __restrict__ v,
              long long stride_tok, long long stride_head, const Req* __restrict__ reqs, int n_req,
-             int n_kv_heads, long long total_rows, const int* __restrict__ kept_idx,
-             const int* __restrict__ row_ptr, const int* __restrict__ member_pos,
-             const float* __restrict__ member_w, int varlen_output,
+             int n_kv_heads, long long T, long long total_units, const int* __restrict__ row_ptr,
+             const int* __restrict__ ent_pos, const float* __restrict__ ent_w,
+             const int* __restrict__ unit_slot, int varlen_output,
              __nv_bfloat16* __restrict__ out_k, __nv_bfloat16* __restrict__ out_v, int* status) {
+    extern __shared__ uint8_t merge_smem_raw[];
+    MergeShared& sh = *reinterpret_cast<MergeShared*>(
+        (reinterpret_cast<uintptr_t>(merge_smem_raw) + 127) & ~static_cast<uintptr_t>(127));
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const long long g = (long long)blockIdx.x * kMergeWarps + warp;
-    if (g >= total_rows) return;
-    const Req& rq = find_req_by_slot(reqs, n_req, g);
-    const long long u = g - rq.slot_begin;
-    const int B = rq.B, L = rq.L, mode = rq.mode;
-    const int h = (int)(u / B), slot = (int)(u % B);
     const int l16 = lane & 15;
-    const __nv_bfloat16* src = (lane < 16 ? k : v) + (long long)rq.tok_begin * stride_tok +
-                               (long long)h * stride_head + l16 * 8;
-    const long long kept_base = rq.kept_off + (long long)h * B;
-    const long long ev_base = rq.ev_off + (long long)h * rq.E;
-    const int* rp = row_ptr + rq.rp_off + (long long)h * (B + 1);
+    if (lane < 2) {
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;"
+                     ::"r"((uint32_t)__cvta_generic_to_shared(&sh.bar[warp][lane])) : "memory");
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    __syncthreads();
+    const uint32_t bar0 = (uint32_t)__cvta_generic_to_shared(&sh.bar[warp][0]);
+    const uint32_t buf0 = (uint32_t)__cvta_generic_to_shared(&sh.rows[warp][0][0][0]);
+    const __nv_bfloat16* tensor = lane < 16 ? k : v;
+    __nv_bfloat16* dst_base = lane < 16 ? out_k : out_v;
+    uint32_t n_chunks_done = 0;                      // chunks this warp has consumed (barrier phases)
+    bool failed = false;
 
-    // lane 0: kept position, lane 1: first member, lane 2: one past the last member
-    int meta = 0;
-    if (lane == 0) meta = kept_idx[kept_base + slot];
-    else if (lane <= 2) meta = rp[slot + lane - 1];
-    int pos_c = __shfl_sync(0xffffffffu, meta, 0);
-    const int m_begin = __shfl_sync(0xffffffffu, meta, 1);
-    const int m_end = __shfl_sync(0xffffffffu, meta, 2);
-    if (pos_c < 0 || pos_c >= L) { if (lane == 0) atomicExch(status, (int)LOOKM_ERR_DEVICE_BAD_INDEX); pos_c = 0; }
-    const uint4 raw_c = ld_stream(src + (long long)pos_c * stride_tok);
-    const int n = m_end - m_begin;
-    uint4 result = raw_c;
-    if (n > 0) {
-        const bool weighted = (mode == LOOKM_MERGE_WEIGHTED);
+    for (long long g = (long long)blockIdx.x * kMergeWarps + warp; g < total_units && !failed;
+         g += (long long)gridDim.x * kMergeWarps) {
+        const Req& rq = find_req_by_unit(reqs, n_req, g);
+        const int L = rq.L, B = rq.B, mode = rq.mode;
+        const int n_units = (L + kUnitEntries - 1) / kUnitEntries;
+        const long long ul = g - rq.unit_begin;
+        const int h = (int)(ul / n_units), u = (int)(ul % n_units);
+        const int* units = unit_slot + rq.unit_store + (long long)h * (n_units + 1);
+        const int* rp = row_ptr + rq.rp_off + (long long)h * (B + 1);
+        // lanes 0/1: first slot / one past the last slot of the unit, and their entry indices
+        int c_edge = 0, e_edge = 0;
+        if (lane < 2) {
+            c_edge = units[u + lane];
+            e_edge = c_edge + rp[c_edge];
+        }
+        const int c_lo = __shfl_sync(0xffffffffu, c_edge, 0), c_hi = __shfl_sync(0xffffffffu, c_edge, 1);
+        const int e_lo = __shfl_sync(0xffffffffu, e_edge, 0), e_hi = __shfl_sync(0xffffffffu, e_edge, 1);
+        if (c_lo >= c_hi) continue;
+        const int* ent = ent_pos + (long long)h * T + rq.tok_begin;
+        const float* entw = ent_w + (long long)h * T + rq.tok_begin;
+        const __nv_bfloat16* src = tensor + (long long)rq.tok_begin * stride_tok + (long long)h * stride_head;
+        const int n_chunks = (e_hi - e_lo + kChunk - 1) / kChunk;
+
+        // entry metadata of a chunk (lanes 0-15: one entry each)
+        auto load_meta = [&](int kc, int& pos, float& w) {
+            pos = 0;
+            w = 0.f;
+            const int e = e_lo + kc * kChunk + l16;
+            if (kc < n_chunks && e < e_hi) { pos = ent[e]; w = entw[e]; }
+        };
+        // start the row copies of chunk kc (lane l < 16: K row of entry l, lane l + 16: V row)
+        auto issue = [&](int kc, int pos) {
+            const int cnt = min(kChunk, e_hi - e_lo - kc * kChunk);
+            const uint32_t b = (n_chunks_done + (uint32_t)kc) & 1u;
+            const uint32_t bar = bar0 + 8u * b;
+            if (lane == 0)
+                asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;"
+                             ::"r"(bar), "r"((uint32_t)(cnt * 2 * kRowBytes)) : "memory");
+            __syncwarp();
+            if (l16 < cnt) {
+                const int tok = pos & 0x7fffffff;
+                const uint32_t dst = buf0 + b * (kChunk * 2 * kRowBytes) + l16 * (2 * kRowBytes) +
+                                     (lane < 16 ? 0 : kRowBytes);
+                asm volatile(
+                    "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                    ::"r"(dst), "l"(reinterpret_cast<uint64_t>(src + (long long)tok * stride_tok)),
+                      "r"((uint32_t)kRowBytes), "r"(bar) : "memory");
+            }
+        };
+
+        int pos_a, pos_b;
+        float w_a, w_b;
+        load_meta(0, pos_a, w_a);
+        issue(0, __shfl_sync(0xffffffffu, pos_a, l16));
+        load_meta(1, pos_b, w_b);
+
+        // running row
+        int slot = c_lo - 1, n_mem = 0;
+        uint4 raw_c = make_uint4(0u, 0u, 0u, 0u);
         float acc[8];
 #pragma unroll
         for (int i = 0; i < 8; ++i) acc[i] = 0.f;
-        for (int m0 = m_begin; m0 < m_end; m0 += 32) {
-            const int cnt = min(32, m_end - m0);
-            int my_pos = 0;
-            float my_w = 1.f;
-            if (lane < cnt) {
-                my_pos = member_pos[ev_base + m0 + lane];
-                if (weighted) my_w = member_w[ev_base + m0 + lane];
+        auto flush = [&]() {
+            if (slot < c_lo) return;
+            uint4 result = raw_c;
+            if (n_mem > 0) {
+                const Row8 xc = unpack8(raw_c);
+                const float inv = 1.0f / (float)(n_mem + 1);
+                // pivotal: each member contributes (x_e + x_c) / 2
+                const float wc = (mode == LOOKM_MERGE_PIVOTAL) ? 1.f + 0.5f * (float)n_mem : 1.f;
+                const float wm = (mode == LOOKM_MERGE_PIVOTAL) ? 0.5f : 1.f;
+                Row8 o;
+#pragma unroll
+                for (int i = 0; i < 8; ++i) o.v[i] = fmaf(wc, xc.v[i], wm * acc[i]) * inv;
+                result = pack8(o);
             }
-            for (int q0 = 0; q0 < cnt; q0 += 8) {
-                uint4 raw[8];
-                float w[8];
-#pragma unroll
-                for (int q = 0; q < 8; ++q) {
-                    const int pe = __shfl_sync(0xffffffffu, my_pos, (q0 + q) & 31);
-                    w[q] = __shfl_sync(0xffffffffu, my_w, (q0 + q) & 31);
-                    if (q0 + q < cnt) raw[q] = ld_stream(src + (long long)pe * stride_tok);
-                    else { raw[q] = make_uint4(0u, 0u, 0u, 0u); w[q] = 0.f; }
+            long long row;
+            if (varlen_output) row = ((long long)rq.out_begin + slot) * n_kv_heads + h;
+            else row = (long long)h * B + slot;
+            *reinterpret_cast<uint4*>(dst_base + row * kHeadDim + l16 * 8) = result;
+        };
+
+        for (int kc = 0; kc < n_chunks; ++kc) {
+            // next chunk's copies go to the other buffer, whose rows were consumed one iteration ago
+            if (kc + 1 < n_chunks) {
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                issue(kc + 1, __shfl_sync(0xffffffffu, pos_b, l16));
+            }
+            int pos_c;
+            float w_c;
+            load_meta(kc + 2, pos_c, w_c);
+            // wait for this chunk's rows (bounded)
+            const uint32_t b = (n_chunks_done + (uint32_t)kc) & 1u;
+            const uint32_t parity = ((n_chunks_done + (uint32_t)kc) >> 1) & 1u;
+            {
+                uint32_t ok = 0;
+                for (uint32_t spin = 0; spin < 4000000u && !ok; ++spin) {
+                    asm volatile(
+                        "{\n\t.reg .pred p;\n\t"
+                        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+                        "selp.u32 %0, 1, 0, p;\n\t}"
+                        : "=r"(ok) : "r"(bar0 + 8u * b), "r"(parity) : "memory");
                 }
+                if (!ok) { failed = true; }
+                failed = __any_sync(0xffffffffu, failed);
+                if (failed) break;
+            }
+            const int cnt = min(kChunk, e_hi - e_lo - kc * kChunk);
+            const uint8_t* base = &sh.rows[warp][b][0][0] + lane * 16;
+            for (int q = 0; q < cnt; ++q) {
+                const int pe = __shfl_sync(0xffffffffu, pos_a, q);
+                const float w = __shfl_sync(0xffffffffu, w_a, q);
+                const uint4 x4 = *reinterpret_cast<const uint4*>(base + q * (2 * kRowBytes));
+                if (pe < 0) {                        // a kept row starts the next slot
+                    flush();
+                    ++slot;
+                    raw_c = x4;
+                    n_mem = (int)w;
 #pragma unroll
-                for (int q = 0; q < 8; ++q) {
-                    const Row8 x = unpack8(raw[q]);
+                    for (int i = 0; i < 8; ++i) acc[i] = 0.f;
+                } else {
+                    const Row8 x = unpack8(x4);
 #pragma unroll
-                    for (int i = 0; i < 8; ++i) acc[i] = fmaf(w[q], x.v[i], acc[i]);
+                    for (int i = 0; i < 8; ++i) acc[i] = fmaf(w, x.v[i], acc[i]);
                 }
             }
+            __syncwarp();
+            pos_a = pos_b; w_a = w_b;
+            pos_b = pos_c; w_b = w_c;
         }
-        const Row8 xc = unpack8(raw_c);
-        const float inv = 1.0f / (float)(n + 1);
-        // pivotal: each member contributes (x_e + x_c) / 2
-        const float wc = (mode == LOOKM_MERGE_PIVOTAL) ? 1.f + 0.5f * (float)n : 1.f;
-        const float wm = (mode == LOOKM_MERGE_PIVOTAL) ? 0.5f : 1.f;
-        Row8 o;
-#pragma unroll
-        for (int i = 0; i < 8; ++i) o.v[i] = fmaf(wc, xc.v[i], wm * acc[i]) * inv;
-        result = pack8(o);
+        if (!failed) flush();
+        n_chunks_done += (uint32_t)n_chunks;
     }
-    __nv_bfloat16* dst_base = lane < 16 ? out_k : out_v;
-    long long row;
-    if (varlen_output) row = ((long long)rq.out_begin + slot) * n_kv_heads + h;
-    else row = (long long)h * B + slot;
-    *reinterpret_cast<uint4*>(dst_base + row * kHeadDim + l16 * 8) = result;
+    if (failed && lane == 0) atomicExch(status, (int)LOOKM_ERR_DEVICE_TIMEOUT);
 }
 
 // Inverse map of given kept / evicted lists (used when the lists come from the caller).
@@ -401,28 +529,32 @@ cudaError_t launch_gather_kept(const void* k, long long stride_tok, long long st
     return cudaGetLastError();
 }
 
-cudaError_t launch_invert_assignment(const int* assign, const int* evict_idx, const float* sim,
-                                     const Req* reqs, int n_req, int n_kv_heads, int* row_ptr,
-                                     int* member_pos, float* member_w, unsigned* sort_a,
-                                     unsigned* sort_b, int* status, cudaStream_t stream) {
+cudaError_t launch_invert_assignment(const int* assign, const int* kept_idx, const int* evict_idx,
+                                     const float* sim, const Req* reqs, int n_req, int n_kv_heads,
+                                     long long T, int* row_ptr, int* ent_pos, float* ent_w,
+                                     int* unit_slot, unsigned* sort_a, unsigned* sort_b, int* status,
+                                     cudaStream_t stream) {
     dim3 grid(n_kv_heads, n_req);
-    invert_assignment_kernel<<<grid, kInvThreads, 0, stream>>>(assign, evict_idx, sim, reqs, n_kv_heads,
-                                                               row_ptr, member_pos, member_w, sort_a,
-                                                               sort_b, status);
+    invert_assignment_kernel<<<grid, kInvThreads, 0, stream>>>(assign, kept_idx, evict_idx, sim, reqs,
+                                                               n_kv_heads, T, row_ptr, ent_pos, ent_w,
+                                                               unit_slot, sort_a, sort_b, status);
     return cudaGetLastError();
 }
 
 cudaError_t launch_merge(const void* k, const void* v, long long stride_tok, long long stride_head,
                          const Req* reqs, int n_req, int n_kv_heads, long long T,
-                         long long total_kept_rows, const int* kept_idx, const int* row_ptr,
-                         const int* member_pos, const float* member_w, int varlen_output,
-                         void* out_k, void* out_v, int* status, cudaStream_t stream) {
-    (void)T;
-    if (total_kept_rows <= 0) return cudaSuccess;
-    const long long blocks = (total_kept_rows + kMergeWarps - 1) / kMergeWarps;
-    merge_kernel<<<(unsigned)blocks, kMergeWarps * 32, 0, stream>>>(
+                         long long total_units, const int* row_ptr, const int* ent_pos,
+                         const float* ent_w, const int* unit_slot, int varlen_output, void* out_k,
+                         void* out_v, int* status, int num_sms, cudaStream_t stream) {
+    if (total_units <= 0) return cudaSuccess;
+    const int smem = (int)sizeof(MergeShared) + 128;
+    cudaError_t err = cudaFuncSetAttribute(merge_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (err != cudaSuccess) return err;
+    long long blocks = (total_units + kMergeWarps - 1) / kMergeWarps;
+    if (blocks > num_sms) blocks = num_sms;              // persistent: one CTA per SM
+    merge_kernel<<<(unsigned)blocks, kMergeWarps * 32, smem, stream>>>(
         (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, stride_tok, stride_head, reqs, n_req,
-        n_kv_heads, total_kept_rows, kept_idx, row_ptr, member_pos, member_w, varlen_output,
+        n_kv_heads, T, total_units, row_ptr, ent_pos, ent_w, unit_slot, varlen_output,
         (__nv_bfloat16*)out_k, (__nv_bfloat16*)out_v, status);
     return cudaGetLastError();
 }
