@@ -279,9 +279,10 @@ invert_assignment_kernel(const int* __restrict__ assign, const int* __restrict__
 // Merge + compact (Eq. 6-7, 10-12).  Every K and V row of the prompt is read exactly once: the
 // entry list of a (request, head) names, slot by slot, the kept row and then its members.  A warp
 // takes a work unit of about 64 consecutive entries (whole slots), fetches the rows 16 entries at
-// a time with bulk async copies into its own shared-memory ring (256 bytes per row and tensor, two
-// buffers, completion on an mbarrier), and walks the staged rows in order: lanes 0-15 hold the K
-// row, lanes 16-31 the V row, 16 bytes per lane, fp32 accumulation in member order, one rounding.
+// a time with 16-byte cp.async copies into its own shared-memory ring (two buffers; every lane
+// later reads back exactly the bytes it copied, so cp.async.wait_group is all the synchronisation
+// needed), and walks the staged rows in order: lanes 0-15 hold the K row, lanes 16-31 the V row,
+// 16 bytes per lane, fp32 accumulation in member order, one rounding.
 //   averaged : (x_c + sum x_e) / (n + 1)                       (Eq. 10)
 //   pivotal  : (x_c + 1/2 sum (x_e + x_c)) / (n + 1)           (Eq. 11)
 //   weighted : (x_c + sum sim_e x_e) / (n + 1)                 (Eq. 12)
@@ -294,7 +295,6 @@ constexpr int kRowBytes = kHeadDim * 2;              // one bf16 row of K or V
 
 struct MergeShared {
     alignas(128) uint8_t rows[kMergeWarps][2][kChunk][2 * kRowBytes];   // [warp][buffer][entry][K|V]
-    unsigned long long bar[kMergeWarps][2];
 };
 
 __device__ __forceinline__ const Req& find_req_by_unit(const Req* reqs, int n_req, long long g) {
@@ -318,20 +318,12 @@ merge_kernel(const __nv_bfloat16* __restrict__ k, const __nv_bfloat16* __restric
         (reinterpret_cast<uintptr_t>(merge_smem_raw) + 127) & ~static_cast<uintptr_t>(127));
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int l16 = lane & 15;
-    if (lane < 2) {
-        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;"
-                     ::"r"((uint32_t)__cvta_generic_to_shared(&sh.bar[warp][lane])) : "memory");
-    }
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    __syncthreads();
-    const uint32_t bar0 = (uint32_t)__cvta_generic_to_shared(&sh.bar[warp][0]);
-    const uint32_t buf0 = (uint32_t)__cvta_generic_to_shared(&sh.rows[warp][0][0][0]);
+    const uint32_t buf0 = (uint32_t)__cvta_generic_to_shared(&sh.rows[warp][0][0][0]) + lane * 16;
     const __nv_bfloat16* tensor = lane < 16 ? k : v;
     __nv_bfloat16* dst_base = lane < 16 ? out_k : out_v;
-    uint32_t n_chunks_done = 0;                      // chunks this warp has consumed (barrier phases)
-    bool failed = false;
+    uint32_t n_chunks_done = 0;                      // chunks this warp has consumed (buffer parity)
 
-    for (long long g = (long long)blockIdx.x * kMergeWarps + warp; g < total_units && !failed;
+    for (long long g = (long long)blockIdx.x * kMergeWarps + warp; g < total_units;
          g += (long long)gridDim.x * kMergeWarps) {
         const Req& rq = find_req_by_unit(reqs, n_req, g);
         const int L = rq.L, B = rq.B, mode = rq.mode;
@@ -361,30 +353,24 @@ merge_kernel(const __nv_bfloat16* __restrict__ k, const __nv_bfloat16* __restric
             const int e = e_lo + kc * kChunk + l16;
             if (kc < n_chunks && e < e_hi) { pos = ent[e]; w = entw[e]; }
         };
-        // start the row copies of chunk kc (lane l < 16: K row of entry l, lane l + 16: V row)
+        // start the row copies of chunk kc: for every entry, lanes 0-15 copy its K row and lanes
+        // 16-31 its V row, 16 bytes each; one commit group per chunk
         auto issue = [&](int kc, int pos) {
             const int cnt = min(kChunk, e_hi - e_lo - kc * kChunk);
-            const uint32_t b = (n_chunks_done + (uint32_t)kc) & 1u;
-            const uint32_t bar = bar0 + 8u * b;
-            if (lane == 0)
-                asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;"
-                             ::"r"(bar), "r"((uint32_t)(cnt * 2 * kRowBytes)) : "memory");
-            __syncwarp();
-            if (l16 < cnt) {
-                const int tok = pos & 0x7fffffff;
-                const uint32_t dst = buf0 + b * (kChunk * 2 * kRowBytes) + l16 * (2 * kRowBytes) +
-                                     (lane < 16 ? 0 : kRowBytes);
-                asm volatile(
-                    "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                    ::"r"(dst), "l"(reinterpret_cast<uint64_t>(src + (long long)tok * stride_tok)),
-                      "r"((uint32_t)kRowBytes), "r"(bar) : "memory");
+            const uint32_t dst = buf0 + ((n_chunks_done + (uint32_t)kc) & 1u) * (kChunk * 2 * kRowBytes);
+            for (int q = 0; q < cnt; ++q) {
+                const int tok = __shfl_sync(0xffffffffu, pos, q) & 0x7fffffff;
+                asm volatile("cp.async.cg.shared.global [%0], [%1], 16;"
+                             ::"r"(dst + q * (2 * kRowBytes)), "l"(src + (long long)tok * stride_tok + l16 * 8)
+                             : "memory");
             }
+            asm volatile("cp.async.commit_group;" ::: "memory");
         };
 
         int pos_a, pos_b;
         float w_a, w_b;
         load_meta(0, pos_a, w_a);
-        issue(0, __shfl_sync(0xffffffffu, pos_a, l16));
+        issue(0, pos_a);
         load_meta(1, pos_b, w_b);
 
         // running row
@@ -415,29 +401,14 @@ merge_kernel(const __nv_bfloat16* __restrict__ k, const __nv_bfloat16* __restric
 
         for (int kc = 0; kc < n_chunks; ++kc) {
             // next chunk's copies go to the other buffer, whose rows were consumed one iteration ago
-            if (kc + 1 < n_chunks) {
-                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                issue(kc + 1, __shfl_sync(0xffffffffu, pos_b, l16));
-            }
+            if (kc + 1 < n_chunks) issue(kc + 1, pos_b);
             int pos_c;
             float w_c;
             load_meta(kc + 2, pos_c, w_c);
-            // wait for this chunk's rows (bounded)
+            // this chunk's copies: everything but the group just committed must have landed
+            if (kc + 1 < n_chunks) asm volatile("cp.async.wait_group 1;" ::: "memory");
+            else asm volatile("cp.async.wait_group 0;" ::: "memory");
             const uint32_t b = (n_chunks_done + (uint32_t)kc) & 1u;
-            const uint32_t parity = ((n_chunks_done + (uint32_t)kc) >> 1) & 1u;
-            {
-                uint32_t ok = 0;
-                for (uint32_t spin = 0; spin < 4000000u && !ok; ++spin) {
-                    asm volatile(
-                        "{\n\t.reg .pred p;\n\t"
-                        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-                        "selp.u32 %0, 1, 0, p;\n\t}"
-                        : "=r"(ok) : "r"(bar0 + 8u * b), "r"(parity) : "memory");
-                }
-                if (!ok) { failed = true; }
-                failed = __any_sync(0xffffffffu, failed);
-                if (failed) break;
-            }
             const int cnt = min(kChunk, e_hi - e_lo - kc * kChunk);
             const uint8_t* base = &sh.rows[warp][b][0][0] + lane * 16;
             for (int q = 0; q < cnt; ++q) {
@@ -461,10 +432,10 @@ merge_kernel(const __nv_bfloat16* __restrict__ k, const __nv_bfloat16* __restric
             pos_a = pos_b; w_a = w_b;
             pos_b = pos_c; w_b = w_c;
         }
-        if (!failed) flush();
+        flush();
         n_chunks_done += (uint32_t)n_chunks;
     }
-    if (failed && lane == 0) atomicExch(status, (int)LOOKM_ERR_DEVICE_TIMEOUT);
+    (void)status;
 }
 
 // Inverse map of given kept / evicted lists (used when the lists come from the caller).
