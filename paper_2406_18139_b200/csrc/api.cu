@@ -100,8 +100,9 @@ int build_plan(Plan& pl, const lookm_layout* lay, int n_req, const int* cu_seqle
         q.slot_begin = (int)slots;
         q.unit_begin = (int)units;
         q.unit_store = unit_ints;
-        units += (long long)pl.n_kv_heads * ((q.L + 63) / 64);
-        unit_ints += (long long)pl.n_kv_heads * ((q.L + 63) / 64 + 1);
+        const long long n_units = (q.L + kUnitEntries - 1) / kUnitEntries;
+        units += (long long)pl.n_kv_heads * n_units;
+        unit_ints += (long long)pl.n_kv_heads * (n_units + 1);
         it0 += (long long)q.nblk * pl.n_q_heads;
         it1 += (long long)q.nblk * pl.n_kv_heads;
         it2 += q.E > 0 ? (long long)q.nblk * pl.n_kv_heads : 0;
@@ -133,7 +134,7 @@ int build_plan(Plan& pl, const lookm_layout* lay, int n_req, const int* cu_seqle
     pl.o_row_ptr = carve(4 * (Hkv * T + Hkv * (size_t)n_req));
     pl.o_members = carve(4 * Hkv * T);
     pl.o_member_w = carve(4 * Hkv * T);
-    pl.o_units = carve(4 * Hkv * (T / 64 + 2 * (size_t)n_req));
+    pl.o_units = carve(4 * Hkv * (T / kUnitEntries + 2 * (size_t)n_req));
     pl.o_sort_a = carve(8 * Hkv * T);
     pl.o_sort_b = carve(8 * Hkv * T);
     pl.total = o;
@@ -621,7 +622,7 @@ extern "C" int lookm_merge_noalloc(const void* k, const void* v, const int* kept
     pl.o_row_ptr = carve(4 * (units + (size_t)pl.n_kv_heads * (size_t)n_requests));
     pl.o_members = carve(4 * units);
     pl.o_member_w = carve(4 * units);
-    pl.o_units = carve(4 * ((size_t)pl.n_kv_heads * ((size_t)pl.T / 64 + 2 * (size_t)n_requests)));
+    pl.o_units = carve(4 * ((size_t)pl.n_kv_heads * ((size_t)pl.T / kUnitEntries + 2 * (size_t)n_requests)));
     pl.o_sort_a = carve(8 * units);
     pl.o_sort_b = carve(8 * units);
     pl.total = o;

@@ -11,6 +11,7 @@ namespace lookm {
 
 constexpr int kTile = 128;      // tokens per tile on either operand of the tensor-core kernels
 constexpr int kHeadDim = 128;   // only supported head_dim
+constexpr int kUnitEntries = 32; // rows read per work unit of the merge kernel (whole slots)
 
 // One request of the packed batch as the kernels see it (device copy lives in the workspace).
 // Requests are stored longest first so that the heaviest work items are issued first.
@@ -31,8 +32,8 @@ struct Req {
     int item_begin[3];    // first work item of this request in sweep 1 / sweep 2 / match order
     int slot_begin;       // first (head, slot) row of this request in merge order (table order)
     int unit_begin;       // first merge work unit of this request (table order); a unit is
-                          // about kUnitEntries = 64 rows to read, n_kv_heads * ceil(L / 64) per request
-    long long unit_store; // start of its unit-boundary arrays (ceil(L / 64) + 1 ints per head)
+                          // about kUnitEntries rows to read, n_kv_heads * ceil(L / kUnitEntries) per request
+    long long unit_store; // start of its unit-boundary arrays (ceil(L / kUnitEntries) + 1 ints per head)
 };
 
 enum TileKind { kSweep1 = 0, kSweep2 = 1, kMatch = 2 };

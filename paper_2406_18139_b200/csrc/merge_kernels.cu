@@ -129,7 +129,6 @@ argmax_rows_kernel(const float* __restrict__ sim_matrix, const Req* __restrict__
 // earlier warps.  Keys are packed as (slot << 0) in one array and values in the other.
 // ---------------------------------------------------------------------------------------------
 constexpr int kInvThreads = 1024;
-constexpr int kUnitEntries = 64;     // entries (rows to read) per work unit of the merge kernel
 
 // Second half of the entry list: the kept rows (flagged with the sign bit, weight = member count)
 // and the work-unit boundaries: unit u covers the slots [units[u], units[u+1]), where units[u] is
@@ -278,7 +277,7 @@ invert_assignment_kernel(const int* __restrict__ assign, const int* __restrict__
 // ---------------------------------------------------------------------------------------------
 // Merge + compact (Eq. 6-7, 10-12).  Every K and V row of the prompt is read exactly once: the
 // entry list of a (request, head) names, slot by slot, the kept row and then its members.  A warp
-// takes a work unit of about 64 consecutive entries (whole slots), fetches the rows 16 entries at
+// takes a work unit of about 32 consecutive entries (whole slots), fetches the rows 8 entries at
 // a time with 16-byte cp.async copies into its own shared-memory ring (two buffers; every lane
 // later reads back exactly the bytes it copied, so cp.async.wait_group is all the synchronisation
 // needed), and walks the staged rows in order: lanes 0-15 hold the K row, lanes 16-31 the V row,
@@ -286,11 +285,11 @@ invert_assignment_kernel(const int* __restrict__ assign, const int* __restrict__
 //   averaged : (x_c + sum x_e) / (n + 1)                       (Eq. 10)
 //   pivotal  : (x_c + 1/2 sum (x_e + x_c)) / (n + 1)           (Eq. 11)
 //   weighted : (x_c + sum sim_e x_e) / (n + 1)                 (Eq. 12)
-// A row without members is copied bit for bit.  With 8 KB of copies in flight per warp the kernel
-// is bound by HBM, not by the latency of the dependent index loads.
+// A row without members is copied bit for bit.  Sixteen warps per SM with 4 KB of copies in flight each keep
+// HBM busy while the dependent index loads of the next unit are outstanding.
 // ---------------------------------------------------------------------------------------------
-constexpr int kMergeWarps = 8;
-constexpr int kChunk = 16;                           // entries staged per buffer
+constexpr int kMergeWarps = 16;
+constexpr int kChunk = 8;                            // entries staged per buffer
 constexpr int kRowBytes = kHeadDim * 2;              // one bf16 row of K or V
 
 struct MergeShared {
@@ -346,12 +345,12 @@ merge_kernel(const __nv_bfloat16* __restrict__ k, const __nv_bfloat16* __restric
         const __nv_bfloat16* src = tensor + (long long)rq.tok_begin * stride_tok + (long long)h * stride_head;
         const int n_chunks = (e_hi - e_lo + kChunk - 1) / kChunk;
 
-        // entry metadata of a chunk (lanes 0-15: one entry each)
+        // entry metadata of a chunk (lanes 0-7: one entry each)
         auto load_meta = [&](int kc, int& pos, float& w) {
             pos = 0;
             w = 0.f;
-            const int e = e_lo + kc * kChunk + l16;
-            if (kc < n_chunks && e < e_hi) { pos = ent[e]; w = entw[e]; }
+            const int e = e_lo + kc * kChunk + lane;
+            if (lane < kChunk && kc < n_chunks && e < e_hi) { pos = ent[e]; w = entw[e]; }
         };
         // start the row copies of chunk kc: for every entry, lanes 0-15 copy its K row and lanes
         // 16-31 its V row, 16 bytes each; one commit group per chunk
