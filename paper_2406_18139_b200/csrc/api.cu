@@ -38,6 +38,9 @@ struct Plan {
         o_rnorm_kept, o_assign, o_sim, o_row_ptr, o_members, o_member_w, o_units, o_sort_a, o_sort_b, total;
 };
 
+struct DeviceInfo { int sms = 0; int cc_major = 0; bool ok = false; };
+int device_info(DeviceInfo& out);
+
 // Returns LOOKM_OK or the status describing the first bad argument.
 int build_plan(Plan& pl, const lookm_layout* lay, int n_req, const int* cu_seqlens,
                const int* seq_lens, const int* budgets, const int* windows, const int* modes) {
@@ -93,6 +96,14 @@ int build_plan(Plan& pl, const lookm_layout* lay, int n_req, const int* cu_seqle
     // table order: longest request first
     std::stable_sort(pl.reqs.begin(), pl.reqs.end(), [](const Req& a, const Req& b) { return a.L > b.L; });
     long long it0 = 0, it1 = 0, it2 = 0, slots = 0, units = 0, unit_ints = 0;
+    // merge work units: about one per warp of the merge kernel (it reads n_kv_heads * T rows)
+    int unit_entries = kMinUnitEntries;
+    {
+        DeviceInfo di;
+        const int sms = (device_info(di) == LOOKM_OK && di.sms > 0) ? di.sms : 148;
+        const long long per_warp = ((long long)pl.n_kv_heads * pl.T) / ((long long)sms * merge_warps_per_sm());
+        if (per_warp > unit_entries) unit_entries = (int)std::min<long long>((per_warp + 7) / 8 * 8, 1 << 20);
+    }
     for (Req& q : pl.reqs) {
         q.item_begin[kSweep1] = (int)it0;
         q.item_begin[kSweep2] = (int)it1;
@@ -100,7 +111,8 @@ int build_plan(Plan& pl, const lookm_layout* lay, int n_req, const int* cu_seqle
         q.slot_begin = (int)slots;
         q.unit_begin = (int)units;
         q.unit_store = unit_ints;
-        const long long n_units = (q.L + kUnitEntries - 1) / kUnitEntries;
+        q.unit_entries = unit_entries;
+        const long long n_units = (q.L + unit_entries - 1) / unit_entries;
         units += (long long)pl.n_kv_heads * n_units;
         unit_ints += (long long)pl.n_kv_heads * (n_units + 1);
         it0 += (long long)q.nblk * pl.n_q_heads;
@@ -134,7 +146,7 @@ int build_plan(Plan& pl, const lookm_layout* lay, int n_req, const int* cu_seqle
     pl.o_row_ptr = carve(4 * (Hkv * T + Hkv * (size_t)n_req));
     pl.o_members = carve(4 * Hkv * T);
     pl.o_member_w = carve(4 * Hkv * T);
-    pl.o_units = carve(4 * Hkv * (T / kUnitEntries + 2 * (size_t)n_req));
+    pl.o_units = carve(4 * Hkv * (T / kMinUnitEntries + 2 * (size_t)n_req));
     pl.o_sort_a = carve(8 * Hkv * T);
     pl.o_sort_b = carve(8 * Hkv * T);
     pl.total = o;
@@ -161,8 +173,6 @@ int check_workspace(const Plan& pl, void* ws, size_t bytes) {
 }
 
 // ---- device facts and the tensor-map encoder ---------------------------------------------------
-struct DeviceInfo { int sms = 0; int cc_major = 0; bool ok = false; };
-
 int device_info(DeviceInfo& out) {
     static std::mutex mu;
     static DeviceInfo cache[64];
@@ -622,7 +632,7 @@ extern "C" int lookm_merge_noalloc(const void* k, const void* v, const int* kept
     pl.o_row_ptr = carve(4 * (units + (size_t)pl.n_kv_heads * (size_t)n_requests));
     pl.o_members = carve(4 * units);
     pl.o_member_w = carve(4 * units);
-    pl.o_units = carve(4 * ((size_t)pl.n_kv_heads * ((size_t)pl.T / kUnitEntries + 2 * (size_t)n_requests)));
+    pl.o_units = carve(4 * ((size_t)pl.n_kv_heads * ((size_t)pl.T / kMinUnitEntries + 2 * (size_t)n_requests)));
     pl.o_sort_a = carve(8 * units);
     pl.o_sort_b = carve(8 * units);
     pl.total = o;

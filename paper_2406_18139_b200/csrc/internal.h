@@ -11,7 +11,7 @@ namespace lookm {
 
 constexpr int kTile = 128;      // tokens per tile on either operand of the tensor-core kernels
 constexpr int kHeadDim = 128;   // only supported head_dim
-constexpr int kUnitEntries = 32; // rows read per work unit of the merge kernel (whole slots)
+constexpr int kMinUnitEntries = 32; // least number of rows in a work unit of the merge kernel
 
 // One request of the packed batch as the kernels see it (device copy lives in the workspace).
 // Requests are stored longest first so that the heaviest work items are issued first.
@@ -31,9 +31,11 @@ struct Req {
                           // which hold B + 1 entries per head
     int item_begin[3];    // first work item of this request in sweep 1 / sweep 2 / match order
     int slot_begin;       // first (head, slot) row of this request in merge order (table order)
-    int unit_begin;       // first merge work unit of this request (table order); a unit is
-                          // about kUnitEntries rows to read, n_kv_heads * ceil(L / kUnitEntries) per request
-    long long unit_store; // start of its unit-boundary arrays (ceil(L / kUnitEntries) + 1 ints per head)
+    int unit_entries;     // rows read per merge work unit (whole slots): chosen per call so that
+                          // every warp of the merge kernel gets about one unit
+    int unit_begin;       // first merge work unit of this request (table order);
+                          // n_kv_heads * ceil(L / unit_entries) units per request
+    long long unit_store; // start of its unit-boundary arrays (ceil(L / unit_entries) + 1 ints per head)
 };
 
 enum TileKind { kSweep1 = 0, kSweep2 = 1, kMatch = 2 };
@@ -90,6 +92,8 @@ cudaError_t launch_invert_assignment(const int* assign, const int* kept_idx, con
                                      long long T, int* row_ptr, int* ent_pos, float* ent_w,
                                      int* unit_slot, unsigned* sort_a, unsigned* sort_b, int* status,
                                      cudaStream_t stream);
+
+int merge_warps_per_sm();
 
 cudaError_t launch_merge(const void* k, const void* v, long long stride_tok, long long stride_head,
                          const Req* reqs, int n_req, int n_kv_heads, long long T,

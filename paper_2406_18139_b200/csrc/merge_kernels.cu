@@ -132,11 +132,12 @@ constexpr int kInvThreads = 1024;
 
 // Second half of the entry list: the kept rows (flagged with the sign bit, weight = member count)
 // and the work-unit boundaries: unit u covers the slots [units[u], units[u+1]), where units[u] is
-// the first slot whose entry index c + row_ptr[c] is >= u * kUnitEntries.
+// the first slot whose entry index c + row_ptr[c] is >= u * unit_entries.
 __device__ __forceinline__ void write_kept_entries(const Req& rq, int h, int B, int E, const int* rp,
                                                    const int* kept_idx_head, int* ent, float* entw,
                                                    int* units, int* status) {
-    const int n_units = (rq.L + kUnitEntries - 1) / kUnitEntries;
+    const int ue = rq.unit_entries;
+    const int n_units = (rq.L + ue - 1) / ue;
     for (int c = threadIdx.x; c < B; c += blockDim.x) {
         int pc = kept_idx_head[c];
         if (pc < 0 || pc >= rq.L) { atomicExch(status, (int)LOOKM_ERR_DEVICE_BAD_INDEX); pc = 0; }
@@ -144,9 +145,9 @@ __device__ __forceinline__ void write_kept_entries(const Req& rq, int h, int B, 
         ent[s_c] = pc | (int)0x80000000;
         entw[s_c] = (float)(rp[c + 1] - rp[c]);
         const int s_prev = c ? (c - 1) + rp[c - 1] : -1;
-        for (int u = s_prev / kUnitEntries + (s_prev >= 0 ? 1 : 0); u * kUnitEntries <= s_c; ++u) units[u] = c;
+        for (int u = s_prev / ue + (s_prev >= 0 ? 1 : 0); u * ue <= s_c; ++u) units[u] = c;
         if (c == B - 1)
-            for (int u = s_c / kUnitEntries + 1; u <= n_units; ++u) units[u] = B;
+            for (int u = s_c / ue + 1; u <= n_units; ++u) units[u] = B;
     }
     (void)h; (void)E;
 }
@@ -172,7 +173,7 @@ invert_assignment_kernel(const int* __restrict__ assign, const int* __restrict__
     // entry list of this (request, head): for every kept slot its kept row, then its members
     int* ent = ent_pos + (long long)h * T + rq.tok_begin;
     float* entw = ent_w + (long long)h * T + rq.tok_begin;
-    const int n_units = (rq.L + kUnitEntries - 1) / kUnitEntries;
+    const int n_units = (rq.L + rq.unit_entries - 1) / rq.unit_entries;
     int* units = unit_slot + rq.unit_store + (long long)h * (n_units + 1);
     const int* kept_idx_head = kept_idx + rq.kept_off + (long long)h * B;
     const bool weighted = (rq.mode == LOOKM_MERGE_WEIGHTED);
@@ -277,7 +278,8 @@ invert_assignment_kernel(const int* __restrict__ assign, const int* __restrict__
 // ---------------------------------------------------------------------------------------------
 // Merge + compact (Eq. 6-7, 10-12).  Every K and V row of the prompt is read exactly once: the
 // entry list of a (request, head) names, slot by slot, the kept row and then its members.  A warp
-// takes a work unit of about 32 consecutive entries (whole slots), fetches the rows 8 entries at
+// takes a work unit of consecutive entries (whole slots; sized so that each warp gets about one
+// unit, at least 32 entries), fetches the rows 8 entries at
 // a time with 16-byte cp.async copies into its own shared-memory ring (two buffers; every lane
 // later reads back exactly the bytes it copied, so cp.async.wait_group is all the synchronisation
 // needed), and walks the staged rows in order: lanes 0-15 hold the K row, lanes 16-31 the V row,
@@ -288,7 +290,7 @@ invert_assignment_kernel(const int* __restrict__ assign, const int* __restrict__
 // A row without members is copied bit for bit.  Sixteen warps per SM with 4 KB of copies in flight each keep
 // HBM busy while the dependent index loads of the next unit are outstanding.
 // ---------------------------------------------------------------------------------------------
-constexpr int kMergeWarps = 16;
+constexpr int kMergeWarps = 16;                      // per CTA; one CTA per SM
 constexpr int kChunk = 8;                            // entries staged per buffer
 constexpr int kRowBytes = kHeadDim * 2;              // one bf16 row of K or V
 
@@ -326,9 +328,11 @@ merge_kernel(const __nv_bfloat16* __restrict__ k, const __nv_bfloat16* __restric
          g += (long long)gridDim.x * kMergeWarps) {
         const Req& rq = find_req_by_unit(reqs, n_req, g);
         const int L = rq.L, B = rq.B, mode = rq.mode;
-        const int n_units = (L + kUnitEntries - 1) / kUnitEntries;
+        const int n_units = (L + rq.unit_entries - 1) / rq.unit_entries;
         const long long ul = g - rq.unit_begin;
-        const int h = (int)(ul / n_units), u = (int)(ul % n_units);
+        // heads vary fastest: warps running at the same time then read the same token range of
+        // different heads, i.e. neighbouring 256-byte rows of the same DRAM pages
+        const int h = (int)(ul % n_kv_heads), u = (int)(ul / n_kv_heads);
         const int* units = unit_slot + rq.unit_store + (long long)h * (n_units + 1);
         const int* rp = row_ptr + rq.rp_off + (long long)h * (B + 1);
         // lanes 0/1: first slot / one past the last slot of the unit, and their entry indices
@@ -510,6 +514,8 @@ cudaError_t launch_invert_assignment(const int* assign, const int* kept_idx, con
                                                                unit_slot, sort_a, sort_b, status);
     return cudaGetLastError();
 }
+
+int merge_warps_per_sm() { return kMergeWarps; }
 
 cudaError_t launch_merge(const void* k, const void* v, long long stride_tok, long long stride_head,
                          const Req* reqs, int n_req, int n_kv_heads, long long T,
