@@ -280,7 +280,7 @@ invert_assignment_kernel(const int* __restrict__ assign, const int* __restrict__
 // entry list of a (request, head) names, slot by slot, the kept row and then its members.  A warp
 // takes a work unit of consecutive entries (whole slots; sized so that each warp gets about one
 // unit, at least 32 entries), fetches the rows 8 entries at
-// a time with 16-byte cp.async copies into its own shared-memory ring (two buffers; every lane
+// a time with 16-byte cp.async copies into its own shared-memory ring (three buffers; every lane
 // later reads back exactly the bytes it copied, so cp.async.wait_group is all the synchronisation
 // needed), and walks the staged rows in order: lanes 0-15 hold the K row, lanes 16-31 the V row,
 // 16 bytes per lane, fp32 accumulation in member order, one rounding.
@@ -292,10 +292,11 @@ invert_assignment_kernel(const int* __restrict__ assign, const int* __restrict__
 // ---------------------------------------------------------------------------------------------
 constexpr int kMergeWarps = 16;                      // per CTA; one CTA per SM
 constexpr int kChunk = 8;                            // entries staged per buffer
+constexpr int kRing = 3;                             // buffers per warp: two chunks in flight while one is read
 constexpr int kRowBytes = kHeadDim * 2;              // one bf16 row of K or V
 
 struct MergeShared {
-    alignas(128) uint8_t rows[kMergeWarps][2][kChunk][2 * kRowBytes];   // [warp][buffer][entry][K|V]
+    alignas(128) uint8_t rows[kMergeWarps][kRing][kChunk][2 * kRowBytes];   // [warp][buffer][entry][K|V]
 };
 
 __device__ __forceinline__ const Req& find_req_by_unit(const Req* reqs, int n_req, long long g) {
@@ -359,8 +360,8 @@ merge_kernel(const __nv_bfloat16* __restrict__ k, const __nv_bfloat16* __restric
         // start the row copies of chunk kc: for every entry, lanes 0-15 copy its K row and lanes
         // 16-31 its V row, 16 bytes each; one commit group per chunk
         auto issue = [&](int kc, int pos) {
-            const int cnt = min(kChunk, e_hi - e_lo - kc * kChunk);
-            const uint32_t dst = buf0 + ((n_chunks_done + (uint32_t)kc) & 1u) * (kChunk * 2 * kRowBytes);
+            const int cnt = min(kChunk, e_hi - e_lo - kc * kChunk);      // <= 0 past the unit: empty group
+            const uint32_t dst = buf0 + ((n_chunks_done + (uint32_t)kc) % kRing) * (kChunk * 2 * kRowBytes);
             for (int q = 0; q < cnt; ++q) {
                 const int tok = __shfl_sync(0xffffffffu, pos, q) & 0x7fffffff;
                 asm volatile("cp.async.cg.shared.global [%0], [%1], 16;"
@@ -370,11 +371,13 @@ merge_kernel(const __nv_bfloat16* __restrict__ k, const __nv_bfloat16* __restric
             asm volatile("cp.async.commit_group;" ::: "memory");
         };
 
-        int pos_a, pos_b;
-        float w_a, w_b;
+        int pos_a, pos_b, pos_c;
+        float w_a, w_b, w_c;
         load_meta(0, pos_a, w_a);
-        issue(0, pos_a);
         load_meta(1, pos_b, w_b);
+        load_meta(2, pos_c, w_c);
+        issue(0, pos_a);
+        issue(1, pos_b);
 
         // running row
         int slot = c_lo - 1, n_mem = 0;
@@ -403,15 +406,15 @@ merge_kernel(const __nv_bfloat16* __restrict__ k, const __nv_bfloat16* __restric
         };
 
         for (int kc = 0; kc < n_chunks; ++kc) {
-            // next chunk's copies go to the other buffer, whose rows were consumed one iteration ago
-            if (kc + 1 < n_chunks) issue(kc + 1, pos_b);
-            int pos_c;
-            float w_c;
-            load_meta(kc + 2, pos_c, w_c);
-            // this chunk's copies: everything but the group just committed must have landed
-            if (kc + 1 < n_chunks) asm volatile("cp.async.wait_group 1;" ::: "memory");
-            else asm volatile("cp.async.wait_group 0;" ::: "memory");
-            const uint32_t b = (n_chunks_done + (uint32_t)kc) & 1u;
+            // chunk kc + 2 goes to the buffer whose rows were consumed one iteration ago; a commit
+            // group is made for every chunk index (empty past the unit), so "all but the two
+            // newest groups" always means: chunk kc has landed
+            issue(kc + 2, pos_c);
+            int pos_d;
+            float w_d;
+            load_meta(kc + 3, pos_d, w_d);
+            asm volatile("cp.async.wait_group 2;" ::: "memory");
+            const uint32_t b = (n_chunks_done + (uint32_t)kc) % kRing;
             const int cnt = min(kChunk, e_hi - e_lo - kc * kChunk);
             const uint8_t* base = &sh.rows[warp][b][0][0] + lane * 16;
             for (int q = 0; q < cnt; ++q) {
@@ -434,6 +437,7 @@ merge_kernel(const __nv_bfloat16* __restrict__ k, const __nv_bfloat16* __restric
             __syncwarp();
             pos_a = pos_b; w_a = w_b;
             pos_b = pos_c; w_b = w_c;
+            pos_c = pos_d; w_c = w_d;
         }
         flush();
         n_chunks_done += (uint32_t)n_chunks;
