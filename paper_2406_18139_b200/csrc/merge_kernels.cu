@@ -347,7 +347,7 @@ merge_kernel(const __nv_bfloat16* __restrict__ k, const __nv_bfloat16* __restric
         if (c_lo >= c_hi) continue;
         const int* ent = ent_pos + (long long)h * T + rq.tok_begin;
         const float* entw = ent_w + (long long)h * T + rq.tok_begin;
-        const __nv_bfloat16* src = tensor + (long long)rq.tok_begin * stride_tok + (long long)h * stride_head;
+        const __nv_bfloat16* src = tensor + (long long)rq.tok_begin * stride_tok + (long long)h * stride_head + l16 * 8;
         const int n_chunks = (e_hi - e_lo + kChunk - 1) / kChunk;
 
         // entry metadata of a chunk (lanes 0-7: one entry each)
@@ -362,11 +362,13 @@ merge_kernel(const __nv_bfloat16* __restrict__ k, const __nv_bfloat16* __restric
         auto issue = [&](int kc, int pos) {
             const int cnt = min(kChunk, e_hi - e_lo - kc * kChunk);      // <= 0 past the unit: empty group
             const uint32_t dst = buf0 + ((n_chunks_done + (uint32_t)kc) % kRing) * (kChunk * 2 * kRowBytes);
-            for (int q = 0; q < cnt; ++q) {
+#pragma unroll
+            for (int q = 0; q < kChunk; ++q) {
                 const int tok = __shfl_sync(0xffffffffu, pos, q) & 0x7fffffff;
-                asm volatile("cp.async.cg.shared.global [%0], [%1], 16;"
-                             ::"r"(dst + q * (2 * kRowBytes)), "l"(src + (long long)tok * stride_tok + l16 * 8)
-                             : "memory");
+                if (q < cnt)
+                    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;"
+                                 ::"r"(dst + q * (2 * kRowBytes)), "l"(src + (long long)tok * stride_tok)
+                                 : "memory");
             }
             asm volatile("cp.async.commit_group;" ::: "memory");
         };
@@ -417,9 +419,11 @@ merge_kernel(const __nv_bfloat16* __restrict__ k, const __nv_bfloat16* __restric
             const uint32_t b = (n_chunks_done + (uint32_t)kc) % kRing;
             const int cnt = min(kChunk, e_hi - e_lo - kc * kChunk);
             const uint8_t* base = &sh.rows[warp][b][0][0] + lane * 16;
-            for (int q = 0; q < cnt; ++q) {
+#pragma unroll
+            for (int q = 0; q < kChunk; ++q) {
                 const int pe = __shfl_sync(0xffffffffu, pos_a, q);
                 const float w = __shfl_sync(0xffffffffu, w_a, q);
+                if (q >= cnt) break;
                 const uint4 x4 = *reinterpret_cast<const uint4*>(base + q * (2 * kRowBytes));
                 if (pe < 0) {                        // a kept row starts the next slot
                     flush();
