@@ -307,9 +307,16 @@ def run_ours(args):
     stages["merge"].update({"gbs": round(gbs, 1), "frac_of_%s_hbm" % peaks["source"]: round(gbs / peaks["hbm_gbs"], 4)})
     dom = max(("score_sweep1", "score_sweep2"), key=lambda n: stages[n]["ms"])
     achieved = sweep_flops / (stages[dom]["ms"] * 1e-3) / 1e12
+    # DRAM traffic per launch of the dominant kernel: dram__bytes_read + write of one ncu capture
+    # on the 4096-token x 16-head case (profiles/tile_kernels_4096x16.txt), scaled by tokens x heads
+    # (the kernels read Q and K once from DRAM and re-read tiles from L2, so traffic grows with
+    # the input size).  Must be set to None when the tile kernels change after the capture.
+    captured = {"score_sweep1": 33.584896e6, "score_sweep2": 33.846784e6}
+    traffic = captured[dom] * (L * Hq) / (4096.0 * 16.0)
     roofline = {"kernel": "tile_kernel<%s>" % dom, "bound": "tensor", "achieved": round(achieved, 2),
                 "peak": peaks["tflops"], "peak_source": peaks["source"] + " (cuBLAS bf16, sustained)",
-                "unit": "TFLOP/s", "frac": round(achieved / peaks["tflops"], 4), "traffic": None}
+                "unit": "TFLOP/s", "frac": round(achieved / peaks["tflops"], 4), "traffic": traffic,
+                "traffic_unit": "bytes per launch (ncu capture of a 4096x16 case, scaled)"}
     e2e_value = world * e2e_steps * units_per_step / (e2e_ms * 1e-3)
     h2d = sum(t.numel() * t.element_size() for t in host_sets[0]) + mask_host.numel()
     d2h = (out_k.numel() + out_v.numel()) * 2
