@@ -349,19 +349,40 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                             }
                         }
                     } else {
-                        // running arg-max of dot / |kept key| over kept slots; ascending slot order
-                        // with a strict comparison keeps the lowest slot on ties
+                        // running arg-max of dot / |kept key| over kept slots.  Per 16 columns the
+                        // maximum is taken first (two instructions per element); only when it beats
+                        // the running best (rare after the first tiles) is its first column looked
+                        // up, so a strict comparison in ascending slot order keeps the lowest slot
                         const float4* sd = reinterpret_cast<const float4*>(side + c0);
                         const int slot0 = t * kTile + c0;
 #pragma unroll
-                        for (int c4 = 0; c4 < 8; ++c4) {
-                            const float4 r4 = sd[c4];
-                            const float rn[4] = {r4.x, r4.y, r4.z, r4.w};
+                        for (int g16 = 0; g16 < 2; ++g16) {
+                            float v[16];
 #pragma unroll
-                            for (int q = 0; q < 4; ++q) {
-                                const int c = c4 * 4 + q;
-                                const float v = __uint_as_float(raw[c]) * rn[q];
-                                if (c0 + c < col_limit && v > best) { best = v; best_slot = slot0 + c; }
+                            for (int c4 = 0; c4 < 4; ++c4) {
+                                const float4 r4 = sd[g16 * 4 + c4];
+                                const int c = g16 * 16 + c4 * 4;
+                                v[c4 * 4 + 0] = __uint_as_float(raw[c + 0]) * r4.x;
+                                v[c4 * 4 + 1] = __uint_as_float(raw[c + 1]) * r4.y;
+                                v[c4 * 4 + 2] = __uint_as_float(raw[c + 2]) * r4.z;
+                                v[c4 * 4 + 3] = __uint_as_float(raw[c + 3]) * r4.w;
+                            }
+                            if (col_limit < kTile) {       // last tile of the kept list only
+#pragma unroll
+                                for (int c = 0; c < 16; ++c)
+                                    if (c0 + g16 * 16 + c >= col_limit) v[c] = -INFINITY;
+                            }
+                            const float m0 = fmaxf(fmaxf(v[0], v[1]), fmaxf(v[2], v[3]));
+                            const float m1 = fmaxf(fmaxf(v[4], v[5]), fmaxf(v[6], v[7]));
+                            const float m2 = fmaxf(fmaxf(v[8], v[9]), fmaxf(v[10], v[11]));
+                            const float m3 = fmaxf(fmaxf(v[12], v[13]), fmaxf(v[14], v[15]));
+                            const float mx = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
+                            if (mx > best) {
+                                best = mx;
+                                int idx = 15;
+#pragma unroll
+                                for (int c = 14; c >= 0; --c) if (v[c] == mx) idx = c;
+                                best_slot = slot0 + g16 * 16 + idx;
                             }
                         }
                     }
