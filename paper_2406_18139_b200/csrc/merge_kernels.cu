@@ -51,34 +51,20 @@ key_norms_kernel(const __nv_bfloat16* __restrict__ k, long long stride_tok, long
                  int n_kv_heads, long long T, float* __restrict__ rnorm_all) {
     const int half = threadIdx.x >> 4, l16 = threadIdx.x & 15;
     const long long n_rows = T * n_kv_heads;
-    const long long step = (long long)gridDim.x * 16;
-    // four rows per half-warp and iteration: four 16-byte loads in flight per lane
     // the loop bound is the warp's first row, so that both half-warps always reach the shuffles
-    for (long long rw = (long long)blockIdx.x * 16 + (half & ~1); rw < n_rows; rw += 4 * step) {
-        const long long r0 = rw + (half & 1);
-        uint4 u[4];
+    for (long long rw = (long long)blockIdx.x * 16 + (half & ~1); rw < n_rows; rw += (long long)gridDim.x * 16) {
+        const long long r = rw + (half & 1);
+        const bool valid = r < n_rows;
+        const long long tok = valid ? r / n_kv_heads : 0;
+        const int h = valid ? (int)(r % n_kv_heads) : 0;
+        const uint4 u = *reinterpret_cast<const uint4*>(k + tok * stride_tok + h * stride_head + l16 * 8);
+        const Row8 x = unpack8(u);
+        float ss = 0.f;
 #pragma unroll
-        for (int q = 0; q < 4; ++q) {
-            const long long r = r0 + q * step;
-            u[q] = make_uint4(0u, 0u, 0u, 0u);
-            if (r < n_rows) {
-                const long long tok = r / n_kv_heads;
-                const int h = (int)(r % n_kv_heads);
-                u[q] = *reinterpret_cast<const uint4*>(k + tok * stride_tok + h * stride_head + l16 * 8);
-            }
-        }
+        for (int i = 0; i < 8; ++i) ss = fmaf(x.v[i], x.v[i], ss);
 #pragma unroll
-        for (int q = 0; q < 4; ++q) {
-            const long long r = r0 + q * step;
-            const Row8 x = unpack8(u[q]);
-            float ss = 0.f;
-#pragma unroll
-            for (int i = 0; i < 8; ++i) ss = fmaf(x.v[i], x.v[i], ss);
-#pragma unroll
-            for (int o = 8; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o, 16);
-            if (l16 == 0 && r < n_rows)
-                rnorm_all[(long long)(r % n_kv_heads) * T + r / n_kv_heads] = ss > 0.f ? 1.0f / sqrtf(ss) : 0.f;
-        }
+        for (int o = 8; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o, 16);
+        if (l16 == 0 && valid) rnorm_all[(long long)h * T + tok] = ss > 0.f ? 1.0f / sqrtf(ss) : 0.f;
     }
 }
 
