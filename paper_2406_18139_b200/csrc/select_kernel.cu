@@ -96,41 +96,21 @@ select_kernel(const float* __restrict__ scores, const uint8_t* __restrict__ mask
         for (int shift = 24; shift >= 0; shift -= 8) {
             for (int i = threadIdx.x; i < 256; i += kSelThreads) hist[i] = 0;
             __syncthreads();
-            // warp-aggregated histogram: lanes with the same digit add once (scores share their
-            // leading bits, so plain shared-memory atomics would all hit the same few bins)
-            for (int j0 = 0; j0 < nc; j0 += kSelThreads) {
-                const int j = j0 + threadIdx.x;
-                unsigned d = 0x100u + (threadIdx.x & 31);        // lanes without a candidate never match
-                if (j < nc && (msk[j] != 0) == (sel_cls != 0)) {
+            for (int j = threadIdx.x; j < nc; j += kSelThreads) {
+                if ((msk[j] != 0) == (sel_cls != 0)) {
                     const unsigned key = order_key(s[j]);
-                    if ((key & pmask) == prefix) d = (key >> shift) & 255u;
+                    if ((key & pmask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1);
                 }
-                const unsigned peers = __match_any_sync(0xffffffffu, d);
-                if (d < 256u && (peers & ((1u << (threadIdx.x & 31)) - 1u)) == 0u)
-                    atomicAdd(&hist[d], __popc(peers));
             }
             __syncthreads();
-            // digit of the remaining-th largest key: first warp, 8 bins per lane, suffix sums by shuffle
-            if (threadIdx.x < 32) {
-                const int lane = threadIdx.x;
-                int loc[8], sum = 0;
-#pragma unroll
-                for (int i = 0; i < 8; ++i) { loc[i] = hist[lane * 8 + i]; sum += loc[i]; }
-                int suf = sum;                                   // bins of this lane and of higher lanes
-#pragma unroll
-                for (int o = 1; o < 32; o <<= 1) {
-                    const int x = __shfl_down_sync(0xffffffffu, suf, o);
-                    if (lane + o < 32) suf += x;
+            if (threadIdx.x == 0) {
+                int acc = 0, d = 255;
+                for (; d > 0; --d) {
+                    if (acc + hist[d] >= remaining) break;
+                    acc += hist[d];
                 }
-                const int above = suf - sum;
-                if (above < remaining && remaining <= above + sum) {
-                    int acc = above;
-#pragma unroll
-                    for (int i = 7; i >= 0; --i) {
-                        if (acc + loc[i] >= remaining) { sh_val[0] = lane * 8 + i; sh_val[1] = remaining - acc; break; }
-                        acc += loc[i];
-                    }
-                }
+                sh_val[0] = d;
+                sh_val[1] = remaining - acc;             // still to take inside digit d
             }
             __syncthreads();
             prefix |= (unsigned)sh_val[0] << shift;
