@@ -99,6 +99,26 @@ class ClockSampler(threading.Thread):
                 "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
 
 
+def rank_layers(rank):
+    """Layers (seeds) whose inputs rank `rank` compresses: every rank gets its own replica."""
+    return [rank * N_INPUT_SETS + s for s in range(N_INPUT_SETS)]
+
+
+def max_over_ranks(values, world, device):
+    """Element-wise maximum of a list of floats over all ranks (the job is as slow as its slowest rank)."""
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor(values, dtype=torch.float64, device=device)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return t.tolist()
+
+
+def job_throughput(world, steps, units_per_step, ms):
+    """Whole-job units per second: all ranks' units over the slowest rank's time."""
+    return world * steps * units_per_step / (ms * 1e-3)
+
+
 def physical_gpu_index(local_rank):
     vis = os.environ.get("CUDA_VISIBLE_DEVICES")
     if vis:
@@ -193,8 +213,8 @@ def run_ours(args):
     L, Hq, Hkv, budget, window = req.seq_len, w.n_q_heads, w.n_kv_heads, req.budget, req.window
     dev = lambda bits: torch.from_numpy(bits.view(np.int16)).cuda().view(torch.bfloat16)
     host_sets, dev_sets, first_bits = [], [], None
-    for s in range(N_INPUT_SETS):
-        qb, kb, vb = synth.layer_tensors(w, layer=rank * N_INPUT_SETS + s)
+    for layer in rank_layers(rank):
+        qb, kb, vb = synth.layer_tensors(w, layer=layer)
         first_bits = first_bits or (qb, kb, vb)
         host_sets.append(tuple(torch.from_numpy(t.view(np.int16)).view(torch.bfloat16).pin_memory()
                                for t in (qb, kb, vb)))
@@ -272,10 +292,7 @@ def run_ours(args):
     fence()
     e2e_ms = e_begin.elapsed_time(e_end)
 
-    times = torch.tensor([ms_total, e2e_ms], dtype=torch.float64, device="cuda")
-    if world > 1:
-        dist.all_reduce(times, op=dist.ReduceOp.MAX)
-    ms_total, e2e_ms = times.tolist()
+    ms_total, e2e_ms = max_over_ranks([ms_total, e2e_ms], world, "cuda")
 
     if rank != 0:
         if world > 1:
@@ -283,7 +300,7 @@ def run_ours(args):
         return
 
     units_per_step = L * Hkv
-    value = world * args.steps * units_per_step / (ms_total * 1e-3)
+    value = job_throughput(world, args.steps, units_per_step, ms_total)
     stage_ms = np.zeros(n_ev - 1)
     for evs in stage_events:
         for s in range(n_ev - 1):
@@ -317,7 +334,7 @@ def run_ours(args):
                 "peak": peaks["tflops"], "peak_source": peaks["source"] + " (cuBLAS bf16, sustained)",
                 "unit": "TFLOP/s", "frac": round(achieved / peaks["tflops"], 4), "traffic": traffic,
                 "traffic_unit": "bytes per launch (ncu capture of a 4096x16 case, scaled)"}
-    e2e_value = world * e2e_steps * units_per_step / (e2e_ms * 1e-3)
+    e2e_value = job_throughput(world, e2e_steps, units_per_step, e2e_ms)
     h2d = sum(t.numel() * t.element_size() for t in host_sets[0]) + mask_host.numel()
     d2h = (out_k.numel() + out_v.numel()) * 2
     out = {
