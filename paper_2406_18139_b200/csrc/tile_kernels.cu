@@ -32,9 +32,8 @@ namespace {
 
 constexpr int kStages = 4;                       // ring of streamed tiles
 constexpr int kAccum = 4;                        // TMEM accumulators (128 fp32 columns each)
-constexpr int kGroups = 3;                       // epilogue groups: one fewer than accumulators, so that a
-                                                 // group finds its next tile's MMA already done
-constexpr int kThreads = 64 + kGroups * 128;     // producer warp, MMA warp, 3 x 4 epilogue warps
+constexpr int kGroups = 4;                       // epilogue groups (one per TMEM accumulator)
+constexpr int kThreads = 64 + kGroups * 128;     // producer warp, MMA warp, 4 x 4 epilogue warps
 constexpr int kHalfBytes = kTile * 64 * 2;       // one TMA box: 128 rows x 64 bf16 (128 B rows)
 constexpr int kTileBytes = 2 * kHalfBytes;       // 128 x 128 bf16
 constexpr int kReqCache = 32;                    // request-table entries cached in shared memory
@@ -260,7 +259,7 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
 
             for (int t = 0; t < it.nt; ++t, ++gb) {
                 if ((int)(gb % kGroups) != wg) continue;
-                const int buf = gb % kAccum;
+                const int buf = wg;
                 float* side = sh.side[wg][lt & 1];
                 bool diag = false;                           // tile crosses the causal diagonal
                 int col_limit = kTile;                       // match: valid kept slots in the tile
