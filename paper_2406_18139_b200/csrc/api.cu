@@ -146,7 +146,7 @@ int build_plan(Plan& pl, const lookm_layout* lay, int n_req, const int* cu_seqle
     pl.o_row_ptr = carve(4 * (Hkv * T + Hkv * (size_t)n_req));
     pl.o_members = carve(4 * Hkv * T);
     pl.o_member_w = carve(4 * Hkv * T);
-    pl.o_units = carve(8 * Hkv * (T / kMinUnitEntries + 2 * (size_t)n_req));
+    pl.o_units = carve(4 * Hkv * (T / kMinUnitEntries + 2 * (size_t)n_req));
     pl.o_sort_a = carve(8 * Hkv * T);
     pl.o_sort_b = carve(8 * Hkv * T);
     pl.total = o;
@@ -345,9 +345,9 @@ int run_merge(const Plan& pl, const lookm_layout* lay, const void* k, const void
     DeviceInfo di;
     LOOKM_TRY(device_info(di));
     LOOKM_CUDA(launch_merge(k, v, lay->kv_stride_tok, lay->kv_stride_head, reqs, pl.n_req,
-                            pl.n_kv_heads, pl.T, pl.total_units, at<int>(ws, pl.o_members),
-                            at<float>(ws, pl.o_member_w), at<int>(ws, pl.o_units), varlen_output,
-                            out_k, out_v, di.sms, st));
+                            pl.n_kv_heads, pl.T, pl.total_units, at<int>(ws, pl.o_row_ptr),
+                            at<int>(ws, pl.o_members), at<float>(ws, pl.o_member_w),
+                            at<int>(ws, pl.o_units), varlen_output, out_k, out_v, status, di.sms, st));
     ++g_launches;
     mark_stage(7, st);
     return LOOKM_OK;
@@ -632,7 +632,7 @@ extern "C" int lookm_merge_noalloc(const void* k, const void* v, const int* kept
     pl.o_row_ptr = carve(4 * (units + (size_t)pl.n_kv_heads * (size_t)n_requests));
     pl.o_members = carve(4 * units);
     pl.o_member_w = carve(4 * units);
-    pl.o_units = carve(8 * ((size_t)pl.n_kv_heads * ((size_t)pl.T / kMinUnitEntries + 2 * (size_t)n_requests)));
+    pl.o_units = carve(4 * ((size_t)pl.n_kv_heads * ((size_t)pl.T / kMinUnitEntries + 2 * (size_t)n_requests)));
     pl.o_sort_a = carve(8 * units);
     pl.o_sort_b = carve(8 * units);
     pl.total = o;

@@ -35,7 +35,7 @@ struct Req {
                           // every warp of the merge kernel gets about one unit
     int unit_begin;       // first merge work unit of this request (table order);
                           // n_kv_heads * ceil(L / unit_entries) units per request
-    long long unit_store; // start of its unit-boundary records (ceil(L / unit_entries) + 1 int pairs per head)
+    long long unit_store; // start of its unit-boundary arrays (ceil(L / unit_entries) + 1 ints per head)
 };
 
 enum TileKind { kSweep1 = 0, kSweep2 = 1, kMatch = 2 };
@@ -97,8 +97,8 @@ int merge_warps_per_sm();
 
 cudaError_t launch_merge(const void* k, const void* v, long long stride_tok, long long stride_head,
                          const Req* reqs, int n_req, int n_kv_heads, long long T,
-                         long long total_units, const int* ent_pos, const float* ent_w,
-                         const int* unit_slot, int varlen_output, void* out_k, void* out_v,
-                         int num_sms, cudaStream_t stream);
+                         long long total_units, const int* row_ptr, const int* ent_pos,
+                         const float* ent_w, const int* unit_slot, int varlen_output, void* out_k,
+                         void* out_v, int* status, int num_sms, cudaStream_t stream);
 
 }  // namespace lookm

@@ -134,9 +134,8 @@ argmax_rows_kernel(const float* __restrict__ sim_matrix, const Req* __restrict__
 constexpr int kInvThreads = 1024;
 
 // Second half of the entry list: the kept rows (flagged with the sign bit, weight = member count)
-// and the work-unit boundaries: unit u covers the slots [units[2u], units[2u+2]), where units[2u]
-// is the first slot whose entry index c + row_ptr[c] is >= u * unit_entries and units[2u+1] is
-// that entry index.
+// and the work-unit boundaries: unit u covers the slots [units[u], units[u+1]), where units[u] is
+// the first slot whose entry index c + row_ptr[c] is >= u * unit_entries.
 __device__ __forceinline__ void write_kept_entries(const Req& rq, int h, int B, int E, const int* rp,
                                                    const int* kept_idx_head, int* ent, float* entw,
                                                    int* units, int* status) {
@@ -149,9 +148,9 @@ __device__ __forceinline__ void write_kept_entries(const Req& rq, int h, int B, 
         ent[s_c] = pc | (int)0x80000000;
         entw[s_c] = (float)(rp[c + 1] - rp[c]);
         const int s_prev = c ? (c - 1) + rp[c - 1] : -1;
-        for (int u = s_prev / ue + (s_prev >= 0 ? 1 : 0); u * ue <= s_c; ++u) { units[2 * u] = c; units[2 * u + 1] = s_c; }
+        for (int u = s_prev / ue + (s_prev >= 0 ? 1 : 0); u * ue <= s_c; ++u) units[u] = c;
         if (c == B - 1)
-            for (int u = s_c / ue + 1; u <= n_units; ++u) { units[2 * u] = B; units[2 * u + 1] = rq.L; }
+            for (int u = s_c / ue + 1; u <= n_units; ++u) units[u] = B;
     }
     (void)h; (void)E;
 }
@@ -178,7 +177,7 @@ invert_assignment_kernel(const int* __restrict__ assign, const int* __restrict__
     int* ent = ent_pos + (long long)h * T + rq.tok_begin;
     float* entw = ent_w + (long long)h * T + rq.tok_begin;
     const int n_units = (rq.L + rq.unit_entries - 1) / rq.unit_entries;
-    int* units = unit_slot + 2 * (rq.unit_store + (long long)h * (n_units + 1));
+    int* units = unit_slot + rq.unit_store + (long long)h * (n_units + 1);
     const int* kept_idx_head = kept_idx + rq.kept_off + (long long)h * B;
     const bool weighted = (rq.mode == LOOKM_MERGE_WEIGHTED);
     if (E == 0) {
@@ -282,35 +281,26 @@ invert_assignment_kernel(const int* __restrict__ assign, const int* __restrict__
 // ---------------------------------------------------------------------------------------------
 // Merge + compact (Eq. 6-7, 10-12).  Every K and V row of the prompt is read exactly once: the
 // entry list of a (request, head) names, slot by slot, the kept row and then its members.  A warp
-// takes a work unit of consecutive entries (whole slots; sized so that there are about as many
-// units as resident warps, at least 32 entries) and walks it eight entries at a time: lanes 0-7
-// hold the entries' positions and weights (fetched one batch ahead), every lane loads 16 bytes of
-// each of the eight rows (lanes 0-15 the K row, lanes 16-31 the V row) and accumulates in fp32 in
-// member order; a kept entry closes the previous slot (one rounding, one 16-byte store per lane)
-// and opens the next.
+// takes a work unit of consecutive entries (whole slots; sized so that each warp gets about one
+// unit, at least 32 entries), fetches the rows 8 entries at
+// a time with 16-byte cp.async copies into its own shared-memory ring (three buffers; every lane
+// later reads back exactly the bytes it copied, so cp.async.wait_group is all the synchronisation
+// needed), and walks the staged rows in order: lanes 0-15 hold the K row, lanes 16-31 the V row,
+// 16 bytes per lane, fp32 accumulation in member order, one rounding.
 //   averaged : (x_c + sum x_e) / (n + 1)                       (Eq. 10)
 //   pivotal  : (x_c + 1/2 sum (x_e + x_c)) / (n + 1)           (Eq. 11)
 //   weighted : (x_c + sum sim_e x_e) / (n + 1)                 (Eq. 12)
-// A row without members is copied bit for bit.  No shared memory and at most 64 registers, so 32
-// warps are resident per SM, each with eight 512-byte row loads in flight: a plain gather of
-// 256-byte rows at full occupancy was measured at 5 TB/s on B200 whatever the order of the rows.
+// A row without members is copied bit for bit.  Sixteen warps per SM with 4 KB of copies in flight each keep
+// HBM busy while the dependent index loads of the next unit are outstanding.
 // ---------------------------------------------------------------------------------------------
-constexpr int kMergeWarps = 8;                       // per CTA
-#ifndef LOOKM_MERGE_CTAS
-#define LOOKM_MERGE_CTAS 4
-#endif
-#ifndef LOOKM_MERGE_BATCH
-#define LOOKM_MERGE_BATCH 8
-#endif
-constexpr int kMergeCtasPerSm = LOOKM_MERGE_CTAS;
-constexpr int kBatch = LOOKM_MERGE_BATCH;            // rows in flight per lane
+constexpr int kMergeWarps = 16;                      // per CTA; one CTA per SM
+constexpr int kChunk = 8;                            // entries staged per buffer
+constexpr int kRing = 3;                             // buffers per warp: two chunks in flight while one is read
+constexpr int kRowBytes = kHeadDim * 2;              // one bf16 row of K or V
 
-__device__ __forceinline__ uint4 ld_stream(const __nv_bfloat16* p) {
-    uint4 r;
-    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0, %1, %2, %3}, [%4];"
-                 : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "l"(p));
-    return r;
-}
+struct MergeShared {
+    alignas(128) uint8_t rows[kMergeWarps][kRing][kChunk][2 * kRowBytes];   // [warp][buffer][entry][K|V]
+};
 
 __device__ __forceinline__ const Req& find_req_by_unit(const Req* reqs, int n_req, long long g) {
     int lo = 0, hi = n_req - 1;
@@ -321,16 +311,22 @@ __device__ __forceinline__ const Req& find_req_by_unit(const Req* reqs, int n_re
     return reqs[lo];
 }
 
-__global__ void __launch_bounds__(kMergeWarps * 32, kMergeCtasPerSm)
+__global__ void __launch_bounds__(kMergeWarps * 32)
 merge_kernel(const __nv_bfloat16* __restrict__ k, const __nv_bfloat16* __restrict__ v,
              long long stride_tok, long long stride_head, const Req* __restrict__ reqs, int n_req,
-             int n_kv_heads, long long T, long long total_units, const int* __restrict__ ent_pos,
-             const float* __restrict__ ent_w, const int* __restrict__ unit_slot, int varlen_output,
-             __nv_bfloat16* __restrict__ out_k, __nv_bfloat16* __restrict__ out_v) {
+             int n_kv_heads, long long T, long long total_units, const int* __restrict__ row_ptr,
+             const int* __restrict__ ent_pos, const float* __restrict__ ent_w,
+             const int* __restrict__ unit_slot, int varlen_output,
+             __nv_bfloat16* __restrict__ out_k, __nv_bfloat16* __restrict__ out_v, int* status) {
+    extern __shared__ uint8_t merge_smem_raw[];
+    MergeShared& sh = *reinterpret_cast<MergeShared*>(
+        (reinterpret_cast<uintptr_t>(merge_smem_raw) + 127) & ~static_cast<uintptr_t>(127));
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int l16 = lane & 15;
+    const uint32_t buf0 = (uint32_t)__cvta_generic_to_shared(&sh.rows[warp][0][0][0]) + lane * 16;
     const __nv_bfloat16* tensor = lane < 16 ? k : v;
     __nv_bfloat16* dst_base = lane < 16 ? out_k : out_v;
+    uint32_t n_chunks_done = 0;                      // chunks this warp has consumed (buffer parity)
 
     for (long long g = (long long)blockIdx.x * kMergeWarps + warp; g < total_units;
          g += (long long)gridDim.x * kMergeWarps) {
@@ -339,30 +335,54 @@ merge_kernel(const __nv_bfloat16* __restrict__ k, const __nv_bfloat16* __restric
         const int n_units = (L + rq.unit_entries - 1) / rq.unit_entries;
         const long long ul = g - rq.unit_begin;
         // heads vary fastest: warps running at the same time then read the same token range of
-        // different heads
+        // different heads, i.e. neighbouring 256-byte rows of the same DRAM pages
         const int h = (int)(ul % n_kv_heads), u = (int)(ul / n_kv_heads);
-        const int* units = unit_slot + 2 * (rq.unit_store + (long long)h * (n_units + 1));
-        // lanes 0-3: (first slot, its entry index, one-past-last slot, its entry index)
-        int hdr = 0;
-        if (lane < 4) hdr = units[2 * u + lane];
-        const int c_lo = __shfl_sync(0xffffffffu, hdr, 0), e_lo = __shfl_sync(0xffffffffu, hdr, 1);
-        const int c_hi = __shfl_sync(0xffffffffu, hdr, 2), e_hi = __shfl_sync(0xffffffffu, hdr, 3);
+        const int* units = unit_slot + rq.unit_store + (long long)h * (n_units + 1);
+        const int* rp = row_ptr + rq.rp_off + (long long)h * (B + 1);
+        // lanes 0/1: first slot / one past the last slot of the unit, and their entry indices
+        int c_edge = 0, e_edge = 0;
+        if (lane < 2) {
+            c_edge = units[u + lane];
+            e_edge = c_edge + rp[c_edge];
+        }
+        const int c_lo = __shfl_sync(0xffffffffu, c_edge, 0), c_hi = __shfl_sync(0xffffffffu, c_edge, 1);
+        const int e_lo = __shfl_sync(0xffffffffu, e_edge, 0), e_hi = __shfl_sync(0xffffffffu, e_edge, 1);
         if (c_lo >= c_hi) continue;
         const int* ent = ent_pos + (long long)h * T + rq.tok_begin;
         const float* entw = ent_w + (long long)h * T + rq.tok_begin;
-        const __nv_bfloat16* src = tensor + (long long)rq.tok_begin * stride_tok +
-                                   (long long)h * stride_head + l16 * 8;
+        const __nv_bfloat16* src = tensor + (long long)rq.tok_begin * stride_tok + (long long)h * stride_head + l16 * 8;
+        const int n_chunks = (e_hi - e_lo + kChunk - 1) / kChunk;
 
-        // entry metadata of a batch (lanes 0-7: one entry each)
-        auto load_meta = [&](int e0, int& pos, float& w) {
+        // entry metadata of a chunk (lanes 0-7: one entry each)
+        auto load_meta = [&](int kc, int& pos, float& w) {
             pos = 0;
             w = 0.f;
-            const int e = e0 + lane;
-            if (lane < kBatch && e < e_hi) { pos = ent[e]; w = entw[e]; }
+            const int e = e_lo + kc * kChunk + lane;
+            if (lane < kChunk && kc < n_chunks && e < e_hi) { pos = ent[e]; w = entw[e]; }
         };
-        int pos_a, pos_b;
-        float w_a, w_b;
-        load_meta(e_lo, pos_a, w_a);
+        // start the row copies of chunk kc: for every entry, lanes 0-15 copy its K row and lanes
+        // 16-31 its V row, 16 bytes each; one commit group per chunk
+        auto issue = [&](int kc, int pos) {
+            const int cnt = min(kChunk, e_hi - e_lo - kc * kChunk);      // <= 0 past the unit: empty group
+            const uint32_t dst = buf0 + ((n_chunks_done + (uint32_t)kc) % kRing) * (kChunk * 2 * kRowBytes);
+#pragma unroll
+            for (int q = 0; q < kChunk; ++q) {
+                const int tok = __shfl_sync(0xffffffffu, pos, q) & 0x7fffffff;
+                if (q < cnt)
+                    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;"
+                                 ::"r"(dst + q * (2 * kRowBytes)), "l"(src + (long long)tok * stride_tok)
+                                 : "memory");
+            }
+            asm volatile("cp.async.commit_group;" ::: "memory");
+        };
+
+        int pos_a, pos_b, pos_c;
+        float w_a, w_b, w_c;
+        load_meta(0, pos_a, w_a);
+        load_meta(1, pos_b, w_b);
+        load_meta(2, pos_c, w_c);
+        issue(0, pos_a);
+        issue(1, pos_b);
 
         // running row
         int slot = c_lo - 1, n_mem = 0;
@@ -390,40 +410,46 @@ merge_kernel(const __nv_bfloat16* __restrict__ k, const __nv_bfloat16* __restric
             *reinterpret_cast<uint4*>(dst_base + row * kHeadDim + l16 * 8) = result;
         };
 
-        for (int e0 = e_lo; e0 < e_hi; e0 += kBatch) {
-            load_meta(e0 + kBatch, pos_b, w_b);              // next batch's metadata, used next turn
-            const int cnt = min(kBatch, e_hi - e0);
-            uint4 x4[kBatch];
+        for (int kc = 0; kc < n_chunks; ++kc) {
+            // chunk kc + 2 goes to the buffer whose rows were consumed one iteration ago; a commit
+            // group is made for every chunk index (empty past the unit), so "all but the two
+            // newest groups" always means: chunk kc has landed
+            issue(kc + 2, pos_c);
+            int pos_d;
+            float w_d;
+            load_meta(kc + 3, pos_d, w_d);
+            asm volatile("cp.async.wait_group 2;" ::: "memory");
+            const uint32_t b = (n_chunks_done + (uint32_t)kc) % kRing;
+            const int cnt = min(kChunk, e_hi - e_lo - kc * kChunk);
+            const uint8_t* base = &sh.rows[warp][b][0][0] + lane * 16;
 #pragma unroll
-            for (int q = 0; q < kBatch; ++q) {
-                const int tok = __shfl_sync(0xffffffffu, pos_a, q) & 0x7fffffff;
-                x4[q] = make_uint4(0u, 0u, 0u, 0u);
-                if (q < cnt) x4[q] = ld_stream(src + (long long)tok * stride_tok);
-            }
-#pragma unroll
-            for (int q = 0; q < kBatch; ++q) {
+            for (int q = 0; q < kChunk; ++q) {
                 const int pe = __shfl_sync(0xffffffffu, pos_a, q);
                 const float w = __shfl_sync(0xffffffffu, w_a, q);
-                if (q < cnt) {
-                    if (pe < 0) {                        // a kept row starts the next slot
-                        flush();
-                        ++slot;
-                        raw_c = x4[q];
-                        n_mem = (int)w;
+                if (q >= cnt) break;
+                const uint4 x4 = *reinterpret_cast<const uint4*>(base + q * (2 * kRowBytes));
+                if (pe < 0) {                        // a kept row starts the next slot
+                    flush();
+                    ++slot;
+                    raw_c = x4;
+                    n_mem = (int)w;
 #pragma unroll
-                        for (int i = 0; i < 8; ++i) acc[i] = 0.f;
-                    } else {
-                        const Row8 x = unpack8(x4[q]);
+                    for (int i = 0; i < 8; ++i) acc[i] = 0.f;
+                } else {
+                    const Row8 x = unpack8(x4);
 #pragma unroll
-                        for (int i = 0; i < 8; ++i) acc[i] = fmaf(w, x.v[i], acc[i]);
-                    }
+                    for (int i = 0; i < 8; ++i) acc[i] = fmaf(w, x.v[i], acc[i]);
                 }
             }
-            pos_a = pos_b;
-            w_a = w_b;
+            __syncwarp();
+            pos_a = pos_b; w_a = w_b;
+            pos_b = pos_c; w_b = w_c;
+            pos_c = pos_d; w_c = w_d;
         }
         flush();
+        n_chunks_done += (uint32_t)n_chunks;
     }
+    (void)status;
 }
 
 // Inverse map of given kept / evicted lists (used when the lists come from the caller).
@@ -500,20 +526,23 @@ cudaError_t launch_invert_assignment(const int* assign, const int* kept_idx, con
     return cudaGetLastError();
 }
 
-int merge_warps_per_sm() { return kMergeWarps * kMergeCtasPerSm; }
+int merge_warps_per_sm() { return kMergeWarps; }
 
 cudaError_t launch_merge(const void* k, const void* v, long long stride_tok, long long stride_head,
                          const Req* reqs, int n_req, int n_kv_heads, long long T,
-                         long long total_units, const int* ent_pos, const float* ent_w,
-                         const int* unit_slot, int varlen_output, void* out_k, void* out_v,
-                         int num_sms, cudaStream_t stream) {
+                         long long total_units, const int* row_ptr, const int* ent_pos,
+                         const float* ent_w, const int* unit_slot, int varlen_output, void* out_k,
+                         void* out_v, int* status, int num_sms, cudaStream_t stream) {
     if (total_units <= 0) return cudaSuccess;
+    const int smem = (int)sizeof(MergeShared) + 128;
+    cudaError_t err = cudaFuncSetAttribute(merge_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (err != cudaSuccess) return err;
     long long blocks = (total_units + kMergeWarps - 1) / kMergeWarps;
-    if (blocks > (long long)num_sms * kMergeCtasPerSm) blocks = (long long)num_sms * kMergeCtasPerSm;
-    merge_kernel<<<(unsigned)blocks, kMergeWarps * 32, 0, stream>>>(
+    if (blocks > num_sms) blocks = num_sms;              // persistent: one CTA per SM
+    merge_kernel<<<(unsigned)blocks, kMergeWarps * 32, smem, stream>>>(
         (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, stride_tok, stride_head, reqs, n_req,
-        n_kv_heads, T, total_units, ent_pos, ent_w, unit_slot, varlen_output,
-        (__nv_bfloat16*)out_k, (__nv_bfloat16*)out_v);
+        n_kv_heads, T, total_units, row_ptr, ent_pos, ent_w, unit_slot, varlen_output,
+        (__nv_bfloat16*)out_k, (__nv_bfloat16*)out_v, status);
     return cudaGetLastError();
 }
 
