@@ -161,14 +161,15 @@ int lookm_workspace_layout(const lookm_layout* layout, int n_requests, const int
  * inference server that has handed all device memory to its own pool and forbids driver
  * allocations on the serving path (they serialise with other streams), or a plug-in that runs
  * inside someone else's memory budget and has nowhere to put a workspace.  For them this variant
- * of lookm_merge keeps its scratch (request table, member lists, sort buffers, status word) in a
- * fixed array inside the library's device image, LOOKM_NOALLOC_SCRATCH_BYTES large, which every GPU
- * that loads the library holds until the process exits.  Inputs and outputs are still the
+ * of lookm_merge keeps its scratch (request table, entry lists, sort buffers, partial-sum records,
+ * status word) in a fixed array inside the library's device image, LOOKM_NOALLOC_SCRATCH_BYTES
+ * large, which every GPU that loads the library holds until the process exits.  Inputs and outputs are still the
  * caller's, with the meaning and layouts of lookm_merge.
  *
- * Limits: the scratch needs 28 bytes per (KV head, token) plus a small table, so
- * n_kv_heads * total_tokens may be at most about 299,000 (e.g. 32 heads x 8192 tokens uses
- * 7.3 MB); larger batches return LOOKM_ERR_WORKSPACE_TOO_SMALL before anything is enqueued.
+ * Limits: the scratch needs 28 bytes per (KV head, token), 4 per kept row and about 2.5 KB for
+ * each of the merge kernel's work units (one per warp of the GPU, about 6 MB on a 148-SM part), so
+ * n_kv_heads * total_tokens may be at most about 330,000 (32 heads x 8192 tokens uses 13.7 MB);
+ * larger batches return LOOKM_ERR_WORKSPACE_TOO_SMALL before anything is enqueued.
  * The call performs no cudaMalloc/cudaFree and calls no allocating routine.
  *
  * The first call on each device looks up the array's device address (cudaGetSymbolAddress, with
@@ -179,7 +180,7 @@ int lookm_workspace_layout(const lookm_layout* layout, int n_requests, const int
  * on one stream are safe; calls that can overlap on the GPU (different streams without an
  * ordering between them) race on the array and must be serialised by the caller.
  * lookm_noalloc_status() is lookm_device_status() for this scratch. */
-#define LOOKM_NOALLOC_SCRATCH_BYTES (8u << 20)
+#define LOOKM_NOALLOC_SCRATCH_BYTES (16u << 20)
 int lookm_merge_noalloc(const void* k, const void* v, const int* kept_idx, const int* evict_idx,
                         const int* assign, const float* sim, const int* cu_seqlens_host,
                         int n_requests, const int* budgets_host, const int* merge_modes_host,

@@ -30,12 +30,13 @@ struct Plan {
     int max_L = 0, max_E = 0;
     int n_items[3] = {0, 0, 0};
     long long total_slots = 0;              // n_kv_heads * sum_B
-    long long total_units = 0, unit_ints = 0;  // merge work units; ints in their boundary arrays
+    long long total_units = 0;              // merge work units
     std::vector<Req> reqs;                  // table order (longest first)
     std::vector<int> out_len;               // caller order
     // workspace offsets (bytes)
     size_t o_status, o_reqs, o_lse, o_scores, o_rank, o_rnorm_all, o_kept, o_evict, o_kept_keys,
-        o_rnorm_kept, o_assign, o_sim, o_row_ptr, o_members, o_member_w, o_units, o_sort_a, o_sort_b, total;
+        o_rnorm_kept, o_assign, o_sim, o_row_ptr, o_members, o_member_w, o_units, o_slot_cnt, o_parts, o_sort_a, o_sort_b,
+        total;
 };
 
 struct DeviceInfo { int sms = 0; int cc_major = 0; bool ok = false; };
@@ -95,7 +96,7 @@ int build_plan(Plan& pl, const lookm_layout* lay, int n_req, const int* cu_seqle
         return LOOKM_ERR_UNSUPPORTED;
     // table order: longest request first
     std::stable_sort(pl.reqs.begin(), pl.reqs.end(), [](const Req& a, const Req& b) { return a.L > b.L; });
-    long long it0 = 0, it1 = 0, it2 = 0, slots = 0, units = 0, unit_ints = 0;
+    long long it0 = 0, it1 = 0, it2 = 0, slots = 0, units = 0;
     // merge work units: about one per warp of the merge kernel (it reads n_kv_heads * T rows)
     int unit_entries = kMinUnitEntries;
     {
@@ -110,18 +111,15 @@ int build_plan(Plan& pl, const lookm_layout* lay, int n_req, const int* cu_seqle
         q.item_begin[kMatch] = (int)it2;
         q.slot_begin = (int)slots;
         q.unit_begin = (int)units;
-        q.unit_store = unit_ints;
         q.unit_entries = unit_entries;
         const long long n_units = (q.L + unit_entries - 1) / unit_entries;
         units += (long long)pl.n_kv_heads * n_units;
-        unit_ints += (long long)pl.n_kv_heads * (n_units + 1);
         it0 += (long long)q.nblk * pl.n_q_heads;
         it1 += (long long)q.nblk * pl.n_kv_heads;
         it2 += q.E > 0 ? (long long)q.nblk * pl.n_kv_heads : 0;
         slots += (long long)q.B * pl.n_kv_heads;
     }
     pl.total_units = units;
-    pl.unit_ints = unit_ints;
     pl.n_items[kSweep1] = (int)it0;
     pl.n_items[kSweep2] = (int)it1;
     pl.n_items[kMatch] = (int)it2;
@@ -146,7 +144,9 @@ int build_plan(Plan& pl, const lookm_layout* lay, int n_req, const int* cu_seqle
     pl.o_row_ptr = carve(4 * (Hkv * T + Hkv * (size_t)n_req));
     pl.o_members = carve(4 * Hkv * T);
     pl.o_member_w = carve(4 * Hkv * T);
-    pl.o_units = carve(4 * Hkv * (T / kMinUnitEntries + 2 * (size_t)n_req));
+    pl.o_units = carve(4 * (size_t)pl.total_units);
+    pl.o_slot_cnt = carve(4 * Hkv * T);
+    pl.o_parts = carve((size_t)kMergePartBytes * (size_t)pl.total_units);
     pl.o_sort_a = carve(8 * Hkv * T);
     pl.o_sort_b = carve(8 * Hkv * T);
     pl.total = o;
@@ -338,8 +338,8 @@ int run_merge(const Plan& pl, const lookm_layout* lay, const void* k, const void
     LOOKM_CUDA(launch_invert_assignment(assign, kept_idx, evict_idx, sim, reqs, pl.n_req, pl.n_kv_heads,
                                         pl.T, at<int>(ws, pl.o_row_ptr), at<int>(ws, pl.o_members),
                                         at<float>(ws, pl.o_member_w), at<int>(ws, pl.o_units),
-                                        at<unsigned>(ws, pl.o_sort_a), at<unsigned>(ws, pl.o_sort_b),
-                                        status, st));
+                                        at<int>(ws, pl.o_slot_cnt), at<unsigned>(ws, pl.o_sort_a),
+                                        at<unsigned>(ws, pl.o_sort_b), status, st));
     ++g_launches;
     mark_stage(6, st);
     DeviceInfo di;
@@ -347,7 +347,8 @@ int run_merge(const Plan& pl, const lookm_layout* lay, const void* k, const void
     LOOKM_CUDA(launch_merge(k, v, lay->kv_stride_tok, lay->kv_stride_head, reqs, pl.n_req,
                             pl.n_kv_heads, pl.T, pl.total_units, at<int>(ws, pl.o_row_ptr),
                             at<int>(ws, pl.o_members), at<float>(ws, pl.o_member_w),
-                            at<int>(ws, pl.o_units), varlen_output, out_k, out_v, status, di.sms, st));
+                            at<int>(ws, pl.o_units), at<int>(ws, pl.o_slot_cnt),
+                            at<float>(ws, pl.o_parts), varlen_output, out_k, out_v, status, di.sms, st));
     ++g_launches;
     mark_stage(7, st);
     return LOOKM_OK;
@@ -584,8 +585,8 @@ const char* lookm_strerror(int status) {
 // ------------------------------------------------------------------------------------------------
 namespace {
 
-// Scratch of the no-allocation merge: status word, request table, member lists (CSR) and the two
-// sort buffers.  Lives in the library's device image, so every GPU that loads the library holds
+// Scratch of the no-allocation merge: status word, request table, entry lists, per-slot counters,
+// per-unit records and the two sort buffers.  Lives in the library's device image, so every GPU that loads the library holds
 // these bytes until the process exits.
 static __device__ __align__(256) unsigned char g_noalloc_scratch[LOOKM_NOALLOC_SCRATCH_BYTES];
 
@@ -623,7 +624,8 @@ extern "C" int lookm_merge_noalloc(const void* k, const void* v, const int* kept
     LOOKM_TRY(build_plan(pl, layout, n_requests, cu_seqlens_host, nullptr, budgets_host, nullptr,
                          merge_modes_host));
     LOOKM_TRY(check_layout_ptrs(layout, nullptr, k, v));
-    // compact carving of just what the merge needs (28 bytes per (KV head, token) plus the table)
+    // compact carving of just what the merge needs: 28 bytes per (KV head, token), 4 per kept row,
+    // the per-unit records and the table
     const size_t units = (size_t)pl.n_kv_heads * (size_t)pl.T;
     size_t o = 0;
     auto carve = [&](size_t bytes) { size_t at = o; o = align_up(o + bytes, 256); return at; };
@@ -632,7 +634,9 @@ extern "C" int lookm_merge_noalloc(const void* k, const void* v, const int* kept
     pl.o_row_ptr = carve(4 * (units + (size_t)pl.n_kv_heads * (size_t)n_requests));
     pl.o_members = carve(4 * units);
     pl.o_member_w = carve(4 * units);
-    pl.o_units = carve(4 * ((size_t)pl.n_kv_heads * ((size_t)pl.T / kMinUnitEntries + 2 * (size_t)n_requests)));
+    pl.o_units = carve(4 * (size_t)pl.total_units);
+    pl.o_slot_cnt = carve(4 * (size_t)pl.total_slots);
+    pl.o_parts = carve((size_t)kMergePartBytes * (size_t)pl.total_units);
     pl.o_sort_a = carve(8 * units);
     pl.o_sort_b = carve(8 * units);
     pl.total = o;

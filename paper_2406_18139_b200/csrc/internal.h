@@ -12,6 +12,7 @@ namespace lookm {
 constexpr int kTile = 128;      // tokens per tile on either operand of the tensor-core kernels
 constexpr int kHeadDim = 128;   // only supported head_dim
 constexpr int kMinUnitEntries = 32; // least number of rows in a work unit of the merge kernel
+constexpr int kMergePartBytes = 2560; // per work unit: two fp32 partial K|V rows and one bf16 K|V row
 
 // One request of the packed batch as the kernels see it (device copy lives in the workspace).
 // Requests are stored longest first so that the heaviest work items are issued first.
@@ -31,11 +32,10 @@ struct Req {
                           // which hold B + 1 entries per head
     int item_begin[3];    // first work item of this request in sweep 1 / sweep 2 / match order
     int slot_begin;       // first (head, slot) row of this request in merge order (table order)
-    int unit_entries;     // rows read per merge work unit (whole slots): chosen per call so that
-                          // every warp of the merge kernel gets about one unit
-    int unit_begin;       // first merge work unit of this request (table order);
-                          // n_kv_heads * ceil(L / unit_entries) units per request
-    long long unit_store; // start of its unit-boundary arrays (ceil(L / unit_entries) + 1 ints per head)
+    int unit_entries;     // entries read per merge work unit: chosen per call so that every warp
+                          // of the merge kernel gets about one unit
+    int unit_begin;       // first merge work unit of this request (table order); n_kv_heads *
+                          // ceil(L / unit_entries) units per request, heads varying fastest
 };
 
 enum TileKind { kSweep1 = 0, kSweep2 = 1, kMatch = 2 };
@@ -90,15 +90,16 @@ cudaError_t launch_write_table(const ReqChunk& chunk, int count, Req* dst, cudaS
 cudaError_t launch_invert_assignment(const int* assign, const int* kept_idx, const int* evict_idx,
                                      const float* sim, const Req* reqs, int n_req, int n_kv_heads,
                                      long long T, int* row_ptr, int* ent_pos, float* ent_w,
-                                     int* unit_slot, unsigned* sort_a, unsigned* sort_b, int* status,
-                                     cudaStream_t stream);
+                                     int* unit_first, int* slot_cnt, unsigned* sort_a,
+                                     unsigned* sort_b, int* status, cudaStream_t stream);
 
 int merge_warps_per_sm();
 
 cudaError_t launch_merge(const void* k, const void* v, long long stride_tok, long long stride_head,
                          const Req* reqs, int n_req, int n_kv_heads, long long T,
                          long long total_units, const int* row_ptr, const int* ent_pos,
-                         const float* ent_w, const int* unit_slot, int varlen_output, void* out_k,
-                         void* out_v, int* status, int num_sms, cudaStream_t stream);
+                         const float* ent_w, const int* unit_first, int* slot_cnt, float* parts,
+                         int varlen_output, void* out_k, void* out_v, int* status, int num_sms,
+                         cudaStream_t stream);
 
 }  // namespace lookm

@@ -133,26 +133,24 @@ argmax_rows_kernel(const float* __restrict__ sim_matrix, const Req* __restrict__
 // ---------------------------------------------------------------------------------------------
 constexpr int kInvThreads = 1024;
 
-// Second half of the entry list: the kept rows (flagged with the sign bit, weight = member count)
-// and the work-unit boundaries: unit u covers the slots [units[u], units[u+1]), where units[u] is
-// the first slot whose entry index c + row_ptr[c] is >= u * unit_entries.
-__device__ __forceinline__ void write_kept_entries(const Req& rq, int h, int B, int E, const int* rp,
+// Second half of the entry list: the kept rows (flagged with the sign bit, weight = member count),
+// the slot that the first entry of every work unit belongs to (unit u of a head covers the entries
+// [u * unit_entries, (u + 1) * unit_entries)), and a cleared arrival counter per slot.
+__device__ __forceinline__ void write_kept_entries(const Req& rq, int h, int n_kv_heads, int B, const int* rp,
                                                    const int* kept_idx_head, int* ent, float* entw,
-                                                   int* units, int* status) {
+                                                   int* unit_first, int* slot_cnt, int* status) {
     const int ue = rq.unit_entries;
-    const int n_units = (rq.L + ue - 1) / ue;
     for (int c = threadIdx.x; c < B; c += blockDim.x) {
         int pc = kept_idx_head[c];
         if (pc < 0 || pc >= rq.L) { atomicExch(status, (int)LOOKM_ERR_DEVICE_BAD_INDEX); pc = 0; }
-        const int s_c = c + rp[c];
+        const int s_c = c + rp[c];                       // entry of the kept row
+        const int s_next = c + 1 + rp[c + 1];            // entry of the next kept row (L after the last)
         ent[s_c] = pc | (int)0x80000000;
         entw[s_c] = (float)(rp[c + 1] - rp[c]);
-        const int s_prev = c ? (c - 1) + rp[c - 1] : -1;
-        for (int u = s_prev / ue + (s_prev >= 0 ? 1 : 0); u * ue <= s_c; ++u) units[u] = c;
-        if (c == B - 1)
-            for (int u = s_c / ue + 1; u <= n_units; ++u) units[u] = B;
+        slot_cnt[c] = 0;
+        for (int u = (s_c + ue - 1) / ue; u * ue < s_next; ++u)
+            unit_first[(long long)u * n_kv_heads + h] = c;
     }
-    (void)h; (void)E;
 }
 
 __global__ void __launch_bounds__(kInvThreads)
@@ -161,8 +159,8 @@ invert_assignment_kernel(const int* __restrict__ assign, const int* __restrict__
                          const float* __restrict__ sim, const Req* __restrict__ reqs,
                          int n_kv_heads, long long T, int* __restrict__ row_ptr,
                          int* __restrict__ ent_pos, float* __restrict__ ent_w,
-                         int* __restrict__ unit_slot, unsigned* __restrict__ sort_a,
-                         unsigned* __restrict__ sort_b, int* status) {
+                         int* __restrict__ unit_first, int* __restrict__ slot_cnt,
+                         unsigned* __restrict__ sort_a, unsigned* __restrict__ sort_b, int* status) {
     __shared__ int cnt[32][256];                         // [warp][digit]
     __shared__ int digit_tot[256];
     const Req rq = reqs[blockIdx.y];
@@ -176,14 +174,14 @@ invert_assignment_kernel(const int* __restrict__ assign, const int* __restrict__
     // entry list of this (request, head): for every kept slot its kept row, then its members
     int* ent = ent_pos + (long long)h * T + rq.tok_begin;
     float* entw = ent_w + (long long)h * T + rq.tok_begin;
-    const int n_units = (rq.L + rq.unit_entries - 1) / rq.unit_entries;
-    int* units = unit_slot + rq.unit_store + (long long)h * (n_units + 1);
+    int* units = unit_first + rq.unit_begin;             // [unit of the head][head]
+    int* cnts = slot_cnt + rq.kept_off + (long long)h * B;
     const int* kept_idx_head = kept_idx + rq.kept_off + (long long)h * B;
     const bool weighted = (rq.mode == LOOKM_MERGE_WEIGHTED);
     if (E == 0) {
         for (int c = threadIdx.x; c <= B; c += kInvThreads) rp[c] = 0;
         __syncthreads();
-        write_kept_entries(rq, h, B, E, rp, kept_idx_head, ent, entw, units, status);
+        write_kept_entries(rq, h, n_kv_heads, B, rp, kept_idx_head, ent, entw, units, cnts, status);
         return;
     }
     // segment of the list owned by each warp: a multiple of 32 elements
@@ -275,28 +273,38 @@ invert_assignment_kernel(const int* __restrict__ assign, const int* __restrict__
         if (i == E - 1) for (int c = cur + 1; c <= B; ++c) rp[c] = E;
     }
     __syncthreads();
-    write_kept_entries(rq, h, B, E, rp, kept_idx_head, ent, entw, units, status);
+    write_kept_entries(rq, h, n_kv_heads, B, rp, kept_idx_head, ent, entw, units, cnts, status);
 }
 
 // ---------------------------------------------------------------------------------------------
 // Merge + compact (Eq. 6-7, 10-12).  Every K and V row of the prompt is read exactly once: the
 // entry list of a (request, head) names, slot by slot, the kept row and then its members.  A warp
-// takes a work unit of consecutive entries (whole slots; sized so that each warp gets about one
-// unit, at least 32 entries), fetches the rows 8 entries at
-// a time with 16-byte cp.async copies into its own shared-memory ring (three buffers; every lane
-// later reads back exactly the bytes it copied, so cp.async.wait_group is all the synchronisation
-// needed), and walks the staged rows in order: lanes 0-15 hold the K row, lanes 16-31 the V row,
-// 16 bytes per lane, fp32 accumulation in member order, one rounding.
+// takes a work unit of unit_entries consecutive entries (sized so that each warp gets about one
+// unit, at least 32 entries), fetches the rows 8 entries at a time with 16-byte cp.async copies
+// into its own shared-memory ring (three buffers; every lane later reads back exactly the bytes it
+// copied, so cp.async.wait_group is all the synchronisation needed), and walks the staged rows in
+// order: lanes 0-15 hold the K row, lanes 16-31 the V row, 16 bytes per lane, fp32 accumulation in
+// member order, one rounding.
 //   averaged : (x_c + sum x_e) / (n + 1)                       (Eq. 10)
 //   pivotal  : (x_c + 1/2 sum (x_e + x_c)) / (n + 1)           (Eq. 11)
 //   weighted : (x_c + sum sim_e x_e) / (n + 1)                 (Eq. 12)
-// A row without members is copied bit for bit.  Sixteen warps per SM with 4 KB of copies in flight each keep
-// HBM busy while the dependent index loads of the next unit are outstanding.
+// A row without members is copied bit for bit.
+//
+// Units are cut at fixed entry counts, not at slot boundaries, so that every warp has the same
+// amount to read however skewed the member counts are.  A slot whose entries straddle units is
+// summed piecewise: every unit that holds a piece stores its fp32 partial sum (the unit with the
+// kept row also stores that row) in its own record, then bumps the slot's arrival counter; the
+// warp that arrives last adds the pieces in unit order and writes the row.  Nobody waits for
+// anybody, and the order of the additions does not depend on who came last.
 // ---------------------------------------------------------------------------------------------
 constexpr int kMergeWarps = 16;                      // per CTA; one CTA per SM
 constexpr int kChunk = 8;                            // entries staged per buffer
 constexpr int kRing = 3;                             // buffers per warp: two chunks in flight while one is read
 constexpr int kRowBytes = kHeadDim * 2;              // one bf16 row of K or V
+// Record of a unit: [0, 1024) partial sums of its leading piece (slot begun in an earlier unit),
+// [1024, 2048) partial sums of its trailing piece (slot that goes on in the next unit),
+// [2048, 2560) the kept K|V row of the trailing piece.  Per piece: 8 floats (or 16 bytes) per lane.
+constexpr int kPartFloats = kMergePartBytes / 4;
 
 struct MergeShared {
     alignas(128) uint8_t rows[kMergeWarps][kRing][kChunk][2 * kRowBytes];   // [warp][buffer][entry][K|V]
@@ -311,13 +319,16 @@ __device__ __forceinline__ const Req& find_req_by_unit(const Req* reqs, int n_re
     return reqs[lo];
 }
 
+__device__ __forceinline__ float4 ld_cg_f4(const float* p) { return __ldcg(reinterpret_cast<const float4*>(p)); }
+
 __global__ void __launch_bounds__(kMergeWarps * 32)
 merge_kernel(const __nv_bfloat16* __restrict__ k, const __nv_bfloat16* __restrict__ v,
              long long stride_tok, long long stride_head, const Req* __restrict__ reqs, int n_req,
              int n_kv_heads, long long T, long long total_units, const int* __restrict__ row_ptr,
              const int* __restrict__ ent_pos, const float* __restrict__ ent_w,
-             const int* __restrict__ unit_slot, int varlen_output,
-             __nv_bfloat16* __restrict__ out_k, __nv_bfloat16* __restrict__ out_v, int* status) {
+             const int* __restrict__ unit_first, int* __restrict__ slot_cnt, float* __restrict__ parts,
+             int varlen_output, __nv_bfloat16* __restrict__ out_k, __nv_bfloat16* __restrict__ out_v,
+             int* status) {
     extern __shared__ uint8_t merge_smem_raw[];
     MergeShared& sh = *reinterpret_cast<MergeShared*>(
         (reinterpret_cast<uintptr_t>(merge_smem_raw) + 127) & ~static_cast<uintptr_t>(127));
@@ -331,23 +342,16 @@ merge_kernel(const __nv_bfloat16* __restrict__ k, const __nv_bfloat16* __restric
     for (long long g = (long long)blockIdx.x * kMergeWarps + warp; g < total_units;
          g += (long long)gridDim.x * kMergeWarps) {
         const Req& rq = find_req_by_unit(reqs, n_req, g);
-        const int L = rq.L, B = rq.B, mode = rq.mode;
-        const int n_units = (L + rq.unit_entries - 1) / rq.unit_entries;
+        const int L = rq.L, B = rq.B, mode = rq.mode, ue = rq.unit_entries;
         const long long ul = g - rq.unit_begin;
         // heads vary fastest: warps running at the same time then read the same token range of
         // different heads, i.e. neighbouring 256-byte rows of the same DRAM pages
         const int h = (int)(ul % n_kv_heads), u = (int)(ul / n_kv_heads);
-        const int* units = unit_slot + rq.unit_store + (long long)h * (n_units + 1);
+        const int e_lo = u * ue, e_hi = min(L, e_lo + ue);
+        int first_slot = 0;
+        if (lane == 0) first_slot = unit_first[g];   // used at the first flush only
         const int* rp = row_ptr + rq.rp_off + (long long)h * (B + 1);
-        // lanes 0/1: first slot / one past the last slot of the unit, and their entry indices
-        int c_edge = 0, e_edge = 0;
-        if (lane < 2) {
-            c_edge = units[u + lane];
-            e_edge = c_edge + rp[c_edge];
-        }
-        const int c_lo = __shfl_sync(0xffffffffu, c_edge, 0), c_hi = __shfl_sync(0xffffffffu, c_edge, 1);
-        const int e_lo = __shfl_sync(0xffffffffu, e_edge, 0), e_hi = __shfl_sync(0xffffffffu, e_edge, 1);
-        if (c_lo >= c_hi) continue;
+        int* cnt = slot_cnt + rq.kept_off + (long long)h * B;
         const int* ent = ent_pos + (long long)h * T + rq.tok_begin;
         const float* entw = ent_w + (long long)h * T + rq.tok_begin;
         const __nv_bfloat16* src = tensor + (long long)rq.tok_begin * stride_tok + (long long)h * stride_head + l16 * 8;
@@ -363,12 +367,12 @@ merge_kernel(const __nv_bfloat16* __restrict__ k, const __nv_bfloat16* __restric
         // start the row copies of chunk kc: for every entry, lanes 0-15 copy its K row and lanes
         // 16-31 its V row, 16 bytes each; one commit group per chunk
         auto issue = [&](int kc, int pos) {
-            const int cnt = min(kChunk, e_hi - e_lo - kc * kChunk);      // <= 0 past the unit: empty group
+            const int n_ent = min(kChunk, e_hi - e_lo - kc * kChunk);    // <= 0 past the unit: empty group
             const uint32_t dst = buf0 + ((n_chunks_done + (uint32_t)kc) % kRing) * (kChunk * 2 * kRowBytes);
 #pragma unroll
             for (int q = 0; q < kChunk; ++q) {
                 const int tok = __shfl_sync(0xffffffffu, pos, q) & 0x7fffffff;
-                if (q < cnt)
+                if (q < n_ent)
                     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;"
                                  ::"r"(dst + q * (2 * kRowBytes)), "l"(src + (long long)tok * stride_tok)
                                  : "memory");
@@ -384,30 +388,77 @@ merge_kernel(const __nv_bfloat16* __restrict__ k, const __nv_bfloat16* __restric
         issue(0, pos_a);
         issue(1, pos_b);
 
-        // running row
-        int slot = c_lo - 1, n_mem = 0;
+        // running piece: the slot, whether its kept row was met in this unit, the members met
+        const bool starts_with_kept = __shfl_sync(0xffffffffu, pos_a, 0) < 0;
+        first_slot = __shfl_sync(0xffffffffu, first_slot, 0);
+        int slot = starts_with_kept ? first_slot - 1 : first_slot;
+        bool active = !starts_with_kept, have_kept = false;
+        int n_mem = 0, n_seen = 0;
         uint4 raw_c = make_uint4(0u, 0u, 0u, 0u);
         float acc[8];
 #pragma unroll
         for (int i = 0; i < 8; ++i) acc[i] = 0.f;
-        auto flush = [&]() {
-            if (slot < c_lo) return;
-            uint4 result = raw_c;
-            if (n_mem > 0) {
-                const Row8 xc = unpack8(raw_c);
-                const float inv = 1.0f / (float)(n_mem + 1);
+
+        auto write_row = [&](int c, const uint4& kept_raw, const float* sum, int n) {
+            uint4 result = kept_raw;
+            if (n > 0) {
+                const Row8 xc = unpack8(kept_raw);
+                const float inv = 1.0f / (float)(n + 1);
                 // pivotal: each member contributes (x_e + x_c) / 2
-                const float wc = (mode == LOOKM_MERGE_PIVOTAL) ? 1.f + 0.5f * (float)n_mem : 1.f;
+                const float wc = (mode == LOOKM_MERGE_PIVOTAL) ? 1.f + 0.5f * (float)n : 1.f;
                 const float wm = (mode == LOOKM_MERGE_PIVOTAL) ? 0.5f : 1.f;
                 Row8 o;
 #pragma unroll
-                for (int i = 0; i < 8; ++i) o.v[i] = fmaf(wc, xc.v[i], wm * acc[i]) * inv;
+                for (int i = 0; i < 8; ++i) o.v[i] = fmaf(wc, xc.v[i], wm * sum[i]) * inv;
                 result = pack8(o);
             }
             long long row;
-            if (varlen_output) row = ((long long)rq.out_begin + slot) * n_kv_heads + h;
-            else row = (long long)h * B + slot;
+            if (varlen_output) row = ((long long)rq.out_begin + c) * n_kv_heads + h;
+            else row = (long long)h * B + c;
             *reinterpret_cast<uint4*>(dst_base + row * kHeadDim + l16 * 8) = result;
+        };
+        // a piece of a slot that other units share: publish it, and finish the row if it is the last
+        auto publish_piece = [&]() {
+            float* rec = parts + g * kPartFloats + (have_kept ? 256 : 0) + lane * 8;
+            *reinterpret_cast<float4*>(rec) = make_float4(acc[0], acc[1], acc[2], acc[3]);
+            *reinterpret_cast<float4*>(rec + 4) = make_float4(acc[4], acc[5], acc[6], acc[7]);
+            if (have_kept) *reinterpret_cast<uint4*>(parts + g * kPartFloats + 512 + lane * 4) = raw_c;
+            __threadfence();
+            __syncwarp();
+            int a = 0, b = 0, old = 0;
+            if (lane == 0) {
+                a = rp[slot];
+                b = rp[slot + 1];
+                old = atomicAdd(cnt + slot, 1);
+            }
+            a = __shfl_sync(0xffffffffu, a, 0);
+            b = __shfl_sync(0xffffffffu, b, 0);
+            old = __shfl_sync(0xffffffffu, old, 0);
+            const int u0 = (slot + a) / ue;              // unit of the kept row
+            const int u1 = (slot + b) / ue;              // unit of the last member
+            if (old != u1 - u0) return;                  // pieces still missing
+            __threadfence();
+            const long long g0 = (long long)rq.unit_begin + (long long)u0 * n_kv_heads + h;
+            const float* r0 = parts + g0 * kPartFloats;
+            float sum[8];
+            {
+                const float4 lo = ld_cg_f4(r0 + 256 + lane * 8), hi = ld_cg_f4(r0 + 256 + lane * 8 + 4);
+                sum[0] = lo.x; sum[1] = lo.y; sum[2] = lo.z; sum[3] = lo.w;
+                sum[4] = hi.x; sum[5] = hi.y; sum[6] = hi.z; sum[7] = hi.w;
+            }
+            const uint4 kept_raw = __ldcg(reinterpret_cast<const uint4*>(r0 + 512 + lane * 4));
+            for (int uu = u0 + 1; uu <= u1; ++uu) {
+                const float* r = r0 + (long long)(uu - u0) * n_kv_heads * kPartFloats;
+                const float4 lo = ld_cg_f4(r + lane * 8), hi = ld_cg_f4(r + lane * 8 + 4);
+                sum[0] += lo.x; sum[1] += lo.y; sum[2] += lo.z; sum[3] += lo.w;
+                sum[4] += hi.x; sum[5] += hi.y; sum[6] += hi.z; sum[7] += hi.w;
+            }
+            write_row(slot, kept_raw, sum, b - a);
+        };
+        auto flush = [&]() {
+            if (!active) return;
+            if (have_kept && n_seen == n_mem) write_row(slot, raw_c, acc, n_mem);
+            else publish_piece();
         };
 
         for (int kc = 0; kc < n_chunks; ++kc) {
@@ -420,23 +471,27 @@ merge_kernel(const __nv_bfloat16* __restrict__ k, const __nv_bfloat16* __restric
             load_meta(kc + 3, pos_d, w_d);
             asm volatile("cp.async.wait_group 2;" ::: "memory");
             const uint32_t b = (n_chunks_done + (uint32_t)kc) % kRing;
-            const int cnt = min(kChunk, e_hi - e_lo - kc * kChunk);
+            const int n_ent = min(kChunk, e_hi - e_lo - kc * kChunk);
             const uint8_t* base = &sh.rows[warp][b][0][0] + lane * 16;
 #pragma unroll
             for (int q = 0; q < kChunk; ++q) {
                 const int pe = __shfl_sync(0xffffffffu, pos_a, q);
                 const float w = __shfl_sync(0xffffffffu, w_a, q);
-                if (q >= cnt) break;
+                if (q >= n_ent) break;
                 const uint4 x4 = *reinterpret_cast<const uint4*>(base + q * (2 * kRowBytes));
                 if (pe < 0) {                        // a kept row starts the next slot
                     flush();
                     ++slot;
+                    active = true;
+                    have_kept = true;
                     raw_c = x4;
                     n_mem = (int)w;
+                    n_seen = 0;
 #pragma unroll
                     for (int i = 0; i < 8; ++i) acc[i] = 0.f;
                 } else {
                     const Row8 x = unpack8(x4);
+                    ++n_seen;
 #pragma unroll
                     for (int i = 0; i < 8; ++i) acc[i] = fmaf(w, x.v[i], acc[i]);
                 }
@@ -517,12 +572,13 @@ cudaError_t launch_gather_kept(const void* k, long long stride_tok, long long st
 cudaError_t launch_invert_assignment(const int* assign, const int* kept_idx, const int* evict_idx,
                                      const float* sim, const Req* reqs, int n_req, int n_kv_heads,
                                      long long T, int* row_ptr, int* ent_pos, float* ent_w,
-                                     int* unit_slot, unsigned* sort_a, unsigned* sort_b, int* status,
-                                     cudaStream_t stream) {
+                                     int* unit_first, int* slot_cnt, unsigned* sort_a,
+                                     unsigned* sort_b, int* status, cudaStream_t stream) {
     dim3 grid(n_kv_heads, n_req);
     invert_assignment_kernel<<<grid, kInvThreads, 0, stream>>>(assign, kept_idx, evict_idx, sim, reqs,
                                                                n_kv_heads, T, row_ptr, ent_pos, ent_w,
-                                                               unit_slot, sort_a, sort_b, status);
+                                                               unit_first, slot_cnt, sort_a, sort_b,
+                                                               status);
     return cudaGetLastError();
 }
 
@@ -531,8 +587,9 @@ int merge_warps_per_sm() { return kMergeWarps; }
 cudaError_t launch_merge(const void* k, const void* v, long long stride_tok, long long stride_head,
                          const Req* reqs, int n_req, int n_kv_heads, long long T,
                          long long total_units, const int* row_ptr, const int* ent_pos,
-                         const float* ent_w, const int* unit_slot, int varlen_output, void* out_k,
-                         void* out_v, int* status, int num_sms, cudaStream_t stream) {
+                         const float* ent_w, const int* unit_first, int* slot_cnt, float* parts,
+                         int varlen_output, void* out_k, void* out_v, int* status, int num_sms,
+                         cudaStream_t stream) {
     if (total_units <= 0) return cudaSuccess;
     const int smem = (int)sizeof(MergeShared) + 128;
     cudaError_t err = cudaFuncSetAttribute(merge_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
@@ -541,7 +598,7 @@ cudaError_t launch_merge(const void* k, const void* v, long long stride_tok, lon
     if (blocks > num_sms) blocks = num_sms;              // persistent: one CTA per SM
     merge_kernel<<<(unsigned)blocks, kMergeWarps * 32, smem, stream>>>(
         (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, stride_tok, stride_head, reqs, n_req,
-        n_kv_heads, T, total_units, row_ptr, ent_pos, ent_w, unit_slot, varlen_output,
+        n_kv_heads, T, total_units, row_ptr, ent_pos, ent_w, unit_first, slot_cnt, parts, varlen_output,
         (__nv_bfloat16*)out_k, (__nv_bfloat16*)out_v, status);
     return cudaGetLastError();
 }
