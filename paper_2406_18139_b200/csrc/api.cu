@@ -144,7 +144,7 @@ int build_plan(Plan& pl, const lookm_layout* lay, int n_req, const int* cu_seqle
     pl.o_row_ptr = carve(4 * (Hkv * T + Hkv * (size_t)n_req));
     pl.o_members = carve(4 * Hkv * T);
     pl.o_member_w = carve(4 * Hkv * T);
-    pl.o_units = carve(4 * (size_t)pl.total_units);
+    pl.o_units = carve(16 * (size_t)pl.total_units);
     pl.o_slot_cnt = carve(4 * Hkv * T);
     pl.o_parts = carve((size_t)kMergePartBytes * (size_t)pl.total_units);
     pl.o_sort_a = carve(8 * Hkv * T);
@@ -337,7 +337,7 @@ int run_merge(const Plan& pl, const lookm_layout* lay, const void* k, const void
     int* status = at<int>(ws, pl.o_status);
     LOOKM_CUDA(launch_invert_assignment(assign, kept_idx, evict_idx, sim, reqs, pl.n_req, pl.n_kv_heads,
                                         pl.T, at<int>(ws, pl.o_row_ptr), at<int>(ws, pl.o_members),
-                                        at<float>(ws, pl.o_member_w), at<int>(ws, pl.o_units),
+                                        at<float>(ws, pl.o_member_w), at<int4>(ws, pl.o_units),
                                         at<int>(ws, pl.o_slot_cnt), at<unsigned>(ws, pl.o_sort_a),
                                         at<unsigned>(ws, pl.o_sort_b), status, st));
     ++g_launches;
@@ -347,7 +347,7 @@ int run_merge(const Plan& pl, const lookm_layout* lay, const void* k, const void
     LOOKM_CUDA(launch_merge(k, v, lay->kv_stride_tok, lay->kv_stride_head, reqs, pl.n_req,
                             pl.n_kv_heads, pl.T, pl.total_units, at<int>(ws, pl.o_row_ptr),
                             at<int>(ws, pl.o_members), at<float>(ws, pl.o_member_w),
-                            at<int>(ws, pl.o_units), at<int>(ws, pl.o_slot_cnt),
+                            at<int4>(ws, pl.o_units), at<int>(ws, pl.o_slot_cnt),
                             at<float>(ws, pl.o_parts), varlen_output, out_k, out_v, status, di.sms, st));
     ++g_launches;
     mark_stage(7, st);
@@ -634,7 +634,7 @@ extern "C" int lookm_merge_noalloc(const void* k, const void* v, const int* kept
     pl.o_row_ptr = carve(4 * (units + (size_t)pl.n_kv_heads * (size_t)n_requests));
     pl.o_members = carve(4 * units);
     pl.o_member_w = carve(4 * units);
-    pl.o_units = carve(4 * (size_t)pl.total_units);
+    pl.o_units = carve(16 * (size_t)pl.total_units);
     pl.o_slot_cnt = carve(4 * (size_t)pl.total_slots);
     pl.o_parts = carve((size_t)kMergePartBytes * (size_t)pl.total_units);
     pl.o_sort_a = carve(8 * units);

@@ -90,7 +90,7 @@ cudaError_t launch_write_table(const ReqChunk& chunk, int count, Req* dst, cudaS
 cudaError_t launch_invert_assignment(const int* assign, const int* kept_idx, const int* evict_idx,
                                      const float* sim, const Req* reqs, int n_req, int n_kv_heads,
                                      long long T, int* row_ptr, int* ent_pos, float* ent_w,
-                                     int* unit_first, int* slot_cnt, unsigned* sort_a,
+                                     int4* unit_first, int* slot_cnt, unsigned* sort_a,
                                      unsigned* sort_b, int* status, cudaStream_t stream);
 
 int merge_warps_per_sm();
@@ -98,7 +98,7 @@ int merge_warps_per_sm();
 cudaError_t launch_merge(const void* k, const void* v, long long stride_tok, long long stride_head,
                          const Req* reqs, int n_req, int n_kv_heads, long long T,
                          long long total_units, const int* row_ptr, const int* ent_pos,
-                         const float* ent_w, const int* unit_first, int* slot_cnt, float* parts,
+                         const float* ent_w, const int4* unit_first, int* slot_cnt, float* parts,
                          int varlen_output, void* out_k, void* out_v, int* status, int num_sms,
                          cudaStream_t stream);
 

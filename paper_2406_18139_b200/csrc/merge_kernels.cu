@@ -134,11 +134,12 @@ argmax_rows_kernel(const float* __restrict__ sim_matrix, const Req* __restrict__
 constexpr int kInvThreads = 1024;
 
 // Second half of the entry list: the kept rows (flagged with the sign bit, weight = member count),
-// the slot that the first entry of every work unit belongs to (unit u of a head covers the entries
-// [u * unit_entries, (u + 1) * unit_entries)), and a cleared arrival counter per slot.
+// for every work unit (unit u of a head covers the entries [u * unit_entries, (u + 1) * unit_entries))
+// the slot its first entry belongs to, with that slot's first entry and member count, and a
+// cleared arrival counter per slot.
 __device__ __forceinline__ void write_kept_entries(const Req& rq, int h, int n_kv_heads, int B, const int* rp,
                                                    const int* kept_idx_head, int* ent, float* entw,
-                                                   int* unit_first, int* slot_cnt, int* status) {
+                                                   int4* unit_first, int* slot_cnt, int* status) {
     const int ue = rq.unit_entries;
     for (int c = threadIdx.x; c < B; c += blockDim.x) {
         int pc = kept_idx_head[c];
@@ -149,7 +150,7 @@ __device__ __forceinline__ void write_kept_entries(const Req& rq, int h, int n_k
         entw[s_c] = (float)(rp[c + 1] - rp[c]);
         slot_cnt[c] = 0;
         for (int u = (s_c + ue - 1) / ue; u * ue < s_next; ++u)
-            unit_first[(long long)u * n_kv_heads + h] = c;
+            unit_first[(long long)u * n_kv_heads + h] = make_int4(c, s_c, rp[c + 1] - rp[c], 0);
     }
 }
 
@@ -159,7 +160,7 @@ invert_assignment_kernel(const int* __restrict__ assign, const int* __restrict__
                          const float* __restrict__ sim, const Req* __restrict__ reqs,
                          int n_kv_heads, long long T, int* __restrict__ row_ptr,
                          int* __restrict__ ent_pos, float* __restrict__ ent_w,
-                         int* __restrict__ unit_first, int* __restrict__ slot_cnt,
+                         int4* __restrict__ unit_first, int* __restrict__ slot_cnt,
                          unsigned* __restrict__ sort_a, unsigned* __restrict__ sort_b, int* status) {
     __shared__ int cnt[32][256];                         // [warp][digit]
     __shared__ int digit_tot[256];
@@ -174,7 +175,7 @@ invert_assignment_kernel(const int* __restrict__ assign, const int* __restrict__
     // entry list of this (request, head): for every kept slot its kept row, then its members
     int* ent = ent_pos + (long long)h * T + rq.tok_begin;
     float* entw = ent_w + (long long)h * T + rq.tok_begin;
-    int* units = unit_first + rq.unit_begin;             // [unit of the head][head]
+    int4* units = unit_first + rq.unit_begin;            // [unit of the head][head]
     int* cnts = slot_cnt + rq.kept_off + (long long)h * B;
     const int* kept_idx_head = kept_idx + rq.kept_off + (long long)h * B;
     const bool weighted = (rq.mode == LOOKM_MERGE_WEIGHTED);
@@ -326,7 +327,7 @@ merge_kernel(const __nv_bfloat16* __restrict__ k, const __nv_bfloat16* __restric
              long long stride_tok, long long stride_head, const Req* __restrict__ reqs, int n_req,
              int n_kv_heads, long long T, long long total_units, const int* __restrict__ row_ptr,
              const int* __restrict__ ent_pos, const float* __restrict__ ent_w,
-             const int* __restrict__ unit_first, int* __restrict__ slot_cnt, float* __restrict__ parts,
+             const int4* __restrict__ unit_first, int* __restrict__ slot_cnt, float* __restrict__ parts,
              int varlen_output, __nv_bfloat16* __restrict__ out_k, __nv_bfloat16* __restrict__ out_v,
              int* status) {
     extern __shared__ uint8_t merge_smem_raw[];
@@ -348,9 +349,8 @@ merge_kernel(const __nv_bfloat16* __restrict__ k, const __nv_bfloat16* __restric
         // different heads, i.e. neighbouring 256-byte rows of the same DRAM pages
         const int h = (int)(ul % n_kv_heads), u = (int)(ul / n_kv_heads);
         const int e_lo = u * ue, e_hi = min(L, e_lo + ue);
-        int first_slot = 0;
-        if (lane == 0) first_slot = unit_first[g];   // used at the first flush only
-        const int* rp = row_ptr + rq.rp_off + (long long)h * (B + 1);
+        int4 first = make_int4(0, 0, 0, 0);           // slot of the first entry; its first entry, member count
+        if (lane == 0) first = __ldg(unit_first + g); // needed at the first kept row at the earliest
         int* cnt = slot_cnt + rq.kept_off + (long long)h * B;
         const int* ent = ent_pos + (long long)h * T + rq.tok_begin;
         const float* entw = ent_w + (long long)h * T + rq.tok_begin;
@@ -388,12 +388,14 @@ merge_kernel(const __nv_bfloat16* __restrict__ k, const __nv_bfloat16* __restric
         issue(0, pos_a);
         issue(1, pos_b);
 
-        // running piece: the slot, whether its kept row was met in this unit, the members met
+        // running piece: the slot, whether its kept row was met in this unit (and at which entry),
+        // the members met
         const bool starts_with_kept = __shfl_sync(0xffffffffu, pos_a, 0) < 0;
-        first_slot = __shfl_sync(0xffffffffu, first_slot, 0);
+        const int first_slot = __shfl_sync(0xffffffffu, first.x, 0);
         int slot = starts_with_kept ? first_slot - 1 : first_slot;
         bool active = !starts_with_kept, have_kept = false;
-        int n_mem = 0, n_seen = 0;
+        bool lead_piece = false, trail_piece = false;    // pieces of shared slots this unit has stored
+        int n_mem = 0, n_seen = 0, kept_entry = 0;
         uint4 raw_c = make_uint4(0u, 0u, 0u, 0u);
         float acc[8];
 #pragma unroll
@@ -417,29 +419,27 @@ merge_kernel(const __nv_bfloat16* __restrict__ k, const __nv_bfloat16* __restric
             else row = (long long)h * B + c;
             *reinterpret_cast<uint4*>(dst_base + row * kHeadDim + l16 * 8) = result;
         };
-        // a piece of a slot that other units share: publish it, and finish the row if it is the last
-        auto publish_piece = [&]() {
+        // ends the running piece: a whole slot is written out; a piece of a slot that other units
+        // share goes to this unit's record (announced after the loop)
+        auto flush = [&]() {
+            if (!active) return;
+            if (have_kept && n_seen == n_mem) {
+                write_row(slot, raw_c, acc, n_mem);
+                return;
+            }
             float* rec = parts + g * kPartFloats + (have_kept ? 256 : 0) + lane * 8;
             *reinterpret_cast<float4*>(rec) = make_float4(acc[0], acc[1], acc[2], acc[3]);
             *reinterpret_cast<float4*>(rec + 4) = make_float4(acc[4], acc[5], acc[6], acc[7]);
-            if (have_kept) *reinterpret_cast<uint4*>(parts + g * kPartFloats + 512 + lane * 4) = raw_c;
-            __threadfence();
-            __syncwarp();
-            int a = 0, b = 0, old = 0;
-            if (lane == 0) {
-                a = rp[slot];
-                b = rp[slot + 1];
-                old = atomicAdd(cnt + slot, 1);
+            if (have_kept) {
+                *reinterpret_cast<uint4*>(parts + g * kPartFloats + 512 + lane * 4) = raw_c;
+                trail_piece = true;
+            } else {
+                lead_piece = true;
             }
-            a = __shfl_sync(0xffffffffu, a, 0);
-            b = __shfl_sync(0xffffffffu, b, 0);
-            old = __shfl_sync(0xffffffffu, old, 0);
-            const int u0 = (slot + a) / ue;              // unit of the kept row
-            const int u1 = (slot + b) / ue;              // unit of the last member
-            if (old != u1 - u0) return;                  // pieces still missing
-            __threadfence();
-            const long long g0 = (long long)rq.unit_begin + (long long)u0 * n_kv_heads + h;
-            const float* r0 = parts + g0 * kPartFloats;
+        };
+        // adds the pieces of slot c (kept row in unit u0, last member in unit u1) in unit order
+        auto combine = [&](int c, int u0, int u1, int n) {
+            const float* r0 = parts + ((long long)rq.unit_begin + (long long)u0 * n_kv_heads + h) * kPartFloats;
             float sum[8];
             {
                 const float4 lo = ld_cg_f4(r0 + 256 + lane * 8), hi = ld_cg_f4(r0 + 256 + lane * 8 + 4);
@@ -453,12 +453,7 @@ merge_kernel(const __nv_bfloat16* __restrict__ k, const __nv_bfloat16* __restric
                 sum[0] += lo.x; sum[1] += lo.y; sum[2] += lo.z; sum[3] += lo.w;
                 sum[4] += hi.x; sum[5] += hi.y; sum[6] += hi.z; sum[7] += hi.w;
             }
-            write_row(slot, kept_raw, sum, b - a);
-        };
-        auto flush = [&]() {
-            if (!active) return;
-            if (have_kept && n_seen == n_mem) write_row(slot, raw_c, acc, n_mem);
-            else publish_piece();
+            write_row(c, kept_raw, sum, n);
         };
 
         for (int kc = 0; kc < n_chunks; ++kc) {
@@ -487,6 +482,7 @@ merge_kernel(const __nv_bfloat16* __restrict__ k, const __nv_bfloat16* __restric
                     raw_c = x4;
                     n_mem = (int)w;
                     n_seen = 0;
+                    kept_entry = e_lo + kc * kChunk + q;
 #pragma unroll
                     for (int i = 0; i < 8; ++i) acc[i] = 0.f;
                 } else {
@@ -503,6 +499,24 @@ merge_kernel(const __nv_bfloat16* __restrict__ k, const __nv_bfloat16* __restric
         }
         flush();
         n_chunks_done += (uint32_t)n_chunks;
+        if (lead_piece || trail_piece) {
+            // announce the stored pieces (lane 0: the leading one, lane 1: the trailing one); the
+            // unit that arrives last at a slot finishes its row
+            __threadfence();
+            __syncwarp();
+            int c = 0, s0 = 0, n = 0;
+            bool mine = false;
+            if (lane == 0 && lead_piece) { c = first.x; s0 = first.y; n = first.z; mine = true; }
+            if (lane == 1 && trail_piece) { c = slot; s0 = kept_entry; n = n_mem; mine = true; }
+            const int u0 = s0 / ue, u1 = (s0 + n) / ue;          // units of the kept row / the last member
+            const bool last = mine && atomicAdd(cnt + c, 1) == u1 - u0;
+            const unsigned finish = __ballot_sync(0xffffffffu, last);
+            if (finish) __threadfence();
+            for (int which = 0; which < 2; ++which)
+                if (finish & (1u << which))
+                    combine(__shfl_sync(0xffffffffu, c, which), __shfl_sync(0xffffffffu, u0, which),
+                            __shfl_sync(0xffffffffu, u1, which), __shfl_sync(0xffffffffu, n, which));
+        }
     }
     (void)status;
 }
@@ -572,7 +586,7 @@ cudaError_t launch_gather_kept(const void* k, long long stride_tok, long long st
 cudaError_t launch_invert_assignment(const int* assign, const int* kept_idx, const int* evict_idx,
                                      const float* sim, const Req* reqs, int n_req, int n_kv_heads,
                                      long long T, int* row_ptr, int* ent_pos, float* ent_w,
-                                     int* unit_first, int* slot_cnt, unsigned* sort_a,
+                                     int4* unit_first, int* slot_cnt, unsigned* sort_a,
                                      unsigned* sort_b, int* status, cudaStream_t stream) {
     dim3 grid(n_kv_heads, n_req);
     invert_assignment_kernel<<<grid, kInvThreads, 0, stream>>>(assign, kept_idx, evict_idx, sim, reqs,
@@ -587,7 +601,7 @@ int merge_warps_per_sm() { return kMergeWarps; }
 cudaError_t launch_merge(const void* k, const void* v, long long stride_tok, long long stride_head,
                          const Req* reqs, int n_req, int n_kv_heads, long long T,
                          long long total_units, const int* row_ptr, const int* ent_pos,
-                         const float* ent_w, const int* unit_first, int* slot_cnt, float* parts,
+                         const float* ent_w, const int4* unit_first, int* slot_cnt, float* parts,
                          int varlen_output, void* out_k, void* out_v, int* status, int num_sms,
                          cudaStream_t stream) {
     if (total_units <= 0) return cudaSuccess;
