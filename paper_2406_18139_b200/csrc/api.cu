@@ -162,6 +162,8 @@ int check_layout_ptrs(const lookm_layout* lay, const void* q, const void* k, con
     if (lay->q_stride_tok <= 0 || lay->q_stride_head <= 0 || lay->kv_stride_tok <= 0 ||
         lay->kv_stride_head <= 0)
         return LOOKM_ERR_INVALID_ARG;
+    // the merge kernel keeps the byte stride between tokens in 32 bits
+    if (lay->kv_stride_tok >= (1ll << 31)) return LOOKM_ERR_UNSUPPORTED;
     if (!(lay->softmax_scale >= 0.f) || !std::isfinite(lay->softmax_scale)) return LOOKM_ERR_INVALID_ARG;
     return LOOKM_OK;
 }

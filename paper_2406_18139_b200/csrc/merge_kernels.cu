@@ -338,6 +338,7 @@ merge_kernel(const __nv_bfloat16* __restrict__ k, const __nv_bfloat16* __restric
     const uint32_t buf0 = (uint32_t)__cvta_generic_to_shared(&sh.rows[warp][0][0][0]) + lane * 16;
     const __nv_bfloat16* tensor = lane < 16 ? k : v;
     __nv_bfloat16* dst_base = lane < 16 ? out_k : out_v;
+    const unsigned tok_bytes = (unsigned)stride_tok * 2u;      // the launcher checks that this fits
     uint32_t n_chunks_done = 0;                      // chunks this warp has consumed (buffer parity)
 
     for (long long g = (long long)blockIdx.x * kMergeWarps + warp; g < total_units;
@@ -354,7 +355,8 @@ merge_kernel(const __nv_bfloat16* __restrict__ k, const __nv_bfloat16* __restric
         int* cnt = slot_cnt + rq.kept_off + (long long)h * B;
         const int* ent = ent_pos + (long long)h * T + rq.tok_begin;
         const float* entw = ent_w + (long long)h * T + rq.tok_begin;
-        const __nv_bfloat16* src = tensor + (long long)rq.tok_begin * stride_tok + (long long)h * stride_head + l16 * 8;
+        const char* src = reinterpret_cast<const char*>(tensor + (long long)rq.tok_begin * stride_tok +
+                                                        (long long)h * stride_head + l16 * 8);
         const int n_chunks = (e_hi - e_lo + kChunk - 1) / kChunk;
 
         // entry metadata of a chunk (lanes 0-7: one entry each)
@@ -371,10 +373,10 @@ merge_kernel(const __nv_bfloat16* __restrict__ k, const __nv_bfloat16* __restric
             const uint32_t dst = buf0 + ((n_chunks_done + (uint32_t)kc) % kRing) * (kChunk * 2 * kRowBytes);
 #pragma unroll
             for (int q = 0; q < kChunk; ++q) {
-                const int tok = __shfl_sync(0xffffffffu, pos, q) & 0x7fffffff;
+                const unsigned tok = (unsigned)__shfl_sync(0xffffffffu, pos, q) & 0x7fffffffu;
                 if (q < n_ent)
                     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;"
-                                 ::"r"(dst + q * (2 * kRowBytes)), "l"(src + (long long)tok * stride_tok)
+                                 ::"r"(dst + q * (2 * kRowBytes)), "l"(src + (size_t)tok * tok_bytes)
                                  : "memory");
             }
             asm volatile("cp.async.commit_group;" ::: "memory");
@@ -465,31 +467,35 @@ merge_kernel(const __nv_bfloat16* __restrict__ k, const __nv_bfloat16* __restric
             float w_d;
             load_meta(kc + 3, pos_d, w_d);
             asm volatile("cp.async.wait_group 2;" ::: "memory");
-            const uint32_t b = (n_chunks_done + (uint32_t)kc) % kRing;
             const int n_ent = min(kChunk, e_hi - e_lo - kc * kChunk);
-            const uint8_t* base = &sh.rows[warp][b][0][0] + lane * 16;
+            const uint32_t rows = buf0 + ((n_chunks_done + (uint32_t)kc) % kRing) * (kChunk * 2 * kRowBytes);
+            uint4 x[kChunk];                         // this lane's 16 bytes of every staged row
+#pragma unroll
+            for (int q = 0; q < kChunk; ++q)
+                asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];"
+                             : "=r"(x[q].x), "=r"(x[q].y), "=r"(x[q].z), "=r"(x[q].w)
+                             : "r"(rows + q * (2 * kRowBytes)));
 #pragma unroll
             for (int q = 0; q < kChunk; ++q) {
                 const int pe = __shfl_sync(0xffffffffu, pos_a, q);
                 const float w = __shfl_sync(0xffffffffu, w_a, q);
                 if (q >= n_ent) break;
-                const uint4 x4 = *reinterpret_cast<const uint4*>(base + q * (2 * kRowBytes));
                 if (pe < 0) {                        // a kept row starts the next slot
                     flush();
                     ++slot;
                     active = true;
                     have_kept = true;
-                    raw_c = x4;
+                    raw_c = x[q];
                     n_mem = (int)w;
                     n_seen = 0;
                     kept_entry = e_lo + kc * kChunk + q;
 #pragma unroll
                     for (int i = 0; i < 8; ++i) acc[i] = 0.f;
                 } else {
-                    const Row8 x = unpack8(x4);
+                    const Row8 xe = unpack8(x[q]);
                     ++n_seen;
 #pragma unroll
-                    for (int i = 0; i < 8; ++i) acc[i] = fmaf(w, x.v[i], acc[i]);
+                    for (int i = 0; i < 8; ++i) acc[i] = fmaf(w, xe.v[i], acc[i]);
                 }
             }
             __syncwarp();
@@ -605,6 +611,7 @@ cudaError_t launch_merge(const void* k, const void* v, long long stride_tok, lon
                          int varlen_output, void* out_k, void* out_v, int* status, int num_sms,
                          cudaStream_t stream) {
     if (total_units <= 0) return cudaSuccess;
+    if (stride_tok <= 0 || stride_tok >= (1ll << 31)) return cudaErrorInvalidValue;   // byte stride kept in 32 bits
     const int smem = (int)sizeof(MergeShared) + 128;
     cudaError_t err = cudaFuncSetAttribute(merge_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (err != cudaSuccess) return err;
