@@ -48,7 +48,7 @@ struct __align__(1024) Shared {
     Req reqs[kReqCache];                         // copy of the request table (when it fits)
     unsigned long long a_full[2], a_empty[2];
     unsigned long long b_full[kStages], b_empty[kStages];
-    unsigned long long t_full[kAccum][2], t_empty[kAccum][2];   // per 64-column half of an accumulator
+    unsigned long long t_full[kAccum], t_empty[kAccum];
     unsigned long long mma_done;                 // every MMA of this CTA has completed
     uint32_t tmem_base;
     int abort_flag;
@@ -119,9 +119,9 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
             ptx::mbar_init(ptx::smem_u32(&sh.b_full[i]), 1);
             ptx::mbar_init(ptx::smem_u32(&sh.b_empty[i]), 1);
         }
-        for (int i = 0; i < kAccum * 2; ++i) {
-            ptx::mbar_init(ptx::smem_u32(&sh.t_full[0][0] + i), 1);
-            ptx::mbar_init(ptx::smem_u32(&sh.t_empty[0][0] + i), 4);   // one arrival per epilogue warp
+        for (int i = 0; i < kAccum; ++i) {
+            ptx::mbar_init(ptx::smem_u32(&sh.t_full[i]), 1);
+            ptx::mbar_init(ptx::smem_u32(&sh.t_empty[i]), 4);   // one arrival per epilogue warp
         }
         ptx::mbar_init(ptx::smem_u32(&sh.mma_done), 1);
         sh.abort_flag = 0;
@@ -200,38 +200,7 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issuer ------------
         if (lane == 0) {
-            // A tile is issued as two 128 x 64 halves, each into its own half of the group's
-            // accumulator and with its own full/empty barriers, and the second half of tile g is
-            // issued after the first half of tile g + 1.  The epilogue group therefore hands back
-            // the first half while it still works on the second, and the refill of either half is
-            // done long before the group returns to it.
-            constexpr uint32_t idesc = ptx::umma_idesc_bf16(kTile, kTile / 2);
-            auto issue_half = [&](uint32_t a_addr, uint32_t b_addr, int buf, int half, uint32_t g) {
-                ptx::mbar_wait(ptx::smem_u32(&sh.t_empty[buf][half]), ((g / kAccum) & 1) ^ 1, abort_flag);
-                ptx::tc_fence_after_sync();
-                const uint32_t d_tmem = tmem_base + buf * kTile + half * (kTile / 2);
-                const uint32_t b_half = b_addr + half * (kTile / 2) * 128;      // 64 rows of 128 bytes
-#pragma unroll
-                for (int kk = 0; kk < 8; ++kk) {
-                    // 16 bf16 (32 bytes) per MMA along the 128-byte swizzled row; the second
-                    // half of head_dim lives in the second TMA box.
-                    const uint32_t off = (kk >> 2) * kHalfBytes + (kk & 3) * 32;
-                    ptx::umma_bf16(d_tmem, ptx::umma_desc_sw128(a_addr + off),
-                                   ptx::umma_desc_sw128(b_half + off), idesc, kk > 0);
-                }
-                ptx::umma_commit(ptx::smem_u32(&sh.t_full[buf][half]));
-            };
-            // second half still owed for the previous tile
-            bool owed = false;
-            uint32_t owed_a = 0, owed_b = 0, owed_g = 0;
-            int owed_stage = 0, owed_a_release = -1;
-            auto issue_owed = [&]() {
-                if (!owed) return;
-                issue_half(owed_a, owed_b, owed_g % kAccum, 1, owed_g);
-                ptx::umma_commit(ptx::smem_u32(&sh.b_empty[owed_stage]));
-                if (owed_a_release >= 0) ptx::umma_commit(ptx::smem_u32(&sh.a_empty[owed_a_release]));
-                owed = false;
-            };
+            constexpr uint32_t idesc = ptx::umma_idesc_bf16(kTile, kTile);
             uint32_t gb = 0;
             int n = 0;
             for (int round = 0;; ++round, ++n) {
@@ -243,19 +212,25 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                 const uint32_t a_addr = ptx::smem_u32(&sh.a[ab][0]);
                 for (int t = 0; t < it.nt; ++t, ++gb) {
                     const int s = gb % kStages;
+                    const int buf = gb % kAccum;
                     ptx::mbar_wait(ptx::smem_u32(&sh.b_full[s]), (gb / kStages) & 1, abort_flag);
+                    ptx::mbar_wait(ptx::smem_u32(&sh.t_empty[buf]), ((gb / kAccum) & 1) ^ 1, abort_flag);
+                    ptx::tc_fence_after_sync();
                     const uint32_t b_addr = ptx::smem_u32(&sh.b[s][0]);
-                    issue_half(a_addr, b_addr, gb % kAccum, 0, gb);
-                    issue_owed();
-                    owed = true;
-                    owed_a = a_addr;
-                    owed_b = b_addr;
-                    owed_g = gb;
-                    owed_stage = s;
-                    owed_a_release = (t == it.nt - 1) ? ab : -1;
+                    const uint32_t d_tmem = tmem_base + buf * kTile;
+#pragma unroll
+                    for (int kk = 0; kk < 8; ++kk) {
+                        // 16 bf16 (32 bytes) per MMA along the 128-byte swizzled row; the second
+                        // half of head_dim lives in the second TMA box.
+                        const uint32_t off = (kk >> 2) * kHalfBytes + (kk & 3) * 32;
+                        ptx::umma_bf16(d_tmem, ptx::umma_desc_sw128(a_addr + off),
+                                       ptx::umma_desc_sw128(b_addr + off), idesc, kk > 0);
+                    }
+                    ptx::umma_commit(ptx::smem_u32(&sh.b_empty[s]));
+                    ptx::umma_commit(ptx::smem_u32(&sh.t_full[buf]));
+                    if (t == it.nt - 1) ptx::umma_commit(ptx::smem_u32(&sh.a_empty[ab]));
                 }
             }
-            issue_owed();
             // Nothing may release TMEM or leave the kernel while an MMA is still running, also
             // after an abort: wait for all of them (own time limit, the abort flag is ignored).
             int ignore = 0;
@@ -306,15 +281,20 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                     ptx::named_barrier_sync(1 + wg, 128);
                 }
                 ++lt;
+                ptx::mbar_wait(ptx::smem_u32(&sh.t_full[buf]), (gb / kAccum) & 1, abort_flag);
+                ptx::tc_fence_after_sync();
 #pragma unroll 1
                 for (int ch = 0; ch < 4; ++ch) {
-                    if ((ch & 1) == 0) {                     // columns of the next accumulator half
-                        ptx::mbar_wait(ptx::smem_u32(&sh.t_full[buf][ch >> 1]), (gb / kAccum) & 1, abort_flag);
-                        ptx::tc_fence_after_sync();
-                    }
                     uint32_t raw[32];
                     ptx::tmem_ld_32x32(lane_addr + buf * kTile + ch * 32, raw);
                     ptx::tmem_ld_wait();
+                    if (ch == 3) {
+                        // the last columns are in registers: hand the accumulator back now, so
+                        // that the next tile's MMAs run while this chunk is still being worked on
+                        ptx::tc_fence_before_sync();
+                        __syncwarp();
+                        if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&sh.t_empty[buf]));
+                    }
                     const int c0 = ch * 32;
                     if (KIND == kSweep1) {
                         // online softmax statistics of row `pos` over key columns c0..c0+31
@@ -412,11 +392,6 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                                 best_slot = slot0 + g16 * 16 + idx;
                             }
                         }
-                    }
-                    if (ch & 1) {                            // this half may be overwritten
-                        ptx::tc_fence_before_sync();
-                        __syncwarp();
-                        if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&sh.t_empty[buf][ch >> 1]));
                     }
                 }
             }
