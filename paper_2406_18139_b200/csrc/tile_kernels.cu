@@ -33,7 +33,9 @@ namespace {
 constexpr int kStages = 4;                       // ring of streamed tiles
 constexpr int kAccum = 4;                        // TMEM accumulators (128 fp32 columns each)
 constexpr int kGroups = 4;                       // epilogue groups (one per TMEM accumulator)
-constexpr int kThreads = 64 + kGroups * 128;     // producer warp, MMA warp, 4 x 4 epilogue warps
+constexpr int kIssuers = 2;                      // MMA-issuing threads (tiles alternate between them)
+constexpr int kEpiWarp0 = 2;                     // first epilogue warp
+constexpr int kThreads = 64 + kGroups * 128 + 32;   // producer warp, MMA warp, 4 x 4 epilogue warps, second MMA warp
 constexpr int kHalfBytes = kTile * 64 * 2;       // one TMA box: 128 rows x 64 bf16 (128 B rows)
 constexpr int kTileBytes = 2 * kHalfBytes;       // 128 x 128 bf16
 constexpr int kReqCache = 32;                    // request-table entries cached in shared memory
@@ -113,7 +115,7 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     if (threadIdx.x == 0) {
         for (int i = 0; i < 2; ++i) {
             ptx::mbar_init(ptx::smem_u32(&sh.a_full[i]), 1);
-            ptx::mbar_init(ptx::smem_u32(&sh.a_empty[i]), 1);
+            ptx::mbar_init(ptx::smem_u32(&sh.a_empty[i]), kIssuers);
         }
         for (int i = 0; i < kStages; ++i) {
             ptx::mbar_init(ptx::smem_u32(&sh.b_full[i]), 1);
@@ -123,7 +125,7 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
             ptx::mbar_init(ptx::smem_u32(&sh.t_full[i]), 1);
             ptx::mbar_init(ptx::smem_u32(&sh.t_empty[i]), 4);   // one arrival per epilogue warp
         }
-        ptx::mbar_init(ptx::smem_u32(&sh.mma_done), 1);
+        ptx::mbar_init(ptx::smem_u32(&sh.mma_done), kIssuers);
         sh.abort_flag = 0;
         ptx::fence_mbar_init();
     }
@@ -197,9 +199,14 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                                    200000000ull);
             }
         }
-    } else if (warp == 1) {
-        // ------------------------------------------------------------ MMA issuer ------------
+    } else if (warp == 1 || warp == kEpiWarp0 + kGroups * 4) {
+        // ------------------------------------------------------------ MMA issuers -----------
+        // One thread spends about as long on the waits, fences, commits and loop bookkeeping of a
+        // tile as the tensor core needs for its eight MMAs, and it is blocked while they are
+        // queued.  Two threads (in warps of different SM sub-partitions) therefore take the tiles
+        // alternately: one prepares its next tile while the other one's MMAs run.
         if (lane == 0) {
+            const uint32_t me = (warp == 1) ? 0u : 1u;
             constexpr uint32_t idesc = ptx::umma_idesc_bf16(kTile, kTile);
             uint32_t gb = 0;
             int n = 0;
@@ -210,7 +217,9 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                 const int ab = n & 1;
                 ptx::mbar_wait(ptx::smem_u32(&sh.a_full[ab]), (n >> 1) & 1, abort_flag);
                 const uint32_t a_addr = ptx::smem_u32(&sh.a[ab][0]);
+                bool issued = false;
                 for (int t = 0; t < it.nt; ++t, ++gb) {
+                    if ((gb & (kIssuers - 1)) != me) continue;
                     const int s = gb % kStages;
                     const int buf = gb % kAccum;
                     ptx::mbar_wait(ptx::smem_u32(&sh.b_full[s]), (gb / kStages) & 1, abort_flag);
@@ -228,8 +237,12 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                     }
                     ptx::umma_commit(ptx::smem_u32(&sh.b_empty[s]));
                     ptx::umma_commit(ptx::smem_u32(&sh.t_full[buf]));
-                    if (t == it.nt - 1) ptx::umma_commit(ptx::smem_u32(&sh.a_empty[ab]));
+                    issued = true;
                 }
+                // the stationary tile is free when both issuers are through with the item: an
+                // issuer that used it arrives when its MMAs have completed, the other one at once
+                if (issued) ptx::umma_commit(ptx::smem_u32(&sh.a_empty[ab]));
+                else ptx::mbar_arrive(ptx::smem_u32(&sh.a_empty[ab]));
             }
             // Nothing may release TMEM or leave the kernel while an MMA is still running, also
             // after an abort: wait for all of them (own time limit, the abort flag is ignored).
@@ -239,7 +252,7 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         }
     } else {
         // ------------------------------------------------------------ epilogue --------------
-        const int wg = (warp - 2) >> 2;                      // epilogue group 0..3
+        const int wg = (warp - kEpiWarp0) >> 2;              // epilogue group 0..3
         const int quarter = warp & 3;                        // TMEM lane quarter this warp may read
         const int row = quarter * 32 + lane;                 // row of the stationary tile
         const uint32_t lane_addr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
