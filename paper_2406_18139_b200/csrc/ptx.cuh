@@ -162,6 +162,23 @@ __device__ __forceinline__ float ex2(float x) {
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
+// 2^x on the FMA and integer pipes instead of the special-function unit (which is the busiest
+// unit of the softmax epilogues): x = n + f with n the nearest integer (taken from the low mantissa
+// bits after adding 1.5 * 2^23) and f in [-1/2, 1/2], 2^f by a degree-5 minimax polynomial
+// (relative error 2.4e-7 in fp32), n added to the exponent field.  Arguments below -125 give
+// 2^-125 (about 2.4e-38) instead of a denormal or zero; NaN is not handled.
+__device__ __forceinline__ float ex2_fma(float x) {
+    x = fmaxf(x, -125.f);
+    const float r = x + 12582912.f;
+    const float f = x - (r - 12582912.f);
+    float p = 1.327647245e-03f;
+    p = fmaf(p, f, 9.675540961e-03f);
+    p = fmaf(p, f, 5.550713092e-02f);
+    p = fmaf(p, f, 2.402212024e-01f);
+    p = fmaf(p, f, 6.931469440e-01f);
+    p = fmaf(p, f, 1.000000119e+00f);
+    return __int_as_float(__float_as_int(p) + (__float_as_int(r) << 23));
+}
 __device__ __forceinline__ float lg2(float x) {
     float y;
     asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));

@@ -56,6 +56,13 @@ struct __align__(1024) Shared {
     int abort_flag;
 };
 
+// The softmax epilogues are bound by the special-function unit (16 ex2 per clock and SM), so one
+// column in kPolyEvery is exponentiated on the FMA pipe instead.
+constexpr int kPolyEvery = 4;
+__device__ __forceinline__ float exp2_mixed(int column, float x) {
+    return (column % kPolyEvery == kPolyEvery - 1) ? ptx::ex2_fma(x) : ptx::ex2(x);
+}
+
 struct Item {
     int tok_begin, L, B, blk, head, nt;
     long long kept_row0;      // match: first row of this (request, head) in the kept-key matrix
@@ -327,7 +334,7 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
 #pragma unroll
                                 for (int c = 0; c < 32; c += 2) {
                                     const float e0 = ptx::ex2(fmaf(__uint_as_float(raw[c]), c2, -mc));
-                                    const float e1 = ptx::ex2(fmaf(__uint_as_float(raw[c + 1]), c2, -mc));
+                                    const float e1 = exp2_mixed(c + 1, fmaf(__uint_as_float(raw[c + 1]), c2, -mc));
                                     s0 += (c0 + c <= row) ? e0 : 0.f;
                                     s1 += (c0 + c + 1 <= row) ? e1 : 0.f;
                                 }
@@ -335,7 +342,7 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
 #pragma unroll
                                 for (int c = 0; c < 32; c += 2) {
                                     s0 += ptx::ex2(fmaf(__uint_as_float(raw[c]), c2, -mc));
-                                    s1 += ptx::ex2(fmaf(__uint_as_float(raw[c + 1]), c2, -mc));
+                                    s1 += exp2_mixed(c + 1, fmaf(__uint_as_float(raw[c + 1]), c2, -mc));
                                 }
                             }
                             l_run = l_run * ptx::ex2(m_run * c2 - mc) + (s0 + s1);
@@ -352,7 +359,7 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                                 const float e0 = ptx::ex2(fmaf(__uint_as_float(raw[c4 * 4 + 0]), c2, -l4.x));
                                 const float e1 = ptx::ex2(fmaf(__uint_as_float(raw[c4 * 4 + 1]), c2, -l4.y));
                                 const float e2 = ptx::ex2(fmaf(__uint_as_float(raw[c4 * 4 + 2]), c2, -l4.z));
-                                const float e3 = ptx::ex2(fmaf(__uint_as_float(raw[c4 * 4 + 3]), c2, -l4.w));
+                                const float e3 = exp2_mixed(c4 * 4 + 3, fmaf(__uint_as_float(raw[c4 * 4 + 3]), c2, -l4.w));
                                 acc0 += (c + 0 >= row) ? e0 : 0.f;
                                 acc1 += (c + 1 >= row) ? e1 : 0.f;
                                 acc2 += (c + 2 >= row) ? e2 : 0.f;
@@ -365,7 +372,7 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                                 acc0 += ptx::ex2(fmaf(__uint_as_float(raw[c4 * 4 + 0]), c2, -l4.x));
                                 acc1 += ptx::ex2(fmaf(__uint_as_float(raw[c4 * 4 + 1]), c2, -l4.y));
                                 acc2 += ptx::ex2(fmaf(__uint_as_float(raw[c4 * 4 + 2]), c2, -l4.z));
-                                acc3 += ptx::ex2(fmaf(__uint_as_float(raw[c4 * 4 + 3]), c2, -l4.w));
+                                acc3 += exp2_mixed(c4 * 4 + 3, fmaf(__uint_as_float(raw[c4 * 4 + 3]), c2, -l4.w));
                             }
                         }
                     } else {
