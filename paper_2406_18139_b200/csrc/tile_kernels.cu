@@ -58,7 +58,7 @@ struct __align__(1024) Shared {
 
 // The softmax epilogues are bound by the special-function unit (16 ex2 per clock and SM), so one
 // column in kPolyEvery is exponentiated on the FMA pipe instead.
-constexpr int kPolyEvery = 4;
+constexpr int kPolyEvery = 5;
 __device__ __forceinline__ float exp2_mixed(int column, float x) {
     return (column % kPolyEvery == kPolyEvery - 1) ? ptx::ex2_fma(x) : ptx::ex2(x);
 }
@@ -333,7 +333,7 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                             if (diag) {
 #pragma unroll
                                 for (int c = 0; c < 32; c += 2) {
-                                    const float e0 = ptx::ex2(fmaf(__uint_as_float(raw[c]), c2, -mc));
+                                    const float e0 = exp2_mixed(c, fmaf(__uint_as_float(raw[c]), c2, -mc));
                                     const float e1 = exp2_mixed(c + 1, fmaf(__uint_as_float(raw[c + 1]), c2, -mc));
                                     s0 += (c0 + c <= row) ? e0 : 0.f;
                                     s1 += (c0 + c + 1 <= row) ? e1 : 0.f;
@@ -341,7 +341,7 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                             } else {
 #pragma unroll
                                 for (int c = 0; c < 32; c += 2) {
-                                    s0 += ptx::ex2(fmaf(__uint_as_float(raw[c]), c2, -mc));
+                                    s0 += exp2_mixed(c, fmaf(__uint_as_float(raw[c]), c2, -mc));
                                     s1 += exp2_mixed(c + 1, fmaf(__uint_as_float(raw[c + 1]), c2, -mc));
                                 }
                             }
@@ -356,9 +356,9 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                             for (int c4 = 0; c4 < 8; ++c4) {
                                 const float4 l4 = sd[c4];
                                 const int c = c0 + c4 * 4;
-                                const float e0 = ptx::ex2(fmaf(__uint_as_float(raw[c4 * 4 + 0]), c2, -l4.x));
-                                const float e1 = ptx::ex2(fmaf(__uint_as_float(raw[c4 * 4 + 1]), c2, -l4.y));
-                                const float e2 = ptx::ex2(fmaf(__uint_as_float(raw[c4 * 4 + 2]), c2, -l4.z));
+                                const float e0 = exp2_mixed(c4 * 4 + 0, fmaf(__uint_as_float(raw[c4 * 4 + 0]), c2, -l4.x));
+                                const float e1 = exp2_mixed(c4 * 4 + 1, fmaf(__uint_as_float(raw[c4 * 4 + 1]), c2, -l4.y));
+                                const float e2 = exp2_mixed(c4 * 4 + 2, fmaf(__uint_as_float(raw[c4 * 4 + 2]), c2, -l4.z));
                                 const float e3 = exp2_mixed(c4 * 4 + 3, fmaf(__uint_as_float(raw[c4 * 4 + 3]), c2, -l4.w));
                                 acc0 += (c + 0 >= row) ? e0 : 0.f;
                                 acc1 += (c + 1 >= row) ? e1 : 0.f;
@@ -369,9 +369,9 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
 #pragma unroll
                             for (int c4 = 0; c4 < 8; ++c4) {
                                 const float4 l4 = sd[c4];
-                                acc0 += ptx::ex2(fmaf(__uint_as_float(raw[c4 * 4 + 0]), c2, -l4.x));
-                                acc1 += ptx::ex2(fmaf(__uint_as_float(raw[c4 * 4 + 1]), c2, -l4.y));
-                                acc2 += ptx::ex2(fmaf(__uint_as_float(raw[c4 * 4 + 2]), c2, -l4.z));
+                                acc0 += exp2_mixed(c4 * 4 + 0, fmaf(__uint_as_float(raw[c4 * 4 + 0]), c2, -l4.x));
+                                acc1 += exp2_mixed(c4 * 4 + 1, fmaf(__uint_as_float(raw[c4 * 4 + 1]), c2, -l4.y));
+                                acc2 += exp2_mixed(c4 * 4 + 2, fmaf(__uint_as_float(raw[c4 * 4 + 2]), c2, -l4.z));
                                 acc3 += exp2_mixed(c4 * 4 + 3, fmaf(__uint_as_float(raw[c4 * 4 + 3]), c2, -l4.w));
                             }
                         }
