@@ -4,13 +4,14 @@
 // All three are the same persistent, warp-specialised pipeline over 128 x 128 x 128 bf16 tiles:
 //   - a work item owns one STATIONARY 128-row tile (the A operand, rows on the 128 TMEM lanes)
 //     and streams a sequence of 128-row tiles (the B operand) against it;
-//   - warp 0 (one thread) issues the TMA loads, warp 1 (one thread) issues tcgen05.mma into one of
-//     four 128-column TMEM accumulators, and four groups of four warps read the accumulators with
-//     tcgen05.ld and run the epilogue; group w owns accumulator w and takes the tiles whose running
-//     index is w mod 4, so each SM sub-partition always has four epilogue warps to switch between;
+//   - warp 0 (one thread) issues the TMA loads, warps 1 and 18 (one thread each, tiles taken
+//     alternately) issue tcgen05.mma into one of four 128-column TMEM accumulators, and four
+//     groups of four warps read the accumulators with tcgen05.ld and run the epilogue; group w
+//     owns accumulator w and takes the tiles whose running index is w mod 4, so each SM
+//     sub-partition always has four epilogue warps to switch between;
 //   - each epilogue thread owns one row of the stationary tile, so every reduction over the
 //     streamed axis (row maximum and sum, column-sum of probabilities for one key, running
-//     arg-max) stays in that thread's registers; the two groups are combined through shared
+//     arg-max) stays in that thread's registers; the four groups are combined through shared
 //     memory once per item.  No L x L matrix is ever stored.
 //
 //   sweep 1: A = 128 queries of one query head, B = key tiles 0..diagonal.  Online softmax
