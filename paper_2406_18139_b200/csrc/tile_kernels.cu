@@ -326,7 +326,8 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                                 if (c0 + c <= row) mx = fmaxf(mx, __uint_as_float(raw[c]));
                         } else {
 #pragma unroll
-                            for (int c = 0; c < 32; ++c) mx = fmaxf(mx, __uint_as_float(raw[c]));
+                            for (int c = 0; c < 32; c += 2)
+                                mx = ptx::fmax3(mx, __uint_as_float(raw[c]), __uint_as_float(raw[c + 1]));
                         }
                         if (mx != -INFINITY) {               // false only above the diagonal
                             const float mc = mx * c2;
@@ -400,11 +401,12 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                                 for (int c = 0; c < 16; ++c)
                                     if (c0 + g16 * 16 + c >= col_limit) v[c] = -INFINITY;
                             }
-                            const float m0 = fmaxf(fmaxf(v[0], v[1]), fmaxf(v[2], v[3]));
-                            const float m1 = fmaxf(fmaxf(v[4], v[5]), fmaxf(v[6], v[7]));
-                            const float m2 = fmaxf(fmaxf(v[8], v[9]), fmaxf(v[10], v[11]));
-                            const float m3 = fmaxf(fmaxf(v[12], v[13]), fmaxf(v[14], v[15]));
-                            const float mx = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
+                            const float m0 = ptx::fmax3(v[0], v[1], v[2]);
+                            const float m1 = ptx::fmax3(v[3], v[4], v[5]);
+                            const float m2 = ptx::fmax3(v[6], v[7], v[8]);
+                            const float m3 = ptx::fmax3(v[9], v[10], v[11]);
+                            const float m4 = ptx::fmax3(v[12], v[13], v[14]);
+                            const float mx = fmaxf(ptx::fmax3(m0, m1, m2), ptx::fmax3(m3, m4, v[15]));
                             if (mx > best) {
                                 best = mx;
                                 int idx = 15;
