@@ -278,22 +278,6 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
             float best = -INFINITY;                          // match
             int best_slot = 0x7fffffff;
 
-            // per-column data of a streamed tile (one value per thread): sweep 2 needs the
-            // log-sum-exp of the tile's queries, the match the inverse norms of its kept keys
-            auto column_value = [&](int t) -> float {
-                if (KIND == kSweep2) {
-                    const int qh = it.head * p.group + t % p.group;
-                    const int i = (it.blk + t / p.group) * kTile + row;   // query column staged by this thread
-                    // +inf turns the probability into 0
-                    return (i < it.L) ? p.lse[(long long)qh * p.T + it.tok_begin + i] * kLog2e : INFINITY;
-                } else {
-                    const int slot = t * kTile + row;
-                    return (slot < it.B) ? p.rnorm_kept[it.kept_row0 + slot] : 0.f;
-                }
-            };
-            float col_next = 0.f;                            // value for this group's next tile,
-            bool have_next = false;                          // loaded one tile ahead
-
             for (int t = 0; t < it.nt; ++t, ++gb) {
                 if ((int)(gb % kGroups) != wg) continue;
                 const int buf = wg;
@@ -302,13 +286,19 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                 int col_limit = kTile;                       // match: valid kept slots in the tile
                 if (KIND == kSweep1) {
                     diag = (t == it.blk);
-                } else {
-                    const float v = have_next ? col_next : column_value(t);
-                    have_next = (t + kGroups < it.nt);       // this group's next tile of the item
-                    if (have_next) col_next = column_value(t + kGroups);
+                } else if (KIND == kSweep2) {
+                    const int ib = it.blk + t / p.group;
+                    const int qh = it.head * p.group + t % p.group;
+                    const int i = ib * kTile + row;          // query column staged by this thread
+                    float v = INFINITY;                      // +inf turns the probability into 0
+                    if (i < it.L) v = p.lse[(long long)qh * p.T + it.tok_begin + i] * kLog2e;
                     side[row] = v;
-                    if (KIND == kSweep2) diag = (t / p.group == 0);
-                    else col_limit = min(kTile, it.B - t * kTile);
+                    diag = (ib == it.blk);
+                    ptx::named_barrier_sync(1 + wg, 128);
+                } else {
+                    const int slot = t * kTile + row;
+                    side[row] = (slot < it.B) ? p.rnorm_kept[it.kept_row0 + slot] : 0.f;
+                    col_limit = min(kTile, it.B - t * kTile);
                     ptx::named_barrier_sync(1 + wg, 128);
                 }
                 ++lt;
