@@ -191,8 +191,8 @@ int lookm_noalloc_status(void* cuda_stream);
 /* Optional per-stage timing.  While set (per host thread), every whole-path call records the
  * caller's events (cudaEvent_t handles in a host array that must stay alive) on its stream at the
  * step boundaries: [0] start, [1] after the first score sweep, [2] after the second (Eq. 4),
- * [3] after the selection (Eq. 5-8), [4] after key norms and kept-key compaction, [5] after the
- * matching (Eq. 9), [6] after the assignment inversion, [7] after merge + compaction (Eq. 10-12).
+ * [3] after the selection (Eq. 5-8; the same launch computes the key norms of Eq. 9), [4] after
+ * the kept-key compaction, [5] after the matching (Eq. 9), [6] after the assignment inversion, [7] after merge + compaction (Eq. 10-12).
  * n_events must be LOOKM_N_STAGE_EVENTS; pass NULL, 0 to stop.  Nothing is recorded otherwise. */
 #define LOOKM_N_STAGE_EVENTS 8
 int lookm_set_stage_events(void* const* events_host, int n_events);

@@ -24,7 +24,7 @@ EXPORTS = ["lookm_workspace_size", "lookm_workspace_layout", "lookm_compress_lay
            "lookm_select", "lookm_match", "lookm_match_from_sim", "lookm_merge",
            "lookm_set_stage_events", "lookm_merge_noalloc", "lookm_noalloc_status", "lookm_device_status", "lookm_last_launch_count", "lookm_strerror"]
 N_STAGE_EVENTS = 8
-STAGE_NAMES = ["score_sweep1", "score_sweep2", "select", "norms_gather", "match", "invert", "merge"]
+STAGE_NAMES = ["score_sweep1", "score_sweep2", "select_norms", "gather", "match", "invert", "merge"]
 
 
 class WorkspaceOffsets(C.Structure):

@@ -300,17 +300,20 @@ int run_score(const Plan& pl, const DeviceInfo& di, const lookm_layout* lay, con
     return LOOKM_OK;
 }
 
+// norms_done: 1 / |k| of every key row is already in the workspace (written by the selection launch)
 int run_match(const Plan& pl, const DeviceInfo& di, const lookm_layout* lay, const void* k,
               const int* kept_idx, const int* rank, int* assign, float* sim, void* ws,
-              cudaStream_t st) {
+              bool norms_done, cudaStream_t st) {
     if (pl.n_items[kMatch] == 0) { mark_stage(4, st); mark_stage(5, st); return LOOKM_OK; }
     float* rnorm_all = at<float>(ws, pl.o_rnorm_all);
     float* rnorm_kept = at<float>(ws, pl.o_rnorm_kept);
     void* kept_keys = at<void>(ws, pl.o_kept_keys);
     const Req* reqs = at<Req>(ws, pl.o_reqs);
-    LOOKM_CUDA(launch_key_norms(k, lay->kv_stride_tok, lay->kv_stride_head, pl.n_kv_heads, pl.T,
-                                rnorm_all, st));
-    ++g_launches;
+    if (!norms_done) {
+        LOOKM_CUDA(launch_key_norms(k, lay->kv_stride_tok, lay->kv_stride_head, pl.n_kv_heads, pl.T,
+                                    rnorm_all, st));
+        ++g_launches;
+    }
     LOOKM_CUDA(launch_gather_kept(k, lay->kv_stride_tok, lay->kv_stride_head, reqs, pl.n_req,
                                   pl.n_kv_heads, pl.T, pl.total_slots, kept_idx, rnorm_all,
                                   kept_keys, rnorm_kept, at<int>(ws, pl.o_status), st));
@@ -382,11 +385,13 @@ int compress_common(const void* q, const void* k, const void* v, const uint8_t* 
     int* assign = at<int>(ws, pl.o_assign);
     float* sim = at<float>(ws, pl.o_sim);
     LOOKM_TRY(run_score(pl, di, lay, q, k, scores, at<float>(ws, pl.o_lse), false, ws, st));
+    // the selection launch also computes the key norms that the matching needs
     LOOKM_CUDA(launch_select(scores, mask, at<Req>(ws, pl.o_reqs), pl.n_req, pl.n_kv_heads, pl.T,
-                             kept, evict, rank, st));
+                             kept, evict, rank, k, lay->kv_stride_tok, lay->kv_stride_head,
+                             at<float>(ws, pl.o_rnorm_all), di.sms, st));
     ++g_launches;
     mark_stage(3, st);
-    LOOKM_TRY(run_match(pl, di, lay, k, kept, rank, assign, sim, ws, st));
+    LOOKM_TRY(run_match(pl, di, lay, k, kept, rank, assign, sim, ws, true, st));
     LOOKM_TRY(run_merge(pl, lay, k, v, kept, evict, assign, sim, varlen_output, out_k, out_v, ws, st));
     return LOOKM_OK;
 }
@@ -482,7 +487,7 @@ int lookm_select(const float* scores, const uint8_t* modality_mask, const int* c
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     LOOKM_TRY(begin_call(pl, workspace, st));
     LOOKM_CUDA(launch_select(scores, modality_mask, at<Req>(workspace, pl.o_reqs), pl.n_req,
-                             pl.n_kv_heads, pl.T, kept_idx, evict_idx, rank, st));
+                             pl.n_kv_heads, pl.T, kept_idx, evict_idx, rank, nullptr, 0, 0, nullptr, 0, st));
     ++g_launches;
     return LOOKM_OK;
 }
@@ -506,7 +511,7 @@ int lookm_match(const void* k, const int* kept_idx, const int* evict_idx, const 
                                       pl.max_L, kept_idx, evict_idx, rank,
                                       at<int>(workspace, pl.o_status), st));
     ++g_launches;
-    return run_match(pl, di, layout, k, kept_idx, rank, assign, sim, workspace, st);
+    return run_match(pl, di, layout, k, kept_idx, rank, assign, sim, workspace, false, st);
 }
 
 int lookm_match_from_sim(const float* sim_matrix, const int* cu_seqlens_host, int n_requests,

@@ -63,7 +63,8 @@ cudaError_t launch_tile_kernel(int kind, const CUtensorMap& map_a, const CUtenso
 
 cudaError_t launch_select(const float* scores, const uint8_t* mask, const Req* reqs, int n_req,
                           int n_kv_heads, long long T, int* kept_idx, int* evict_idx, int* rank,
-                          cudaStream_t stream);
+                          const void* k_for_norms, long long stride_tok, long long stride_head,
+                          float* rnorm_all, int num_sms, cudaStream_t stream);
 
 cudaError_t launch_key_norms(const void* k, long long stride_tok, long long stride_head,
                              int n_kv_heads, long long T, float* rnorm_all, cudaStream_t stream);

@@ -8,6 +8,14 @@
 // Either way one class is kept wholesale or not at all and the other needs an exact top-k, done
 // by a 4-pass radix select on an order-preserving 32-bit key; ties at the threshold go to the
 // lowest positions.  A final ordered pass writes the kept and evicted lists in ascending position.
+//
+// The selection occupies only n_requests * n_kv_heads CTAs, so the same launch carries, in further
+// CTAs, work that does not depend on it and is needed next: 1 / |k| of every key row (the cosine
+// denominators of Eq. 9).
+#include <cuda_bf16.h>
+
+#include <algorithm>
+
 #include "internal.h"
 
 namespace lookm {
@@ -56,16 +64,52 @@ __device__ __forceinline__ void block_scan2(int a, int b, int& ea, int& eb, int&
     tb = warp_tot[31][1];
 }
 
+// 1 / |k| of every key row (0 for a zero row): half a warp per row, 16 bytes per lane.
+__device__ __forceinline__ void key_norms(const __nv_bfloat16* __restrict__ k, long long stride_tok,
+                                          long long stride_head, int n_kv_heads, long long T,
+                                          float* __restrict__ rnorm_all, int block, int n_blocks) {
+    constexpr int kRowsPerBlock = kSelThreads / 16;
+    const int half = threadIdx.x >> 4, l16 = threadIdx.x & 15;
+    const long long n_rows = T * n_kv_heads;
+    // the loop bound is the warp's first row, so that both half-warps always reach the shuffles
+    for (long long rw = (long long)block * kRowsPerBlock + (half & ~1); rw < n_rows;
+         rw += (long long)n_blocks * kRowsPerBlock) {
+        const long long r = rw + (half & 1);
+        const bool valid = r < n_rows;
+        const long long tok = valid ? r / n_kv_heads : 0;
+        const int h = valid ? (int)(r % n_kv_heads) : 0;
+        const uint4 u = *reinterpret_cast<const uint4*>(k + tok * stride_tok + h * stride_head + l16 * 8);
+        const unsigned w[4] = {u.x, u.y, u.z, u.w};
+        float ss = 0.f;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const float lo = __uint_as_float(w[i] << 16), hi = __uint_as_float(w[i] & 0xffff0000u);
+            ss = fmaf(lo, lo, ss);
+            ss = fmaf(hi, hi, ss);
+        }
+#pragma unroll
+        for (int o = 8; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o, 16);
+        if (l16 == 0 && valid) rnorm_all[(long long)h * T + tok] = ss > 0.f ? 1.0f / sqrtf(ss) : 0.f;
+    }
+}
+
 __global__ void __launch_bounds__(kSelThreads)
 select_kernel(const float* __restrict__ scores, const uint8_t* __restrict__ mask,
-              const Req* __restrict__ reqs, int n_kv_heads, long long T, int* __restrict__ kept_idx,
-              int* __restrict__ evict_idx, int* __restrict__ rank) {
+              const Req* __restrict__ reqs, int n_select_blocks, int n_kv_heads, long long T,
+              int* __restrict__ kept_idx, int* __restrict__ evict_idx, int* __restrict__ rank,
+              const __nv_bfloat16* __restrict__ k, long long stride_tok, long long stride_head,
+              float* __restrict__ rnorm_all) {
     __shared__ int hist[256];
     __shared__ int warp_tot[32][2];
     __shared__ int sh_val[4];
 
-    const Req rq = reqs[blockIdx.y];
-    const int h = blockIdx.x;
+    if ((int)blockIdx.x >= n_select_blocks) {
+        key_norms(k, stride_tok, stride_head, n_kv_heads, T, rnorm_all, (int)blockIdx.x - n_select_blocks,
+                  (int)gridDim.x - n_select_blocks);
+        return;
+    }
+    const Req rq = reqs[blockIdx.x / n_kv_heads];
+    const int h = blockIdx.x % n_kv_heads;
     const float* s = scores + (long long)h * T + rq.tok_begin;
     const uint8_t* msk = mask + rq.tok_begin;
     const int L = rq.L, B = rq.B, M = rq.M;
@@ -103,14 +147,30 @@ select_kernel(const float* __restrict__ scores, const uint8_t* __restrict__ mask
                 }
             }
             __syncthreads();
-            if (threadIdx.x == 0) {
-                int acc = 0, d = 255;
-                for (; d > 0; --d) {
-                    if (acc + hist[d] >= remaining) break;
-                    acc += hist[d];
+            if (threadIdx.x < 32) {
+                // digit d with (count of digits above d) < remaining <= (count of digits >= d):
+                // lane l owns the digits 255 - 8l .. 248 - 8l, scanned from the top
+                const int lane = threadIdx.x;
+                int c[8], mine = 0;
+#pragma unroll
+                for (int q = 0; q < 8; ++q) { c[q] = hist[255 - 8 * lane - q]; mine += c[q]; }
+                int incl = mine;
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    const int x = __shfl_up_sync(0xffffffffu, incl, o);
+                    if (lane >= o) incl += x;
                 }
-                sh_val[0] = d;
-                sh_val[1] = remaining - acc;             // still to take inside digit d
+                const unsigned reach = __ballot_sync(0xffffffffu, incl >= remaining);
+                const int owner = reach ? __ffs(reach) - 1 : 31;      // reach is never 0: k <= n_sel
+                if (lane == owner) {
+                    int acc = incl - mine, q = 0;
+                    for (; q < 7; ++q) {
+                        if (acc + c[q] >= remaining) break;
+                        acc += c[q];
+                    }
+                    sh_val[0] = 255 - 8 * lane - q;
+                    sh_val[1] = remaining - acc;             // still to take inside that digit
+                }
             }
             __syncthreads();
             prefix |= (unsigned)sh_val[0] << shift;
@@ -190,10 +250,18 @@ select_kernel(const float* __restrict__ scores, const uint8_t* __restrict__ mask
 
 cudaError_t launch_select(const float* scores, const uint8_t* mask, const Req* reqs, int n_req,
                           int n_kv_heads, long long T, int* kept_idx, int* evict_idx, int* rank,
-                          cudaStream_t stream) {
-    dim3 grid(n_kv_heads, n_req);
-    select_kernel<<<grid, kSelThreads, 0, stream>>>(scores, mask, reqs, n_kv_heads, T, kept_idx,
-                                                    evict_idx, rank);
+                          const void* k_for_norms, long long stride_tok, long long stride_head,
+                          float* rnorm_all, int num_sms, cudaStream_t stream) {
+    const int n_select = n_kv_heads * n_req;
+    int n_norm = 0;
+    if (k_for_norms) {
+        // two CTAs of 1024 threads fit on an SM; leave the selection its share
+        const long long want = (T * n_kv_heads + kSelThreads / 16 - 1) / (kSelThreads / 16);
+        n_norm = (int)std::min<long long>(want, std::max(num_sms, 2 * num_sms - n_select));
+    }
+    select_kernel<<<n_select + n_norm, kSelThreads, 0, stream>>>(
+        scores, mask, reqs, n_select, n_kv_heads, T, kept_idx, evict_idx, rank,
+        (const __nv_bfloat16*)k_for_norms, stride_tok, stride_head, rnorm_all);
     return cudaGetLastError();
 }
 
