@@ -97,14 +97,14 @@ __global__ void __launch_bounds__(kSelThreads)
 select_kernel(const float* __restrict__ scores, const uint8_t* __restrict__ mask,
               const Req* __restrict__ reqs, int n_select_blocks, int n_kv_heads, long long T,
               int* __restrict__ kept_idx, int* __restrict__ evict_idx, int* __restrict__ rank,
-              const __nv_bfloat16* __restrict__ k, long long stride_tok, long long stride_head,
+              const __nv_bfloat16* __restrict__ keys, long long stride_tok, long long stride_head,
               float* __restrict__ rnorm_all) {
     __shared__ int hist[256];
     __shared__ int warp_tot[32][2];
     __shared__ int sh_val[4];
 
     if ((int)blockIdx.x >= n_select_blocks) {
-        key_norms(k, stride_tok, stride_head, n_kv_heads, T, rnorm_all, (int)blockIdx.x - n_select_blocks,
+        key_norms(keys, stride_tok, stride_head, n_kv_heads, T, rnorm_all, (int)blockIdx.x - n_select_blocks,
                   (int)gridDim.x - n_select_blocks);
         return;
     }
