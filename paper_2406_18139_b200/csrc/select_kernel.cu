@@ -64,32 +64,55 @@ __device__ __forceinline__ void block_scan2(int a, int b, int& ea, int& eb, int&
     tb = warp_tot[31][1];
 }
 
-// 1 / |k| of every key row (0 for a zero row): half a warp per row, 16 bytes per lane.
+// 1 / |k| of every key row (0 for a zero row): half a warp per row, 16 bytes per lane, four rows
+// in flight per half-warp (the loop is bound by memory latency otherwise).  Row r is token
+// r / n_kv_heads of head r % n_kv_heads; the quotient and remainder are carried along instead of
+// divided out every time.
 __device__ __forceinline__ void key_norms(const __nv_bfloat16* __restrict__ k, long long stride_tok,
                                           long long stride_head, int n_kv_heads, long long T,
                                           float* __restrict__ rnorm_all, int block, int n_blocks) {
     constexpr int kRowsPerBlock = kSelThreads / 16;
+    constexpr int kFlight = 4;
     const int half = threadIdx.x >> 4, l16 = threadIdx.x & 15;
     const long long n_rows = T * n_kv_heads;
+    const long long step = (long long)n_blocks * kRowsPerBlock;      // rows between two of my rows
+    const long long step_tok = step / n_kv_heads;
+    const int step_h = (int)(step % n_kv_heads);
+    long long r = (long long)block * kRowsPerBlock + half;
+    long long tok = r / n_kv_heads;
+    int h = (int)(r % n_kv_heads);
     // the loop bound is the warp's first row, so that both half-warps always reach the shuffles
-    for (long long rw = (long long)block * kRowsPerBlock + (half & ~1); rw < n_rows;
-         rw += (long long)n_blocks * kRowsPerBlock) {
-        const long long r = rw + (half & 1);
-        const bool valid = r < n_rows;
-        const long long tok = valid ? r / n_kv_heads : 0;
-        const int h = valid ? (int)(r % n_kv_heads) : 0;
-        const uint4 u = *reinterpret_cast<const uint4*>(k + tok * stride_tok + h * stride_head + l16 * 8);
-        const unsigned w[4] = {u.x, u.y, u.z, u.w};
-        float ss = 0.f;
+    for (long long rw = r - (half & 1); rw < n_rows; rw += kFlight * step) {
+        uint4 u[kFlight];
+        long long tok_i[kFlight];
+        int h_i[kFlight];
+        bool valid[kFlight];
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            const float lo = __uint_as_float(w[i] << 16), hi = __uint_as_float(w[i] & 0xffff0000u);
-            ss = fmaf(lo, lo, ss);
-            ss = fmaf(hi, hi, ss);
+        for (int i = 0; i < kFlight; ++i) {
+            valid[i] = r < n_rows;
+            tok_i[i] = tok;
+            h_i[i] = h;
+            u[i] = make_uint4(0u, 0u, 0u, 0u);
+            if (valid[i]) u[i] = *reinterpret_cast<const uint4*>(k + tok * stride_tok + h * stride_head + l16 * 8);
+            r += step;
+            tok += step_tok;
+            h += step_h;
+            if (h >= n_kv_heads) { h -= n_kv_heads; ++tok; }
         }
 #pragma unroll
-        for (int o = 8; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o, 16);
-        if (l16 == 0 && valid) rnorm_all[(long long)h * T + tok] = ss > 0.f ? 1.0f / sqrtf(ss) : 0.f;
+        for (int i = 0; i < kFlight; ++i) {
+            const unsigned w[4] = {u[i].x, u[i].y, u[i].z, u[i].w};
+            float ss = 0.f;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const float lo = __uint_as_float(w[j] << 16), hi = __uint_as_float(w[j] & 0xffff0000u);
+                ss = fmaf(lo, lo, ss);
+                ss = fmaf(hi, hi, ss);
+            }
+#pragma unroll
+            for (int o = 8; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o, 16);
+            if (l16 == 0 && valid[i]) rnorm_all[(long long)h_i[i] * T + tok_i[i]] = ss > 0.f ? 1.0f / sqrtf(ss) : 0.f;
+        }
     }
 }
 
