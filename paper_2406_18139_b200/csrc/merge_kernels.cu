@@ -154,6 +154,8 @@ __device__ __forceinline__ void write_kept_entries(const Req& rq, int h, int n_k
     }
 }
 
+constexpr int kInvBatch = 8;                         // loop steps whose loads are issued together
+
 __global__ void __launch_bounds__(kInvThreads)
 invert_assignment_kernel(const int* __restrict__ assign, const int* __restrict__ kept_idx,
                          const int* __restrict__ evict_idx,
@@ -203,23 +205,28 @@ invert_assignment_kernel(const int* __restrict__ assign, const int* __restrict__
         unsigned* dst_v = key_buf[pass & 1] + E;
         for (int i = threadIdx.x; i < 32 * 256; i += kInvThreads) (&cnt[0][0])[i] = 0;
         __syncthreads();
-        // count
-        for (int base = s_begin; base < s_end; base += 32) {
-            const int i = base + lane;
-            const bool valid = i < s_end;
-            unsigned key = 0;
-            if (valid) {
-                if (pass) key = src_k[i];
-                else {
-                    int a = assign[ev_base + i];
-                    if (a < 0 || a >= B) { atomicExch(status, (int)LOOKM_ERR_DEVICE_BAD_INDEX); a = 0; }
-                    key = (unsigned)a;
-                }
+        // count (the loads of kInvBatch steps are issued together: the loop is bound by their latency)
+        for (int b0 = s_begin; b0 < s_end; b0 += 32 * kInvBatch) {
+            unsigned key[kInvBatch];
+#pragma unroll
+            for (int q = 0; q < kInvBatch; ++q) {
+                const int i = b0 + q * 32 + lane;
+                key[q] = 0u;
+                if (i < s_end) key[q] = pass ? src_k[i] : (unsigned)assign[ev_base + i];
             }
-            const unsigned d = valid ? ((key >> shift) & 255u) : 256u + lane;   // invalid lanes never match
-            const unsigned peers = __match_any_sync(0xffffffffu, d);
-            if (valid && (peers & lt_mask) == 0u) cnt[warp][d] += __popc(peers);
-            __syncwarp();
+#pragma unroll
+            for (int q = 0; q < kInvBatch; ++q) {
+                const int i = b0 + q * 32 + lane;
+                const bool valid = i < s_end;
+                if (valid && !pass && key[q] >= (unsigned)B) {
+                    atomicExch(status, (int)LOOKM_ERR_DEVICE_BAD_INDEX);
+                    key[q] = 0u;
+                }
+                const unsigned d = valid ? ((key[q] >> shift) & 255u) : 256u + lane;   // invalid lanes never match
+                const unsigned peers = __match_any_sync(0xffffffffu, d);
+                if (valid && (peers & lt_mask) == 0u) cnt[warp][d] += __popc(peers);
+                __syncwarp();
+            }
         }
         __syncthreads();
         // exclusive scan over (digit major, warp minor)
@@ -235,43 +242,70 @@ invert_assignment_kernel(const int* __restrict__ assign, const int* __restrict__
         }
         __syncthreads();
         // scatter
-        for (int base = s_begin; base < s_end; base += 32) {
-            const int i = base + lane;
-            const bool valid = i < s_end;
-            unsigned key = 0, val = 0;
-            if (valid) {
-                if (pass) { key = src_k[i]; val = src_v[i]; }
-                else {
-                    int a = assign[ev_base + i];
-                    if (a < 0 || a >= B) a = 0;
-                    key = (unsigned)a;
-                    val = (unsigned)i;
+        for (int b0 = s_begin; b0 < s_end; b0 += 32 * kInvBatch) {
+            unsigned key[kInvBatch], val[kInvBatch];
+#pragma unroll
+            for (int q = 0; q < kInvBatch; ++q) {
+                const int i = b0 + q * 32 + lane;
+                key[q] = 0u;
+                val[q] = (unsigned)i;
+                if (i < s_end) {
+                    if (pass) { key[q] = src_k[i]; val[q] = src_v[i]; }
+                    else key[q] = (unsigned)assign[ev_base + i];
                 }
             }
-            const unsigned d = valid ? ((key >> shift) & 255u) : 256u + lane;
-            const unsigned peers = __match_any_sync(0xffffffffu, d);
-            int off = 0;
-            if (valid) off = digit_tot[d] + cnt[warp][d] + __popc(peers & lt_mask);
-            __syncwarp();
-            if (valid && (peers & lt_mask) == 0u) cnt[warp][d] += __popc(peers);
-            __syncwarp();
-            if (valid) { dst_k[off] = key; dst_v[off] = val; }
+#pragma unroll
+            for (int q = 0; q < kInvBatch; ++q) {
+                const int i = b0 + q * 32 + lane;
+                const bool valid = i < s_end;
+                if (!pass && key[q] >= (unsigned)B) key[q] = 0u;
+                const unsigned d = valid ? ((key[q] >> shift) & 255u) : 256u + lane;
+                const unsigned peers = __match_any_sync(0xffffffffu, d);
+                int off = 0;
+                if (valid) off = digit_tot[d] + cnt[warp][d] + __popc(peers & lt_mask);
+                __syncwarp();
+                if (valid && (peers & lt_mask) == 0u) cnt[warp][d] += __popc(peers);
+                __syncwarp();
+                if (valid) { dst_k[off] = key[q]; dst_v[off] = val[q]; }
+            }
         }
         __syncthreads();
     }
     const unsigned* fin_k = key_buf[(n_pass - 1) & 1];
     const unsigned* fin_v = fin_k + E;
     // member entries and the row boundaries: row_ptr[c] = first sorted index whose slot is >= c
-    for (int i = threadIdx.x; i < E; i += kInvThreads) {
-        const int e = (int)fin_v[i];
-        int pe = evict_idx[ev_base + e];
-        if (pe < 0 || pe >= rq.L) { atomicExch(status, (int)LOOKM_ERR_DEVICE_BAD_INDEX); pe = 0; }
-        const int cur = (int)fin_k[i];
-        ent[i + cur + 1] = pe;                           // i-th member sits after cur + 1 kept rows
-        entw[i + cur + 1] = weighted ? sim[ev_base + e] : 1.0f;
-        const int prev = i ? (int)fin_k[i - 1] : -1;
-        for (int c = prev + 1; c <= cur; ++c) rp[c] = i;
-        if (i == E - 1) for (int c = cur + 1; c <= B; ++c) rp[c] = E;
+    for (int i0 = threadIdx.x; i0 < E; i0 += kInvThreads * kInvBatch) {
+        int e[kInvBatch], cur[kInvBatch], prev[kInvBatch], pe[kInvBatch];
+        float w[kInvBatch];
+#pragma unroll
+        for (int q = 0; q < kInvBatch; ++q) {
+            const int i = i0 + q * kInvThreads;
+            e[q] = 0; cur[q] = 0; prev[q] = -1;
+            if (i < E) {
+                e[q] = (int)fin_v[i];
+                cur[q] = (int)fin_k[i];
+                if (i) prev[q] = (int)fin_k[i - 1];
+            }
+        }
+#pragma unroll
+        for (int q = 0; q < kInvBatch; ++q) {
+            const int i = i0 + q * kInvThreads;
+            pe[q] = 0; w[q] = 1.0f;
+            if (i < E) {
+                pe[q] = evict_idx[ev_base + e[q]];
+                if (weighted) w[q] = sim[ev_base + e[q]];
+            }
+        }
+#pragma unroll
+        for (int q = 0; q < kInvBatch; ++q) {
+            const int i = i0 + q * kInvThreads;
+            if (i >= E) continue;
+            if (pe[q] < 0 || pe[q] >= rq.L) { atomicExch(status, (int)LOOKM_ERR_DEVICE_BAD_INDEX); pe[q] = 0; }
+            ent[i + cur[q] + 1] = pe[q];                 // i-th member sits after cur + 1 kept rows
+            entw[i + cur[q] + 1] = w[q];
+            for (int c = prev[q] + 1; c <= cur[q]; ++c) rp[c] = i;
+            if (i == E - 1) for (int c = cur[q] + 1; c <= B; ++c) rp[c] = E;
+        }
     }
     __syncthreads();
     write_kept_entries(rq, h, n_kv_heads, B, rp, kept_idx_head, ent, entw, units, cnts, status);
