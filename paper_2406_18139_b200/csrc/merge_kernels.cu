@@ -154,6 +154,19 @@ __device__ __forceinline__ void write_kept_entries(const Req& rq, int h, int n_k
     }
 }
 
+// Lanes of the warp that hold a valid element with the same 8-bit digit as the caller: one ballot
+// per bit (match.any takes a step per distinct value, i.e. up to 32 for well-mixed digits).
+__device__ __forceinline__ unsigned same_digit_lanes(unsigned d, bool valid) {
+    unsigned peers = __ballot_sync(0xffffffffu, valid);
+#pragma unroll
+    for (int b = 0; b < 8; ++b) {
+        const bool bit = (d >> b) & 1u;
+        const unsigned bal = __ballot_sync(0xffffffffu, bit);
+        peers &= bit ? bal : ~bal;
+    }
+    return peers;
+}
+
 constexpr int kInvBatch = 8;                         // loop steps whose loads are issued together
 
 __global__ void __launch_bounds__(kInvThreads)
@@ -222,8 +235,8 @@ invert_assignment_kernel(const int* __restrict__ assign, const int* __restrict__
                     atomicExch(status, (int)LOOKM_ERR_DEVICE_BAD_INDEX);
                     key[q] = 0u;
                 }
-                const unsigned d = valid ? ((key[q] >> shift) & 255u) : 256u + lane;   // invalid lanes never match
-                const unsigned peers = __match_any_sync(0xffffffffu, d);
+                const unsigned d = (key[q] >> shift) & 255u;
+                const unsigned peers = same_digit_lanes(d, valid);
                 if (valid && (peers & lt_mask) == 0u) cnt[warp][d] += __popc(peers);
                 __syncwarp();
             }
@@ -236,9 +249,19 @@ invert_assignment_kernel(const int* __restrict__ assign, const int* __restrict__
             digit_tot[threadIdx.x] = tot;
         }
         __syncthreads();
-        if (threadIdx.x == 0) {
-            int run = 0;
-            for (int d = 0; d < 256; ++d) { const int c = digit_tot[d]; digit_tot[d] = run; run += c; }
+        if (threadIdx.x < 32) {                          // exclusive scan of the 256 totals: 8 per lane
+            int c[8], mine = 0;
+#pragma unroll
+            for (int q = 0; q < 8; ++q) { c[q] = digit_tot[8 * lane + q]; mine += c[q]; }
+            int incl = mine;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int x = __shfl_up_sync(0xffffffffu, incl, o);
+                if (lane >= o) incl += x;
+            }
+            int run = incl - mine;
+#pragma unroll
+            for (int q = 0; q < 8; ++q) { digit_tot[8 * lane + q] = run; run += c[q]; }
         }
         __syncthreads();
         // scatter
@@ -259,8 +282,8 @@ invert_assignment_kernel(const int* __restrict__ assign, const int* __restrict__
                 const int i = b0 + q * 32 + lane;
                 const bool valid = i < s_end;
                 if (!pass && key[q] >= (unsigned)B) key[q] = 0u;
-                const unsigned d = valid ? ((key[q] >> shift) & 255u) : 256u + lane;
-                const unsigned peers = __match_any_sync(0xffffffffu, d);
+                const unsigned d = (key[q] >> shift) & 255u;
+                const unsigned peers = same_digit_lanes(d, valid);
                 int off = 0;
                 if (valid) off = digit_tot[d] + cnt[warp][d] + __popc(peers & lt_mask);
                 __syncwarp();
