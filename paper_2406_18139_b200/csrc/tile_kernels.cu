@@ -47,11 +47,12 @@ struct __align__(1024) Shared {
     uint8_t a[2][kTileBytes];                    // stationary tiles (double-buffered across items)
     uint8_t b[kStages][kTileBytes];              // streamed tiles
     float side[kGroups][2][kTile];               // per epilogue group, double-buffered column data
-    float comb[2][kGroups - 1][2][kTile];        // partial results of groups 1.., double-buffered
+    float comb[2][kGroups][2][kTile];            // partial results of the groups, double-buffered
     Req reqs[kReqCache];                         // copy of the request table (when it fits)
     unsigned long long a_full[2], a_empty[2];
     unsigned long long b_full[kStages], b_empty[kStages];
     unsigned long long t_full[kAccum], t_empty[kAccum];
+    unsigned long long comb_full[2], comb_free[2];   // partial results of an item written / read
     unsigned long long mma_done;                 // every MMA of this CTA has completed
     uint32_t tmem_base;
     int abort_flag;
@@ -132,6 +133,10 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         for (int i = 0; i < kAccum; ++i) {
             ptx::mbar_init(ptx::smem_u32(&sh.t_full[i]), 1);
             ptx::mbar_init(ptx::smem_u32(&sh.t_empty[i]), 4);   // one arrival per epilogue warp
+        }
+        for (int i = 0; i < 2; ++i) {
+            ptx::mbar_init(ptx::smem_u32(&sh.comb_full[i]), (kGroups - 1) * 4);   // warps of the other groups
+            ptx::mbar_init(ptx::smem_u32(&sh.comb_free[i]), 4);                   // warps of the combining group
         }
         ptx::mbar_init(ptx::smem_u32(&sh.mma_done), kIssuers);
         sh.abort_flag = 0;
@@ -420,44 +425,64 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
             }
 
             // ---- combine the four groups and write this item's results -----------------------
-            if (wg > 0) {
-                float* cb0 = sh.comb[n & 1][wg - 1][0];
-                float* cb1 = sh.comb[n & 1][wg - 1][1];
-                if (KIND == kSweep1) { cb0[row] = m_run; cb1[row] = l_run; }
-                else if (KIND == kSweep2) { cb0[row] = (acc0 + acc1) + (acc2 + acc3); }
-                else { cb0[row] = best; cb1[row] = __int_as_float(best_slot); }
-            }
-            ptx::named_barrier_sync(1 + kGroups, kGroups * 128);
-            if (wg == 0 && pos < it.L && !*abort_flag) {
-                if (KIND == kSweep1) {
-                    float m = m_run;
+            // The group that owns the item's last tile finishes last anyway, so it combines: the
+            // others leave their partial results in shared memory, signal, and go on to the next
+            // item without waiting for anybody.  Values are always combined in group order.
+            const int cslot = n & 1;
+            const uint32_t cuse = static_cast<uint32_t>(n) >> 1;         // earlier uses of this buffer
+            const int combiner = static_cast<int>((gb - 1u) % kGroups);
+            float (*cb)[2][kTile] = sh.comb[cslot];
+            if (wg != combiner) {
+                // the buffer's previous contents (two items ago) have been read
+                ptx::mbar_wait(ptx::smem_u32(&sh.comb_free[cslot]), (cuse & 1u) ^ 1u, abort_flag);
+                if (KIND == kSweep1) { cb[wg][0][row] = m_run; cb[wg][1][row] = l_run; }
+                else if (KIND == kSweep2) { cb[wg][0][row] = (acc0 + acc1) + (acc2 + acc3); }
+                else { cb[wg][0][row] = best; cb[wg][1][row] = __int_as_float(best_slot); }
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&sh.comb_full[cslot]));
+            } else {
+                ptx::mbar_wait(ptx::smem_u32(&sh.comb_full[cslot]), cuse & 1u, abort_flag);
+                if (pos < it.L && !*abort_flag) {
+                    if (KIND == kSweep1) {
+                        float mg[kGroups], lg[kGroups];
 #pragma unroll
-                    for (int g = 0; g < kGroups - 1; ++g) m = fmaxf(m, sh.comb[n & 1][g][0][row]);
-                    float l = l_run * ptx::ex2((m_run - m) * c2);
-#pragma unroll
-                    for (int g = 0; g < kGroups - 1; ++g)
-                        l += sh.comb[n & 1][g][1][row] * ptx::ex2((sh.comb[n & 1][g][0][row] - m) * c2);
-                    // natural-log log-sum-exp of the scaled logits
-                    p.lse[(long long)it.head * p.T + it.tok_begin + pos] = (m * c2 + ptx::lg2(l)) * kLn2;
-                } else if (KIND == kSweep2) {
-                    float a = (acc0 + acc1) + (acc2 + acc3);
-#pragma unroll
-                    for (int g = 0; g < kGroups - 1; ++g) a += sh.comb[n & 1][g][0][row];
-                    p.scores[(long long)it.head * p.T + it.tok_begin + pos] = a;
-                } else {
-                    const long long g = (long long)it.head * p.T + it.tok_begin + pos;
-                    const int e = p.rank[g];
-                    if (e >= 0) {
-#pragma unroll
-                        for (int gi = 0; gi < kGroups - 1; ++gi) {
-                            const float b1 = sh.comb[n & 1][gi][0][row];
-                            const int s1 = __float_as_int(sh.comb[n & 1][gi][1][row]);
-                            if (b1 > best || (b1 == best && s1 < best_slot)) { best = b1; best_slot = s1; }
+                        for (int g = 0; g < kGroups; ++g) {
+                            mg[g] = (g == wg) ? m_run : cb[g][0][row];
+                            lg[g] = (g == wg) ? l_run : cb[g][1][row];
                         }
-                        p.assign[it.ev0 + e] = best_slot;
-                        p.sim[it.ev0 + e] = best * p.rnorm_all[g];
+                        float m = mg[0];
+#pragma unroll
+                        for (int g = 1; g < kGroups; ++g) m = fmaxf(m, mg[g]);
+                        float l = lg[0] * ptx::ex2((mg[0] - m) * c2);
+#pragma unroll
+                        for (int g = 1; g < kGroups; ++g) l += lg[g] * ptx::ex2((mg[g] - m) * c2);
+                        // natural-log log-sum-exp of the scaled logits
+                        p.lse[(long long)it.head * p.T + it.tok_begin + pos] = (m * c2 + ptx::lg2(l)) * kLn2;
+                    } else if (KIND == kSweep2) {
+                        const float own = (acc0 + acc1) + (acc2 + acc3);
+                        float a = (wg == 0) ? own : cb[0][0][row];
+#pragma unroll
+                        for (int g = 1; g < kGroups; ++g) a += (g == wg) ? own : cb[g][0][row];
+                        p.scores[(long long)it.head * p.T + it.tok_begin + pos] = a;
+                    } else {
+                        const long long gi = (long long)it.head * p.T + it.tok_begin + pos;
+                        const int e = p.rank[gi];
+                        if (e >= 0) {
+                            float bb = (wg == 0) ? best : cb[0][0][row];
+                            int bs = (wg == 0) ? best_slot : __float_as_int(cb[0][1][row]);
+#pragma unroll
+                            for (int g = 1; g < kGroups; ++g) {
+                                const float b1 = (g == wg) ? best : cb[g][0][row];
+                                const int s1 = (g == wg) ? best_slot : __float_as_int(cb[g][1][row]);
+                                if (b1 > bb || (b1 == bb && s1 < bs)) { bb = b1; bs = s1; }
+                            }
+                            p.assign[it.ev0 + e] = bs;
+                            p.sim[it.ev0 + e] = bb * p.rnorm_all[gi];
+                        }
                     }
                 }
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&sh.comb_free[cslot]));
             }
         }
     }
