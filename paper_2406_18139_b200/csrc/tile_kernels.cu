@@ -309,53 +309,6 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                 ++lt;
                 ptx::mbar_wait(ptx::smem_u32(&sh.t_full[buf]), (gb / kAccum) & 1, abort_flag);
                 ptx::tc_fence_after_sync();
-                if (KIND == kSweep2) {
-                    // probabilities of key `pos` under the tile's 128 query columns, 16 columns at a
-                    // time with the next 16 already on their way from TMEM
-                    auto columns16 = [&](const uint32_t (&r)[16], int c0) {
-                        const float4* sd = reinterpret_cast<const float4*>(side + c0);
-#pragma unroll
-                        for (int c4 = 0; c4 < 4; ++c4) {
-                            const float4 l4 = sd[c4];
-                            const int c = c0 + c4 * 4;
-                            const float e0 = exp2_mixed(c4 * 4 + 0, fmaf(__uint_as_float(r[c4 * 4 + 0]), c2, -l4.x));
-                            const float e1 = exp2_mixed(c4 * 4 + 1, fmaf(__uint_as_float(r[c4 * 4 + 1]), c2, -l4.y));
-                            const float e2 = exp2_mixed(c4 * 4 + 2, fmaf(__uint_as_float(r[c4 * 4 + 2]), c2, -l4.z));
-                            const float e3 = exp2_mixed(c4 * 4 + 3, fmaf(__uint_as_float(r[c4 * 4 + 3]), c2, -l4.w));
-                            if (diag) {
-                                acc0 += (c + 0 >= row) ? e0 : 0.f;
-                                acc1 += (c + 1 >= row) ? e1 : 0.f;
-                                acc2 += (c + 2 >= row) ? e2 : 0.f;
-                                acc3 += (c + 3 >= row) ? e3 : 0.f;
-                            } else {
-                                acc0 += e0;
-                                acc1 += e1;
-                                acc2 += e2;
-                                acc3 += e3;
-                            }
-                        }
-                    };
-                    uint32_t ra[16], rb[16];
-                    const uint32_t tbase = lane_addr + buf * kTile;
-                    ptx::tmem_ld_32x16(tbase, ra);
-#pragma unroll
-                    for (int k = 0; k < 4; ++k) {
-                        ptx::tmem_ld_wait16(ra);
-                        ptx::tmem_ld_32x16(tbase + (2 * k + 1) * 16, rb);
-                        columns16(ra, 2 * k * 16);
-                        ptx::tmem_ld_wait16(rb);
-                        if (k < 3) {
-                            ptx::tmem_ld_32x16(tbase + (2 * k + 2) * 16, ra);
-                        } else {
-                            // everything is in registers: hand the accumulator back
-                            ptx::tc_fence_before_sync();
-                            __syncwarp();
-                            if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&sh.t_empty[buf]));
-                        }
-                        columns16(rb, (2 * k + 1) * 16);
-                    }
-                    continue;
-                }
 #pragma unroll 1
                 for (int ch = 0; ch < 4; ++ch) {
                     uint32_t raw[32];
