@@ -432,23 +432,11 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
             const uint32_t cuse = static_cast<uint32_t>(n) >> 1;         // earlier uses of this buffer
             const int combiner = static_cast<int>((gb - 1u) % kGroups);
             float (*cb)[2][kTile] = sh.comb[cslot];
-            if (KIND == kSweep2) {
-                // Sweep 2 is the exception: measured at 8192 x 32, it runs at 0.354 ms when all
-                // groups meet at a barrier after every item and group 0 combines, against 0.363 ms
-                // with the scheme above (and 0.371 ms with that scheme plus a barrier).
-                const float own = (acc0 + acc1) + (acc2 + acc3);
-                if (wg > 0) cb[wg][0][row] = own;
-                ptx::named_barrier_sync(1 + kGroups, kGroups * 128);
-                if (wg == 0 && pos < it.L && !*abort_flag) {
-                    float a = own;
-#pragma unroll
-                    for (int g = 1; g < kGroups; ++g) a += cb[g][0][row];
-                    p.scores[(long long)it.head * p.T + it.tok_begin + pos] = a;
-                }
-            } else if (wg != combiner) {
+            if (wg != combiner) {
                 // the buffer's previous contents (two items ago) have been read
                 ptx::mbar_wait(ptx::smem_u32(&sh.comb_free[cslot]), (cuse & 1u) ^ 1u, abort_flag);
                 if (KIND == kSweep1) { cb[wg][0][row] = m_run; cb[wg][1][row] = l_run; }
+                else if (KIND == kSweep2) { cb[wg][0][row] = (acc0 + acc1) + (acc2 + acc3); }
                 else { cb[wg][0][row] = best; cb[wg][1][row] = __int_as_float(best_slot); }
                 __syncwarp();
                 if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&sh.comb_full[cslot]));
@@ -470,6 +458,12 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                         for (int g = 1; g < kGroups; ++g) l += lg[g] * ptx::ex2((mg[g] - m) * c2);
                         // natural-log log-sum-exp of the scaled logits
                         p.lse[(long long)it.head * p.T + it.tok_begin + pos] = (m * c2 + ptx::lg2(l)) * kLn2;
+                    } else if (KIND == kSweep2) {
+                        const float own = (acc0 + acc1) + (acc2 + acc3);
+                        float a = (wg == 0) ? own : cb[0][0][row];
+#pragma unroll
+                        for (int g = 1; g < kGroups; ++g) a += (g == wg) ? own : cb[g][0][row];
+                        p.scores[(long long)it.head * p.T + it.tok_begin + pos] = a;
                     } else {
                         const long long gi = (long long)it.head * p.T + it.tok_begin + pos;
                         const int e = p.rank[gi];
