@@ -278,9 +278,11 @@ cudaError_t launch_select(const float* scores, const uint8_t* mask, const Req* r
     const int n_select = n_kv_heads * n_req;
     int n_norm = 0;
     if (k_for_norms) {
-        // two CTAs of 1024 threads fit on an SM; leave the selection its share
+        // one CTA of this kernel fits on an SM: the norm CTAs take the SMs that the selection
+        // leaves free, so that all of them run at once (a second wave would have to wait for the
+        // selection CTAs, which run longest)
         const long long want = (T * n_kv_heads + kSelThreads / 16 - 1) / (kSelThreads / 16);
-        n_norm = (int)std::min<long long>(want, std::max(num_sms, 2 * num_sms - n_select));
+        n_norm = (int)std::min<long long>(want, n_select < num_sms ? num_sms - n_select : num_sms);
     }
     select_kernel<<<n_select + n_norm, kSelThreads, 0, stream>>>(
         scores, mask, reqs, n_select, n_kv_heads, T, kept_idx, evict_idx, rank,
