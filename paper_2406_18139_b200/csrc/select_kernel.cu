@@ -22,7 +22,7 @@ namespace lookm {
 namespace {
 
 constexpr int kSelThreads = 1024;
-constexpr int kPerThread = 4;
+constexpr int kPerThread = 8;
 
 __device__ __forceinline__ unsigned order_key(float s) {
     unsigned b = __float_as_uint(s);
