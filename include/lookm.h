@@ -193,7 +193,8 @@ int lookm_noalloc_status(void* cuda_stream);
  * step boundaries: [0] start, [1] after the first score sweep, [2] after the second (Eq. 4),
  * [3] after the selection (Eq. 5-8; the same launch computes the key norms of Eq. 9), [4] after
  * the kept-key compaction, [5] after the matching (Eq. 9), [6] after the assignment inversion, [7] after merge + compaction (Eq. 10-12).
- * n_events must be LOOKM_N_STAGE_EVENTS; pass NULL, 0 to stop.  Nothing is recorded otherwise. */
+ * n_events must be LOOKM_N_STAGE_EVENTS; a NULL entry skips that boundary; pass NULL, 0 to stop.
+ * Nothing is recorded otherwise. */
 #define LOOKM_N_STAGE_EVENTS 8
 int lookm_set_stage_events(void* const* events_host, int n_events);
 

@@ -240,12 +240,12 @@ _stage_event_array = None
 
 def lookm_set_stage_events(events) -> int:
     """events: 8 torch.cuda.Event (created with enable_timing=True and recorded once so that their
-    handles exist), or None to stop per-stage timing."""
+    handles exist; an entry may be None to skip that boundary), or None to stop per-stage timing."""
     global _stage_event_array
     if events is None:
         _stage_event_array = None
         return lib().lookm_set_stage_events(None, 0)
-    arr = (C.c_void_p * len(events))(*[e.cuda_event for e in events])
+    arr = (C.c_void_p * len(events))(*[(e.cuda_event if e is not None else None) for e in events])
     _stage_event_array = arr                     # the library keeps the pointer: keep it alive
     return lib().lookm_set_stage_events(arr, len(events))
 
