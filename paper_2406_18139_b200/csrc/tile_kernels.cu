@@ -309,6 +309,63 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                 ++lt;
                 ptx::mbar_wait(ptx::smem_u32(&sh.t_full[buf]), (gb / kAccum) & 1, abort_flag);
                 ptx::tc_fence_after_sync();
+                if (KIND == kMatch) {
+                    // running arg-max of dot / |kept key| over kept slots, 16 columns at a time with
+                    // the next 16 already on their way from TMEM (a load takes about as long as
+                    // the work on 32 columns).  The maximum of the 16 is taken first; only when it
+                    // beats the running best is its first column looked up, so a strict comparison
+                    // in ascending slot order keeps the lowest slot.
+                    auto columns16 = [&](const uint32_t (&r)[16], int c0) {
+                        const float4* sd = reinterpret_cast<const float4*>(side + c0);
+                        float v[16];
+#pragma unroll
+                        for (int c4 = 0; c4 < 4; ++c4) {
+                            const float4 r4 = sd[c4];
+                            v[c4 * 4 + 0] = __uint_as_float(r[c4 * 4 + 0]) * r4.x;
+                            v[c4 * 4 + 1] = __uint_as_float(r[c4 * 4 + 1]) * r4.y;
+                            v[c4 * 4 + 2] = __uint_as_float(r[c4 * 4 + 2]) * r4.z;
+                            v[c4 * 4 + 3] = __uint_as_float(r[c4 * 4 + 3]) * r4.w;
+                        }
+                        if (col_limit < kTile) {           // last tile of the kept list only
+#pragma unroll
+                            for (int c = 0; c < 16; ++c)
+                                if (c0 + c >= col_limit) v[c] = -INFINITY;
+                        }
+                        const float m0 = ptx::fmax3(v[0], v[1], v[2]);
+                        const float m1 = ptx::fmax3(v[3], v[4], v[5]);
+                        const float m2 = ptx::fmax3(v[6], v[7], v[8]);
+                        const float m3 = ptx::fmax3(v[9], v[10], v[11]);
+                        const float m4 = ptx::fmax3(v[12], v[13], v[14]);
+                        const float mx = fmaxf(ptx::fmax3(m0, m1, m2), ptx::fmax3(m3, m4, v[15]));
+                        if (mx > best) {
+                            best = mx;
+                            int idx = 15;
+#pragma unroll
+                            for (int c = 14; c >= 0; --c) if (v[c] == mx) idx = c;
+                            best_slot = t * kTile + c0 + idx;
+                        }
+                    };
+                    uint32_t ra[16], rb[16];
+                    const uint32_t tbase = lane_addr + buf * kTile;
+                    ptx::tmem_ld_32x16(tbase, ra);
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        ptx::tmem_ld_wait16(ra);
+                        ptx::tmem_ld_32x16(tbase + (2 * k + 1) * 16, rb, ra);
+                        columns16(ra, 2 * k * 16);
+                        ptx::tmem_ld_wait16(rb);
+                        if (k < 3) {
+                            ptx::tmem_ld_32x16(tbase + (2 * k + 2) * 16, ra, rb);
+                        } else {
+                            // everything is in registers: hand the accumulator back
+                            ptx::tc_fence_before_sync();
+                            __syncwarp();
+                            if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&sh.t_empty[buf]));
+                        }
+                        columns16(rb, (2 * k + 1) * 16);
+                    }
+                    continue;
+                }
 #pragma unroll 1
                 for (int ch = 0; ch < 4; ++ch) {
                     uint32_t raw[32];
