@@ -439,44 +439,6 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                                 acc3 += exp2_mixed(c4 * 4 + 3, fmaf(__uint_as_float(raw[c4 * 4 + 3]), c2, -l4.w));
                             }
                         }
-                    } else {
-                        // running arg-max of dot / |kept key| over kept slots.  Per 16 columns the
-                        // maximum is taken first (two instructions per element); only when it beats
-                        // the running best (rare after the first tiles) is its first column looked
-                        // up, so a strict comparison in ascending slot order keeps the lowest slot
-                        const float4* sd = reinterpret_cast<const float4*>(side + c0);
-                        const int slot0 = t * kTile + c0;
-#pragma unroll
-                        for (int g16 = 0; g16 < 2; ++g16) {
-                            float v[16];
-#pragma unroll
-                            for (int c4 = 0; c4 < 4; ++c4) {
-                                const float4 r4 = sd[g16 * 4 + c4];
-                                const int c = g16 * 16 + c4 * 4;
-                                v[c4 * 4 + 0] = __uint_as_float(raw[c + 0]) * r4.x;
-                                v[c4 * 4 + 1] = __uint_as_float(raw[c + 1]) * r4.y;
-                                v[c4 * 4 + 2] = __uint_as_float(raw[c + 2]) * r4.z;
-                                v[c4 * 4 + 3] = __uint_as_float(raw[c + 3]) * r4.w;
-                            }
-                            if (col_limit < kTile) {       // last tile of the kept list only
-#pragma unroll
-                                for (int c = 0; c < 16; ++c)
-                                    if (c0 + g16 * 16 + c >= col_limit) v[c] = -INFINITY;
-                            }
-                            const float m0 = ptx::fmax3(v[0], v[1], v[2]);
-                            const float m1 = ptx::fmax3(v[3], v[4], v[5]);
-                            const float m2 = ptx::fmax3(v[6], v[7], v[8]);
-                            const float m3 = ptx::fmax3(v[9], v[10], v[11]);
-                            const float m4 = ptx::fmax3(v[12], v[13], v[14]);
-                            const float mx = fmaxf(ptx::fmax3(m0, m1, m2), ptx::fmax3(m3, m4, v[15]));
-                            if (mx > best) {
-                                best = mx;
-                                int idx = 15;
-#pragma unroll
-                                for (int c = 14; c >= 0; --c) if (v[c] == mx) idx = c;
-                                best_slot = slot0 + g16 * 16 + idx;
-                            }
-                        }
                     }
                 }
             }
