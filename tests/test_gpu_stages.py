@@ -274,6 +274,49 @@ def test_merge_matches_oracle_on_oracle_lists(B, mode, L, budget, Hkv):
         assert np.array_equal(gk[h][empty], kf[kept[h][empty], h].astype(np.float64))   # bit-exact copy
 
 
+def test_merge_packed_batch_with_slots_spread_over_many_work_units(B):
+    """Two requests, batch output layout, member counts from 0 to many hundreds: the kernel cuts its
+    work units at fixed entry counts, so most of the large slots are summed piecewise by several
+    warps; every merge mode appears once."""
+    import torch
+    Hkv = 3
+    lens, budgets, modes = [1700, 900], [25, 60], [2, 1]
+    w0 = synth.tiny(sum(lens), Hkv, Hkv, 10, 4, 0, seed=77)
+    (q, k, v), (qf, kf, vf), _, _ = _tensors(w0)
+    cu = [0, lens[0], sum(lens)]
+    kept, ev, assign, sim, per = [], [], [], [], []
+    for r, (L, bud) in enumerate(zip(lens, budgets)):
+        E = L - bud
+        for h in range(Hkv):
+            pos = np.sort(synth.uniform_int(synth.stream_key(120, r, h), 4 * bud, 0, L - 1))
+            a = np.unique(pos)[:bud].astype(np.int32)
+            assert len(a) == bud
+            b = np.setdiff1d(np.arange(L, dtype=np.int32), a)
+            asg = synth.uniform_int(synth.stream_key(121, r, h), E, 0, bud - 1).astype(np.int32)
+            asg[: (2 * E) // 3] = 3 + h                      # two thirds of the rows in one slot
+            asg[asg == 1] = 2                                # slot 1 gets nobody
+            sm = np.clip(synth.normal(synth.stream_key(122, r, h), E) * 0.4, -1, 1).astype(np.float32)
+            kept.append(a), ev.append(b), assign.append(asg), sim.append(sm)
+            per.append((r, h, a, b, asg, sm))
+    dev = lambda xs: torch.from_numpy(np.concatenate(xs)).cuda()
+    out_k = torch.zeros(sum(budgets), Hkv, 128, dtype=torch.bfloat16, device="cuda")
+    out_v = torch.zeros_like(out_k)
+    lay = B.make_layout(None, k)
+    ws = B.alloc_workspace(lay, lens)
+    B.check(B.lookm_merge(k, v, dev(kept), dev(ev), dev(assign), dev(sim), cu, budgets, modes, lay,
+                          1, out_k, out_v, ws))
+    assert B.lookm_device_status(ws) == B.OK
+    gk, gv = bf16_to_np(out_k), bf16_to_np(out_v)
+    out_cu = np.concatenate([[0], np.cumsum(budgets)])
+    for r, h, a, b, asg, sm in per:
+        kr, vr = kf[cu[r]:cu[r + 1]], vf[cu[r]:cu[r + 1]]
+        rk = orc.merge(kr, h, a, b, asg, sm.astype(np.float64), modes[r])
+        rv = orc.merge(vr, h, a, b, asg, sm.astype(np.float64), modes[r])
+        assert merged_close(gk[out_cu[r]:out_cu[r + 1], h], rk).all()
+        assert merged_close(gv[out_cu[r]:out_cu[r + 1], h], rv).all()
+        assert np.array_equal(gk[out_cu[r] + 1, h], kr[a[1], h].astype(np.float64))   # no members: copied
+
+
 def test_merge_single_kept_token_and_bad_index_status(B):
     import torch
     L = 700
