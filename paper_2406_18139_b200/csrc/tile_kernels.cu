@@ -368,14 +368,9 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                 }
 #pragma unroll 1
                 for (int ch = 0; ch < 4; ++ch) {
-                    // on the diagonal tile a warp whose 32 rows lie entirely on the masked side of
-                    // these 32 columns has nothing to do with them
-                    const bool masked = diag && (KIND == kSweep1 ? ch > quarter : ch < quarter);
                     uint32_t raw[32];
-                    if (!masked) {
-                        ptx::tmem_ld_32x32(lane_addr + buf * kTile + ch * 32, raw);
-                        ptx::tmem_ld_wait();
-                    }
+                    ptx::tmem_ld_32x32(lane_addr + buf * kTile + ch * 32, raw);
+                    ptx::tmem_ld_wait();
                     if (ch == 3) {
                         // the last columns are in registers: hand the accumulator back now, so
                         // that the next tile's MMAs run while this chunk is still being worked on
@@ -383,7 +378,6 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                         __syncwarp();
                         if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&sh.t_empty[buf]));
                     }
-                    if (masked) continue;
                     const int c0 = ch * 32;
                     if (KIND == kSweep1) {
                         // online softmax statistics of row `pos` over key columns c0..c0+31
