@@ -150,6 +150,50 @@ def test_ragged_batch_equals_oracle_per_request(B):
     assert stats["kept_near_ties"] <= 1
 
 
+def test_batch_of_many_short_requests(B):
+    """90 requests in one call: more than the kernels keep of the request table in shared memory and
+    more than one launch of the table writer carries; lengths from 1 token up, some budgets at or
+    above the length (nothing evicted) and one single-token request."""
+    import torch
+    n = 90
+    lens = (synth.uniform_int(synth.stream_key(300), n, 20, 260)).astype(int).tolist()
+    lens[7], lens[41] = 1, 129
+    budgets = [max(1, L // (2 + i % 4)) for i, L in enumerate(lens)]
+    budgets[3], budgets[60] = lens[3], lens[60] + 5
+    windows = [i % 7 for i in range(n)]
+    modes = [i % 3 for i in range(n)]
+    Hq, Hkv = 2, 2
+    reqs = [synth.tiny(L, Hq, Hkv, b, m, mo, image_spans=[(L // 5, (3 * L) // 4)], seed=400 + i)
+            for i, (L, b, m, mo) in enumerate(zip(lens, budgets, windows, modes))]
+    parts = [synth.layer_tensors(w) for w in reqs]
+    qb, kb, vb = (np.concatenate([p[i] for p in parts]) for i in range(3))
+    mask = np.concatenate([w.requests[0].mask for w in reqs])
+    q, k, v = to_dev(qb), to_dev(kb), to_dev(vb)
+    cu = np.concatenate([[0], np.cumsum(lens)]).tolist()
+    lay = B.make_layout(q, k)
+    ws = B.alloc_workspace(lay, lens)
+    outs = [min(b, L) for b, L in zip(budgets, lens)]
+    out_k = torch.zeros(sum(outs), Hkv, 128, dtype=torch.bfloat16, device="cuda")
+    out_v = torch.zeros_like(out_k)
+    st, out_cu = B.lookm_compress_varlen(q, k, v, torch.from_numpy(mask).cuda(), cu, budgets, windows,
+                                         modes, lay, out_k, out_v, ws)
+    B.check(st)
+    assert out_cu == np.concatenate([[0], np.cumsum(outs)]).tolist()
+    assert B.lookm_device_status(ws) == B.OK
+    _, lists = B.read_intermediates(ws, lay, lens, budgets)
+    gk, gv = bf16_to_np(out_k), bf16_to_np(out_v)
+    stats = {"kept_near_ties": 0, "assign_near_ties": 0}
+    for r in range(n):
+        a, b = cu[r], cu[r + 1]
+        qf, kf, vf = (synth.bf16_to_f32(t[a:b]) for t in (qb, kb, vb))
+        A = orc.scores(qf, kf, threads=2)
+        for h in range(Hkv):
+            kept_g, ev_g, asg_g, _ = lists[r][h]
+            check_head(kf, vf, mask[a:b], h, budgets[r], windows[r], modes[r], A[h], kept_g, ev_g, asg_g,
+                       gk[out_cu[r]:out_cu[r + 1], h], gv[out_cu[r]:out_cu[r + 1], h], stats)
+    assert stats["kept_near_ties"] <= 2
+
+
 def test_gqa_scores_are_summed_over_the_group(B):
     w = synth.tiny(700, 8, 2, 140, 16, 1, image_spans=[(50, 600)], seed=77)
     run_layer(B, w, threads=4)
