@@ -103,4 +103,29 @@ cudaError_t launch_merge(const void* k, const void* v, long long stride_tok, lon
                          int varlen_output, void* out_k, void* out_v, int* status, int num_sms,
                          cudaStream_t stream);
 
+// Launch with programmatic stream serialisation: the grid may be set up while the kernel before it
+// in the stream drains.  Every kernel launched this way starts with grid_dependency_wait(), which
+// returns once that kernel has completed and its writes are visible (a no-op for plain launches).
+#ifdef __CUDACC__
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_chained(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem,
+                                  cudaStream_t stream, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+__device__ __forceinline__ void grid_dependency_wait() {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+#endif
+
 }  // namespace lookm

@@ -78,6 +78,7 @@ gather_kept_kernel(const __nv_bfloat16* __restrict__ k, long long stride_tok, lo
                    long long total_rows, const int* __restrict__ kept_idx,
                    const float* __restrict__ rnorm_all, __nv_bfloat16* __restrict__ kept_keys,
                    float* __restrict__ rnorm_kept, int* status) {
+    grid_dependency_wait();
     const int half = threadIdx.x >> 4, l16 = threadIdx.x & 15;
     const long long g = (long long)blockIdx.x * 16 + half;
     if (g >= total_rows) return;
@@ -177,6 +178,7 @@ invert_assignment_kernel(const int* __restrict__ assign, const int* __restrict__
                          int* __restrict__ ent_pos, float* __restrict__ ent_w,
                          int4* __restrict__ unit_first, int* __restrict__ slot_cnt,
                          unsigned* __restrict__ sort_a, unsigned* __restrict__ sort_b, int* status) {
+    grid_dependency_wait();
     __shared__ int cnt[32][256];                         // [warp][digit]
     __shared__ int digit_tot[256];
     const Req rq = reqs[blockIdx.y];
@@ -397,6 +399,7 @@ merge_kernel(const __nv_bfloat16* __restrict__ k, const __nv_bfloat16* __restric
     __nv_bfloat16* dst_base = lane < 16 ? out_k : out_v;
     const unsigned tok_bytes = (unsigned)stride_tok * 2u;      // the launcher checks that this fits
     uint32_t n_chunks_done = 0;                      // chunks this warp has consumed (buffer parity)
+    grid_dependency_wait();
 
     for (long long g = (long long)blockIdx.x * kMergeWarps + warp; g < total_units;
          g += (long long)gridDim.x * kMergeWarps) {
@@ -640,10 +643,10 @@ cudaError_t launch_gather_kept(const void* k, long long stride_tok, long long st
                                int* status, cudaStream_t stream) {
     if (total_kept_rows <= 0) return cudaSuccess;
     const long long blocks = (total_kept_rows + 15) / 16;
-    gather_kept_kernel<<<(unsigned)blocks, 256, 0, stream>>>(
-        (const __nv_bfloat16*)k, stride_tok, stride_head, reqs, n_req, n_kv_heads, T,
-        total_kept_rows, kept_idx, rnorm_all, (__nv_bfloat16*)kept_keys, rnorm_kept, status);
-    return cudaGetLastError();
+    return launch_chained(gather_kept_kernel, dim3((unsigned)blocks), dim3(256), 0, stream,
+                          (const __nv_bfloat16*)k, stride_tok, stride_head, reqs, n_req, n_kv_heads, T,
+                          total_kept_rows, kept_idx, rnorm_all, (__nv_bfloat16*)kept_keys, rnorm_kept,
+                          status);
 }
 
 cudaError_t launch_invert_assignment(const int* assign, const int* kept_idx, const int* evict_idx,
@@ -652,11 +655,9 @@ cudaError_t launch_invert_assignment(const int* assign, const int* kept_idx, con
                                      int4* unit_first, int* slot_cnt, unsigned* sort_a,
                                      unsigned* sort_b, int* status, cudaStream_t stream) {
     dim3 grid(n_kv_heads, n_req);
-    invert_assignment_kernel<<<grid, kInvThreads, 0, stream>>>(assign, kept_idx, evict_idx, sim, reqs,
-                                                               n_kv_heads, T, row_ptr, ent_pos, ent_w,
-                                                               unit_first, slot_cnt, sort_a, sort_b,
-                                                               status);
-    return cudaGetLastError();
+    return launch_chained(invert_assignment_kernel, grid, dim3(kInvThreads), 0, stream, assign, kept_idx,
+                          evict_idx, sim, reqs, n_kv_heads, T, row_ptr, ent_pos, ent_w, unit_first,
+                          slot_cnt, sort_a, sort_b, status);
 }
 
 int merge_warps_per_sm() { return kMergeWarps; }
@@ -674,11 +675,10 @@ cudaError_t launch_merge(const void* k, const void* v, long long stride_tok, lon
     if (err != cudaSuccess) return err;
     long long blocks = (total_units + kMergeWarps - 1) / kMergeWarps;
     if (blocks > num_sms) blocks = num_sms;              // persistent: one CTA per SM
-    merge_kernel<<<(unsigned)blocks, kMergeWarps * 32, smem, stream>>>(
-        (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, stride_tok, stride_head, reqs, n_req,
-        n_kv_heads, T, total_units, row_ptr, ent_pos, ent_w, unit_first, slot_cnt, parts, varlen_output,
-        (__nv_bfloat16*)out_k, (__nv_bfloat16*)out_v, status);
-    return cudaGetLastError();
+    return launch_chained(merge_kernel, dim3((unsigned)blocks), dim3(kMergeWarps * 32), (size_t)smem, stream,
+                          (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, stride_tok, stride_head, reqs,
+                          n_req, n_kv_heads, T, total_units, row_ptr, ent_pos, ent_w, unit_first, slot_cnt,
+                          parts, varlen_output, (__nv_bfloat16*)out_k, (__nv_bfloat16*)out_v, status);
 }
 
 cudaError_t launch_argmax_rows(const float* sim_matrix, const Req* reqs, int n_req,

@@ -126,6 +126,7 @@ select_kernel(const float* __restrict__ scores, const uint8_t* __restrict__ mask
     __shared__ int warp_tot[32][2];
     __shared__ int sh_val[4];
 
+    grid_dependency_wait();
     if ((int)blockIdx.x >= n_select_blocks) {
         key_norms(keys, stride_tok, stride_head, n_kv_heads, T, rnorm_all, (int)blockIdx.x - n_select_blocks,
                   (int)gridDim.x - n_select_blocks);
@@ -284,10 +285,9 @@ cudaError_t launch_select(const float* scores, const uint8_t* mask, const Req* r
         const long long want = (T * n_kv_heads + kSelThreads / 16 - 1) / (kSelThreads / 16);
         n_norm = (int)std::min<long long>(want, n_select < num_sms ? num_sms - n_select : num_sms);
     }
-    select_kernel<<<n_select + n_norm, kSelThreads, 0, stream>>>(
-        scores, mask, reqs, n_select, n_kv_heads, T, kept_idx, evict_idx, rank,
-        (const __nv_bfloat16*)k_for_norms, stride_tok, stride_head, rnorm_all);
-    return cudaGetLastError();
+    return launch_chained(select_kernel, dim3(n_select + n_norm), dim3(kSelThreads), 0, stream,
+                          scores, mask, reqs, n_select, n_kv_heads, T, kept_idx, evict_idx, rank,
+                          (const __nv_bfloat16*)k_for_norms, stride_tok, stride_head, rnorm_all);
 }
 
 }  // namespace lookm

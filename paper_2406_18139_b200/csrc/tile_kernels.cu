@@ -142,6 +142,9 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         sh.abort_flag = 0;
         ptx::fence_mbar_init();
     }
+    // everything above touches only this CTA's shared memory; from here on global memory written
+    // by the kernel before this one is read
+    grid_dependency_wait();
     const Req* tbl = p.reqs;
     if (p.n_req <= kReqCache) {                  // the table is read once per item by every role
         for (int i = threadIdx.x; i < p.n_req * (int)(sizeof(Req) / 4); i += kThreads)
@@ -526,12 +529,12 @@ cudaError_t launch_tile_kernel(int kind, const CUtensorMap& map_a, const CUtenso
 #define LOOKM_LAUNCH(K)                                                                          \
     err = cudaFuncSetAttribute(tile_kernel<K>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem); \
     if (err != cudaSuccess) return err;                                                          \
-    tile_kernel<K><<<grid, kThreads, smem, stream>>>(map_a, map_b, p);
+    err = launch_chained(tile_kernel<K>, dim3(grid), dim3(kThreads), (size_t)smem, stream, map_a, map_b, p);
     if (kind == kSweep1) { LOOKM_LAUNCH(kSweep1) }
     else if (kind == kSweep2) { LOOKM_LAUNCH(kSweep2) }
     else { LOOKM_LAUNCH(kMatch) }
 #undef LOOKM_LAUNCH
-    return cudaGetLastError();
+    return err;
 }
 
 }  // namespace lookm
