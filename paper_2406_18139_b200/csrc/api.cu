@@ -27,7 +27,7 @@ size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 struct Plan {
     int n_req = 0, n_q_heads = 0, n_kv_heads = 0, group = 1;
     long long T = 0, sum_B = 0, sum_E = 0, sum_EB = 0;
-    int max_L = 0, max_E = 0;
+    int max_L = 0, max_E = 0, max_B = 0;
     int n_items[3] = {0, 0, 0};
     long long total_slots = 0;              // n_kv_heads * sum_B
     long long total_units = 0;              // merge work units
@@ -65,6 +65,7 @@ int build_plan(Plan& pl, const lookm_layout* lay, int n_req, const int* cu_seqle
         const int window = windows ? windows[r] : 0;
         const int mode = modes ? modes[r] : 0;
         if (budget <= 0 || window < 0 || mode < 0 || mode > 2) return LOOKM_ERR_INVALID_ARG;
+        if (L - std::min<long long>(budget, L) > kMaxEvictedPerHead) return LOOKM_ERR_UNSUPPORTED;
         Req& q = pl.reqs[r];
         q.tok_begin = (int)begin;
         q.L = (int)L;
@@ -85,6 +86,7 @@ int build_plan(Plan& pl, const lookm_layout* lay, int n_req, const int* cu_seqle
         eb += (long long)q.E * q.B;
         pl.max_L = std::max(pl.max_L, q.L);
         pl.max_E = std::max(pl.max_E, q.E);
+        pl.max_B = std::max(pl.max_B, q.B);
     }
     pl.T = tok;
     pl.sum_B = out;
@@ -341,7 +343,7 @@ int run_merge(const Plan& pl, const lookm_layout* lay, const void* k, const void
     const Req* reqs = at<Req>(ws, pl.o_reqs);
     int* status = at<int>(ws, pl.o_status);
     LOOKM_CUDA(launch_invert_assignment(assign, kept_idx, evict_idx, sim, reqs, pl.n_req, pl.n_kv_heads,
-                                        pl.T, at<int>(ws, pl.o_row_ptr), at<int>(ws, pl.o_members),
+                                        pl.T, pl.max_B, at<int>(ws, pl.o_row_ptr), at<int>(ws, pl.o_members),
                                         at<float>(ws, pl.o_member_w), at<int4>(ws, pl.o_units),
                                         at<int>(ws, pl.o_slot_cnt), at<unsigned>(ws, pl.o_sort_a),
                                         at<unsigned>(ws, pl.o_sort_b), status, st));

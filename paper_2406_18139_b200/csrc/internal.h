@@ -12,6 +12,7 @@ namespace lookm {
 constexpr int kTile = 128;      // tokens per tile on either operand of the tensor-core kernels
 constexpr int kHeadDim = 128;   // only supported head_dim
 constexpr int kMinUnitEntries = 32; // least number of rows in a work unit of the merge kernel
+constexpr int kMaxEvictedPerHead = 2000000;  // the inversion counts a warp's share of them in 16 bits
 constexpr int kMergePartBytes = 2560; // per work unit: two fp32 partial K|V rows and one bf16 K|V row
 
 // One request of the packed batch as the kernels see it (device copy lives in the workspace).
@@ -90,8 +91,8 @@ cudaError_t launch_write_table(const ReqChunk& chunk, int count, Req* dst, cudaS
 
 cudaError_t launch_invert_assignment(const int* assign, const int* kept_idx, const int* evict_idx,
                                      const float* sim, const Req* reqs, int n_req, int n_kv_heads,
-                                     long long T, int* row_ptr, int* ent_pos, float* ent_w,
-                                     int4* unit_first, int* slot_cnt, unsigned* sort_a,
+                                     long long T, int max_slots, int* row_ptr, int* ent_pos,
+                                     float* ent_w, int4* unit_first, int* slot_cnt, unsigned* sort_a,
                                      unsigned* sort_b, int* status, cudaStream_t stream);
 
 int merge_warps_per_sm();

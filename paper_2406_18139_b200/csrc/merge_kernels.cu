@@ -133,6 +133,7 @@ argmax_rows_kernel(const float* __restrict__ sim_matrix, const Req* __restrict__
 // earlier warps.  Keys are packed as (slot << 0) in one array and values in the other.
 // ---------------------------------------------------------------------------------------------
 constexpr int kInvThreads = 1024;
+constexpr int kInvMaxDigitBits = 11;                 // 2048 digit values: 136 KB of counters per CTA
 
 // Second half of the entry list: the kept rows (flagged with the sign bit, weight = member count),
 // for every work unit (unit u of a head covers the entries [u * unit_entries, (u + 1) * unit_entries))
@@ -155,20 +156,31 @@ __device__ __forceinline__ void write_kept_entries(const Req& rq, int h, int n_k
     }
 }
 
-// Lanes of the warp that hold a valid element with the same 8-bit digit as the caller: one ballot
-// per bit (match.any takes a step per distinct value, i.e. up to 32 for well-mixed digits).
-__device__ __forceinline__ unsigned same_digit_lanes(unsigned d, bool valid) {
+// Lanes of the warp that hold a valid element with the same digit as the caller: one ballot per
+// digit bit (match.any takes a step per distinct value, i.e. up to 32 for well-mixed digits).
+__device__ __forceinline__ unsigned same_digit_lanes(unsigned d, bool valid, int dbits) {
     unsigned peers = __ballot_sync(0xffffffffu, valid);
 #pragma unroll
-    for (int b = 0; b < 8; ++b) {
-        const bool bit = (d >> b) & 1u;
-        const unsigned bal = __ballot_sync(0xffffffffu, bit);
-        peers &= bit ? bal : ~bal;
+    for (int b = 0; b < kInvMaxDigitBits; ++b) {
+        if (b < dbits) {
+            const bool bit = (d >> b) & 1u;
+            const unsigned bal = __ballot_sync(0xffffffffu, bit);
+            peers &= bit ? bal : ~bal;
+        }
     }
     return peers;
 }
 
 constexpr int kInvBatch = 8;                         // loop steps whose loads are issued together
+
+// Digits of the sort: the slot index is split into the fewest digits of at most kInvMaxDigitBits
+// bits, all of the same width.  Budgets up to 2048 rows are sorted in ONE pass.
+__host__ __device__ inline void invert_digits(int B, int& n_pass, int& dbits) {
+    int bits = 1;
+    while ((1 << bits) < B) ++bits;
+    n_pass = (bits + kInvMaxDigitBits - 1) / kInvMaxDigitBits;
+    dbits = (bits + n_pass - 1) / n_pass;
+}
 
 __global__ void __launch_bounds__(kInvThreads)
 invert_assignment_kernel(const int* __restrict__ assign, const int* __restrict__ kept_idx,
@@ -178,9 +190,9 @@ invert_assignment_kernel(const int* __restrict__ assign, const int* __restrict__
                          int* __restrict__ ent_pos, float* __restrict__ ent_w,
                          int4* __restrict__ unit_first, int* __restrict__ slot_cnt,
                          unsigned* __restrict__ sort_a, unsigned* __restrict__ sort_b, int* status) {
+    extern __shared__ __align__(16) unsigned char inv_smem[];
+    __shared__ int warp_sums[32];
     grid_dependency_wait();
-    __shared__ int cnt[32][256];                         // [warp][digit]
-    __shared__ int digit_tot[256];
     const Req rq = reqs[blockIdx.y];
     const int h = blockIdx.x;
     const int E = rq.E, B = rq.B;
@@ -202,23 +214,29 @@ invert_assignment_kernel(const int* __restrict__ assign, const int* __restrict__
         write_kept_entries(rq, h, n_kv_heads, B, rp, kept_idx_head, ent, entw, units, cnts, status);
         return;
     }
-    // segment of the list owned by each warp: a multiple of 32 elements
+    // segment of the list owned by each warp: a multiple of 32 elements (at most 65504, so that
+    // the per-warp counts fit 16 bits; the host checks E)
     const int seg = ((E + 32 * 32 - 1) / (32 * 32)) * 32;
     const int s_begin = min(E, warp * seg), s_end = min(E, s_begin + seg);
 
-    int bits = 1;
-    while ((1 << bits) < B) ++bits;
-    const int n_pass = (bits + 7) / 8;
+    int n_pass, dbits;
+    invert_digits(B, n_pass, dbits);
+    const int nd = 1 << dbits;
+    const unsigned dmask = (unsigned)nd - 1u;
+    unsigned short* cnt = reinterpret_cast<unsigned short*>(inv_smem);          // [warp][digit]
+    int* digit_tot = reinterpret_cast<int*>(inv_smem + (size_t)32 * nd * sizeof(unsigned short));
+    const bool single = (n_pass == 1);
 
-    // pass p reads (key, value) from src and writes to dst; pass 0 reads assign directly
+    // pass p reads (key, value) from src and writes to dst; pass 0 reads assign directly.  With a
+    // single pass the sorted position is final, and the entries are written straight away.
     unsigned* key_buf[2] = {sort_a + 2 * ev_base, sort_b + 2 * ev_base};   // [E keys][E values] each
     for (int pass = 0; pass < n_pass; ++pass) {
-        const int shift = pass * 8;
+        const int shift = pass * dbits;
         const unsigned* src_k = pass ? key_buf[(pass - 1) & 1] : nullptr;
         const unsigned* src_v = pass ? key_buf[(pass - 1) & 1] + E : nullptr;
         unsigned* dst_k = key_buf[pass & 1];
         unsigned* dst_v = key_buf[pass & 1] + E;
-        for (int i = threadIdx.x; i < 32 * 256; i += kInvThreads) (&cnt[0][0])[i] = 0;
+        for (int i = threadIdx.x; i < 16 * nd; i += kInvThreads) reinterpret_cast<unsigned*>(cnt)[i] = 0u;
         __syncthreads();
         // count (the loads of kInvBatch steps are issued together: the loop is bound by their latency)
         for (int b0 = s_begin; b0 < s_end; b0 += 32 * kInvBatch) {
@@ -237,46 +255,75 @@ invert_assignment_kernel(const int* __restrict__ assign, const int* __restrict__
                     atomicExch(status, (int)LOOKM_ERR_DEVICE_BAD_INDEX);
                     key[q] = 0u;
                 }
-                const unsigned d = (key[q] >> shift) & 255u;
-                const unsigned peers = same_digit_lanes(d, valid);
-                if (valid && (peers & lt_mask) == 0u) cnt[warp][d] += __popc(peers);
+                const unsigned d = (key[q] >> shift) & dmask;
+                const unsigned peers = same_digit_lanes(d, valid, dbits);
+                if (valid && (peers & lt_mask) == 0u) cnt[warp * nd + d] += (unsigned short)__popc(peers);
                 __syncwarp();
             }
         }
         __syncthreads();
-        // exclusive scan over (digit major, warp minor)
-        if (threadIdx.x < 256) {
+        // exclusive scan over (digit major, warp minor): first over the warps of every digit ...
+        for (int d = threadIdx.x; d < nd; d += kInvThreads) {
             int tot = 0;
-            for (int w = 0; w < 32; ++w) { const int c = cnt[w][threadIdx.x]; cnt[w][threadIdx.x] = tot; tot += c; }
-            digit_tot[threadIdx.x] = tot;
+            for (int w = 0; w < 32; ++w) {
+                const int c = cnt[w * nd + d];
+                cnt[w * nd + d] = (unsigned short)tot;
+                tot += c;
+            }
+            digit_tot[d] = tot;
         }
         __syncthreads();
-        if (threadIdx.x < 32) {                          // exclusive scan of the 256 totals: 8 per lane
-            int c[8], mine = 0;
-#pragma unroll
-            for (int q = 0; q < 8; ++q) { c[q] = digit_tot[8 * lane + q]; mine += c[q]; }
-            int incl = mine;
+        // ... then over the digit totals (two digits per thread; nd <= 2 * kInvThreads)
+        {
+            const int d0 = 2 * threadIdx.x;
+            const int a = d0 < nd ? digit_tot[d0] : 0;
+            const int b = d0 + 1 < nd ? digit_tot[d0 + 1] : 0;
+            int incl = a + b;
 #pragma unroll
             for (int o = 1; o < 32; o <<= 1) {
                 const int x = __shfl_up_sync(0xffffffffu, incl, o);
                 if (lane >= o) incl += x;
             }
-            int run = incl - mine;
+            if (lane == 31) warp_sums[warp] = incl;
+            __syncthreads();
+            if (warp == 0) {
+                int ws = warp_sums[lane];
 #pragma unroll
-            for (int q = 0; q < 8; ++q) { digit_tot[8 * lane + q] = run; run += c[q]; }
+                for (int o = 1; o < 32; o <<= 1) {
+                    const int x = __shfl_up_sync(0xffffffffu, ws, o);
+                    if (lane >= o) ws += x;
+                }
+                warp_sums[lane] = ws;
+            }
+            __syncthreads();
+            const int base = (warp ? warp_sums[warp - 1] : 0) + incl - (a + b);
+            if (d0 < nd) digit_tot[d0] = base;
+            if (d0 + 1 < nd) digit_tot[d0 + 1] = base + a;
         }
         __syncthreads();
+        if (single) {
+            // row boundaries: row_ptr[c] = first sorted index whose slot is >= c
+            for (int c = threadIdx.x; c <= B; c += kInvThreads) rp[c] = c < nd ? digit_tot[c] : E;
+        }
         // scatter
         for (int b0 = s_begin; b0 < s_end; b0 += 32 * kInvBatch) {
             unsigned key[kInvBatch], val[kInvBatch];
+            int pe[kInvBatch];
+            float w[kInvBatch];
 #pragma unroll
             for (int q = 0; q < kInvBatch; ++q) {
                 const int i = b0 + q * 32 + lane;
                 key[q] = 0u;
                 val[q] = (unsigned)i;
+                pe[q] = 0;
+                w[q] = 1.0f;
                 if (i < s_end) {
                     if (pass) { key[q] = src_k[i]; val[q] = src_v[i]; }
                     else key[q] = (unsigned)assign[ev_base + i];
+                    if (single) {
+                        pe[q] = evict_idx[ev_base + i];
+                        if (weighted) w[q] = sim[ev_base + i];
+                    }
                 }
             }
 #pragma unroll
@@ -284,52 +331,63 @@ invert_assignment_kernel(const int* __restrict__ assign, const int* __restrict__
                 const int i = b0 + q * 32 + lane;
                 const bool valid = i < s_end;
                 if (!pass && key[q] >= (unsigned)B) key[q] = 0u;
-                const unsigned d = (key[q] >> shift) & 255u;
-                const unsigned peers = same_digit_lanes(d, valid);
+                const unsigned d = (key[q] >> shift) & dmask;
+                const unsigned peers = same_digit_lanes(d, valid, dbits);
                 int off = 0;
-                if (valid) off = digit_tot[d] + cnt[warp][d] + __popc(peers & lt_mask);
+                if (valid) off = digit_tot[d] + cnt[warp * nd + d] + __popc(peers & lt_mask);
                 __syncwarp();
-                if (valid && (peers & lt_mask) == 0u) cnt[warp][d] += __popc(peers);
+                if (valid && (peers & lt_mask) == 0u) cnt[warp * nd + d] += (unsigned short)__popc(peers);
                 __syncwarp();
-                if (valid) { dst_k[off] = key[q]; dst_v[off] = val[q]; }
+                if (valid) {
+                    if (single) {
+                        if (pe[q] < 0 || pe[q] >= rq.L) { atomicExch(status, (int)LOOKM_ERR_DEVICE_BAD_INDEX); pe[q] = 0; }
+                        ent[off + (int)key[q] + 1] = pe[q];      // sits after key + 1 kept rows
+                        entw[off + (int)key[q] + 1] = w[q];
+                    } else {
+                        dst_k[off] = key[q];
+                        dst_v[off] = val[q];
+                    }
+                }
             }
         }
         __syncthreads();
     }
-    const unsigned* fin_k = key_buf[(n_pass - 1) & 1];
-    const unsigned* fin_v = fin_k + E;
-    // member entries and the row boundaries: row_ptr[c] = first sorted index whose slot is >= c
-    for (int i0 = threadIdx.x; i0 < E; i0 += kInvThreads * kInvBatch) {
-        int e[kInvBatch], cur[kInvBatch], prev[kInvBatch], pe[kInvBatch];
-        float w[kInvBatch];
+    if (!single) {
+        const unsigned* fin_k = key_buf[(n_pass - 1) & 1];
+        const unsigned* fin_v = fin_k + E;
+        // member entries and the row boundaries: row_ptr[c] = first sorted index whose slot is >= c
+        for (int i0 = threadIdx.x; i0 < E; i0 += kInvThreads * kInvBatch) {
+            int e[kInvBatch], cur[kInvBatch], prev[kInvBatch], pe[kInvBatch];
+            float w[kInvBatch];
 #pragma unroll
-        for (int q = 0; q < kInvBatch; ++q) {
-            const int i = i0 + q * kInvThreads;
-            e[q] = 0; cur[q] = 0; prev[q] = -1;
-            if (i < E) {
-                e[q] = (int)fin_v[i];
-                cur[q] = (int)fin_k[i];
-                if (i) prev[q] = (int)fin_k[i - 1];
+            for (int q = 0; q < kInvBatch; ++q) {
+                const int i = i0 + q * kInvThreads;
+                e[q] = 0; cur[q] = 0; prev[q] = -1;
+                if (i < E) {
+                    e[q] = (int)fin_v[i];
+                    cur[q] = (int)fin_k[i];
+                    if (i) prev[q] = (int)fin_k[i - 1];
+                }
             }
-        }
 #pragma unroll
-        for (int q = 0; q < kInvBatch; ++q) {
-            const int i = i0 + q * kInvThreads;
-            pe[q] = 0; w[q] = 1.0f;
-            if (i < E) {
-                pe[q] = evict_idx[ev_base + e[q]];
-                if (weighted) w[q] = sim[ev_base + e[q]];
+            for (int q = 0; q < kInvBatch; ++q) {
+                const int i = i0 + q * kInvThreads;
+                pe[q] = 0; w[q] = 1.0f;
+                if (i < E) {
+                    pe[q] = evict_idx[ev_base + e[q]];
+                    if (weighted) w[q] = sim[ev_base + e[q]];
+                }
             }
-        }
 #pragma unroll
-        for (int q = 0; q < kInvBatch; ++q) {
-            const int i = i0 + q * kInvThreads;
-            if (i >= E) continue;
-            if (pe[q] < 0 || pe[q] >= rq.L) { atomicExch(status, (int)LOOKM_ERR_DEVICE_BAD_INDEX); pe[q] = 0; }
-            ent[i + cur[q] + 1] = pe[q];                 // i-th member sits after cur + 1 kept rows
-            entw[i + cur[q] + 1] = w[q];
-            for (int c = prev[q] + 1; c <= cur[q]; ++c) rp[c] = i;
-            if (i == E - 1) for (int c = cur[q] + 1; c <= B; ++c) rp[c] = E;
+            for (int q = 0; q < kInvBatch; ++q) {
+                const int i = i0 + q * kInvThreads;
+                if (i >= E) continue;
+                if (pe[q] < 0 || pe[q] >= rq.L) { atomicExch(status, (int)LOOKM_ERR_DEVICE_BAD_INDEX); pe[q] = 0; }
+                ent[i + cur[q] + 1] = pe[q];             // i-th member sits after cur + 1 kept rows
+                entw[i + cur[q] + 1] = w[q];
+                for (int c = prev[q] + 1; c <= cur[q]; ++c) rp[c] = i;
+                if (i == E - 1) for (int c = cur[q] + 1; c <= B; ++c) rp[c] = E;
+            }
         }
     }
     __syncthreads();
@@ -651,11 +709,19 @@ cudaError_t launch_gather_kept(const void* k, long long stride_tok, long long st
 
 cudaError_t launch_invert_assignment(const int* assign, const int* kept_idx, const int* evict_idx,
                                      const float* sim, const Req* reqs, int n_req, int n_kv_heads,
-                                     long long T, int* row_ptr, int* ent_pos, float* ent_w,
-                                     int4* unit_first, int* slot_cnt, unsigned* sort_a,
+                                     long long T, int max_slots, int* row_ptr, int* ent_pos,
+                                     float* ent_w, int4* unit_first, int* slot_cnt, unsigned* sort_a,
                                      unsigned* sort_b, int* status, cudaStream_t stream) {
+    // counters of the widest digit any request of the call needs: 32 warps x 2^dbits 16-bit counts
+    // and 2^dbits totals
+    int n_pass, dbits;
+    invert_digits(max_slots > 0 ? max_slots : 1, n_pass, dbits);
+    const size_t smem = ((size_t)32 * sizeof(unsigned short) + sizeof(int)) << dbits;
+    cudaError_t err = cudaFuncSetAttribute(invert_assignment_kernel,
+                                           cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (err != cudaSuccess) return err;
     dim3 grid(n_kv_heads, n_req);
-    return launch_chained(invert_assignment_kernel, grid, dim3(kInvThreads), 0, stream, assign, kept_idx,
+    return launch_chained(invert_assignment_kernel, grid, dim3(kInvThreads), smem, stream, assign, kept_idx,
                           evict_idx, sim, reqs, n_kv_heads, T, row_ptr, ent_pos, ent_w, unit_first,
                           slot_cnt, sort_a, sort_b, status);
 }
