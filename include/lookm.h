@@ -46,8 +46,7 @@ extern "C" {
 typedef enum {
     LOOKM_OK = 0,
     LOOKM_ERR_INVALID_ARG = 1,
-    LOOKM_ERR_UNSUPPORTED = 2,        /* e.g. head_dim != 128, a device that is not sm_100, or a request
-                                         that evicts more than 2,000,000 tokens */
+    LOOKM_ERR_UNSUPPORTED = 2,        /* e.g. head_dim != 128, or a device that is not sm_100 */
     LOOKM_ERR_WORKSPACE_TOO_SMALL = 3,
     LOOKM_ERR_CUDA = 4,               /* a CUDA runtime/driver call failed */
     LOOKM_ERR_DEVICE_TIMEOUT = 5,     /* a bounded device-side wait expired */

@@ -65,7 +65,6 @@ int build_plan(Plan& pl, const lookm_layout* lay, int n_req, const int* cu_seqle
         const int window = windows ? windows[r] : 0;
         const int mode = modes ? modes[r] : 0;
         if (budget <= 0 || window < 0 || mode < 0 || mode > 2) return LOOKM_ERR_INVALID_ARG;
-        if (L - std::min<long long>(budget, L) > kMaxEvictedPerHead) return LOOKM_ERR_UNSUPPORTED;
         Req& q = pl.reqs[r];
         q.tok_begin = (int)begin;
         q.L = (int)L;
@@ -342,8 +341,16 @@ int run_merge(const Plan& pl, const lookm_layout* lay, const void* k, const void
               int varlen_output, void* out_k, void* out_v, void* ws, cudaStream_t st) {
     const Req* reqs = at<Req>(ws, pl.o_reqs);
     int* status = at<int>(ws, pl.o_status);
+    // counter width and widest digit over the requests of the call
+    const bool wide = pl.max_E > kInvWideCountsAbove;
+    int digit_bits = 1;
+    for (const Req& r : pl.reqs) {
+        int n_pass, dbits;
+        invert_digits(r.B, wide ? kInvDigitBits32 : kInvDigitBits16, n_pass, dbits);
+        digit_bits = std::max(digit_bits, dbits);
+    }
     LOOKM_CUDA(launch_invert_assignment(assign, kept_idx, evict_idx, sim, reqs, pl.n_req, pl.n_kv_heads,
-                                        pl.T, pl.max_B, at<int>(ws, pl.o_row_ptr), at<int>(ws, pl.o_members),
+                                        pl.T, wide, digit_bits, at<int>(ws, pl.o_row_ptr), at<int>(ws, pl.o_members),
                                         at<float>(ws, pl.o_member_w), at<int4>(ws, pl.o_units),
                                         at<int>(ws, pl.o_slot_cnt), at<unsigned>(ws, pl.o_sort_a),
                                         at<unsigned>(ws, pl.o_sort_b), status, st));

@@ -12,7 +12,21 @@ namespace lookm {
 constexpr int kTile = 128;      // tokens per tile on either operand of the tensor-core kernels
 constexpr int kHeadDim = 128;   // only supported head_dim
 constexpr int kMinUnitEntries = 32; // least number of rows in a work unit of the merge kernel
-constexpr int kMaxEvictedPerHead = 2000000;  // the inversion counts a warp's share of them in 16 bits
+// Digits of the assignment inversion's radix sort: the slot index of a request with B kept rows is
+// split into the fewest digits of at most max_bits bits, all of the same width (so B <= 2^max_bits
+// is sorted in one pass).  16-bit counters allow 11-bit digits, 32-bit counters 10-bit ones.
+constexpr int kInvDigitBits16 = 11;
+constexpr int kInvDigitBits32 = 10;
+constexpr int kInvWideCountsAbove = 65535;   // evicted tokens per head beyond which counts need 32 bits
+#ifdef __CUDACC__
+__host__ __device__
+#endif
+inline void invert_digits(int B, int max_bits, int& n_pass, int& dbits) {
+    int bits = 1;
+    while ((1 << bits) < B) ++bits;
+    n_pass = (bits + max_bits - 1) / max_bits;
+    dbits = (bits + n_pass - 1) / n_pass;
+}
 constexpr int kMergePartBytes = 2560; // per work unit: two fp32 partial K|V rows and one bf16 K|V row
 
 // One request of the packed batch as the kernels see it (device copy lives in the workspace).
@@ -91,9 +105,10 @@ cudaError_t launch_write_table(const ReqChunk& chunk, int count, Req* dst, cudaS
 
 cudaError_t launch_invert_assignment(const int* assign, const int* kept_idx, const int* evict_idx,
                                      const float* sim, const Req* reqs, int n_req, int n_kv_heads,
-                                     long long T, int max_slots, int* row_ptr, int* ent_pos,
-                                     float* ent_w, int4* unit_first, int* slot_cnt, unsigned* sort_a,
-                                     unsigned* sort_b, int* status, cudaStream_t stream);
+                                     long long T, bool wide_counts, int digit_bits, int* row_ptr,
+                                     int* ent_pos, float* ent_w, int4* unit_first, int* slot_cnt,
+                                     unsigned* sort_a, unsigned* sort_b, int* status,
+                                     cudaStream_t stream);
 
 int merge_warps_per_sm();
 

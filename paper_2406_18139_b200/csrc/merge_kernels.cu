@@ -133,7 +133,6 @@ argmax_rows_kernel(const float* __restrict__ sim_matrix, const Req* __restrict__
 // earlier warps.  Keys are packed as (slot << 0) in one array and values in the other.
 // ---------------------------------------------------------------------------------------------
 constexpr int kInvThreads = 1024;
-constexpr int kInvMaxDigitBits = 11;                 // 2048 digit values: 136 KB of counters per CTA
 
 // Second half of the entry list: the kept rows (flagged with the sign bit, weight = member count),
 // for every work unit (unit u of a head covers the entries [u * unit_entries, (u + 1) * unit_entries))
@@ -161,7 +160,7 @@ __device__ __forceinline__ void write_kept_entries(const Req& rq, int h, int n_k
 __device__ __forceinline__ unsigned same_digit_lanes(unsigned d, bool valid, int dbits) {
     unsigned peers = __ballot_sync(0xffffffffu, valid);
 #pragma unroll
-    for (int b = 0; b < kInvMaxDigitBits; ++b) {
+    for (int b = 0; b < kInvDigitBits16; ++b) {
         if (b < dbits) {
             const bool bit = (d >> b) & 1u;
             const unsigned bal = __ballot_sync(0xffffffffu, bit);
@@ -173,15 +172,10 @@ __device__ __forceinline__ unsigned same_digit_lanes(unsigned d, bool valid, int
 
 constexpr int kInvBatch = 8;                         // loop steps whose loads are issued together
 
-// Digits of the sort: the slot index is split into the fewest digits of at most kInvMaxDigitBits
-// bits, all of the same width.  Budgets up to 2048 rows are sorted in ONE pass.
-__host__ __device__ inline void invert_digits(int B, int& n_pass, int& dbits) {
-    int bits = 1;
-    while ((1 << bits) < B) ++bits;
-    n_pass = (bits + kInvMaxDigitBits - 1) / kInvMaxDigitBits;
-    dbits = (bits + n_pass - 1) / n_pass;
-}
-
+// CountT / kMaxBits: 16-bit counters with digits of up to 11 bits when no request of the call evicts
+// more than 65535 tokens per head (every count and prefix then fits), else 32-bit counters with
+// digits of up to 10 bits; either way at most 136 KB of counters per CTA.
+template <typename CountT, int kMaxBits>
 __global__ void __launch_bounds__(kInvThreads)
 invert_assignment_kernel(const int* __restrict__ assign, const int* __restrict__ kept_idx,
                          const int* __restrict__ evict_idx,
@@ -214,17 +208,16 @@ invert_assignment_kernel(const int* __restrict__ assign, const int* __restrict__
         write_kept_entries(rq, h, n_kv_heads, B, rp, kept_idx_head, ent, entw, units, cnts, status);
         return;
     }
-    // segment of the list owned by each warp: a multiple of 32 elements (at most 65504, so that
-    // the per-warp counts fit 16 bits; the host checks E)
+    // segment of the list owned by each warp: a multiple of 32 elements
     const int seg = ((E + 32 * 32 - 1) / (32 * 32)) * 32;
     const int s_begin = min(E, warp * seg), s_end = min(E, s_begin + seg);
 
     int n_pass, dbits;
-    invert_digits(B, n_pass, dbits);
+    invert_digits(B, kMaxBits, n_pass, dbits);
     const int nd = 1 << dbits;
     const unsigned dmask = (unsigned)nd - 1u;
-    unsigned short* cnt = reinterpret_cast<unsigned short*>(inv_smem);          // [warp][digit]
-    int* digit_tot = reinterpret_cast<int*>(inv_smem + (size_t)32 * nd * sizeof(unsigned short));
+    CountT* cnt = reinterpret_cast<CountT*>(inv_smem);                          // [warp][digit]
+    int* digit_tot = reinterpret_cast<int*>(inv_smem + (size_t)32 * nd * sizeof(CountT));
     const bool single = (n_pass == 1);
 
     // pass p reads (key, value) from src and writes to dst; pass 0 reads assign directly.  With a
@@ -236,7 +229,8 @@ invert_assignment_kernel(const int* __restrict__ assign, const int* __restrict__
         const unsigned* src_v = pass ? key_buf[(pass - 1) & 1] + E : nullptr;
         unsigned* dst_k = key_buf[pass & 1];
         unsigned* dst_v = key_buf[pass & 1] + E;
-        for (int i = threadIdx.x; i < 16 * nd; i += kInvThreads) reinterpret_cast<unsigned*>(cnt)[i] = 0u;
+        for (int i = threadIdx.x; i < (int)(32 * sizeof(CountT) / 4) * nd; i += kInvThreads)
+            reinterpret_cast<unsigned*>(cnt)[i] = 0u;
         __syncthreads();
         // count (the loads of kInvBatch steps are issued together: the loop is bound by their latency)
         for (int b0 = s_begin; b0 < s_end; b0 += 32 * kInvBatch) {
@@ -257,7 +251,7 @@ invert_assignment_kernel(const int* __restrict__ assign, const int* __restrict__
                 }
                 const unsigned d = (key[q] >> shift) & dmask;
                 const unsigned peers = same_digit_lanes(d, valid, dbits);
-                if (valid && (peers & lt_mask) == 0u) cnt[warp * nd + d] += (unsigned short)__popc(peers);
+                if (valid && (peers & lt_mask) == 0u) cnt[warp * nd + d] += (CountT)__popc(peers);
                 __syncwarp();
             }
         }
@@ -267,7 +261,7 @@ invert_assignment_kernel(const int* __restrict__ assign, const int* __restrict__
             int tot = 0;
             for (int w = 0; w < 32; ++w) {
                 const int c = cnt[w * nd + d];
-                cnt[w * nd + d] = (unsigned short)tot;
+                cnt[w * nd + d] = (CountT)tot;
                 tot += c;
             }
             digit_tot[d] = tot;
@@ -336,7 +330,7 @@ invert_assignment_kernel(const int* __restrict__ assign, const int* __restrict__
                 int off = 0;
                 if (valid) off = digit_tot[d] + cnt[warp * nd + d] + __popc(peers & lt_mask);
                 __syncwarp();
-                if (valid && (peers & lt_mask) == 0u) cnt[warp * nd + d] += (unsigned short)__popc(peers);
+                if (valid && (peers & lt_mask) == 0u) cnt[warp * nd + d] += (CountT)__popc(peers);
                 __syncwarp();
                 if (valid) {
                     if (single) {
@@ -709,21 +703,27 @@ cudaError_t launch_gather_kept(const void* k, long long stride_tok, long long st
 
 cudaError_t launch_invert_assignment(const int* assign, const int* kept_idx, const int* evict_idx,
                                      const float* sim, const Req* reqs, int n_req, int n_kv_heads,
-                                     long long T, int max_slots, int* row_ptr, int* ent_pos,
-                                     float* ent_w, int4* unit_first, int* slot_cnt, unsigned* sort_a,
-                                     unsigned* sort_b, int* status, cudaStream_t stream) {
-    // counters of the widest digit any request of the call needs: 32 warps x 2^dbits 16-bit counts
-    // and 2^dbits totals
-    int n_pass, dbits;
-    invert_digits(max_slots > 0 ? max_slots : 1, n_pass, dbits);
-    const size_t smem = ((size_t)32 * sizeof(unsigned short) + sizeof(int)) << dbits;
-    cudaError_t err = cudaFuncSetAttribute(invert_assignment_kernel,
-                                           cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (err != cudaSuccess) return err;
+                                     long long T, bool wide_counts, int digit_bits, int* row_ptr,
+                                     int* ent_pos, float* ent_w, int4* unit_first, int* slot_cnt,
+                                     unsigned* sort_a, unsigned* sort_b, int* status,
+                                     cudaStream_t stream) {
+    // counters of the widest digit any request of the call needs: 32 warps x 2^digit_bits counts
+    // and 2^digit_bits totals
+    const size_t smem = ((size_t)32 * (wide_counts ? sizeof(unsigned) : sizeof(unsigned short)) + sizeof(int))
+                        << digit_bits;
     dim3 grid(n_kv_heads, n_req);
-    return launch_chained(invert_assignment_kernel, grid, dim3(kInvThreads), smem, stream, assign, kept_idx,
-                          evict_idx, sim, reqs, n_kv_heads, T, row_ptr, ent_pos, ent_w, unit_first,
-                          slot_cnt, sort_a, sort_b, status);
+    cudaError_t err;
+#define LOOKM_LAUNCH_INVERT(CT, BITS)                                                               \
+    err = cudaFuncSetAttribute(invert_assignment_kernel<CT, BITS>,                                  \
+                               cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);             \
+    if (err != cudaSuccess) return err;                                                             \
+    err = launch_chained(invert_assignment_kernel<CT, BITS>, grid, dim3(kInvThreads), smem, stream, \
+                         assign, kept_idx, evict_idx, sim, reqs, n_kv_heads, T, row_ptr, ent_pos,   \
+                         ent_w, unit_first, slot_cnt, sort_a, sort_b, status);
+    if (wide_counts) { LOOKM_LAUNCH_INVERT(unsigned, kInvDigitBits32) }
+    else { LOOKM_LAUNCH_INVERT(unsigned short, kInvDigitBits16) }
+#undef LOOKM_LAUNCH_INVERT
+    return err;
 }
 
 int merge_warps_per_sm() { return kMergeWarps; }

@@ -317,6 +317,33 @@ def test_merge_packed_batch_with_slots_spread_over_many_work_units(B):
         assert np.array_equal(gk[out_cu[r] + 1, h], kr[a[1], h].astype(np.float64))   # no members: copied
 
 
+def test_merge_long_request_with_one_huge_slot(B):
+    """70,000 tokens, 300 kept, 66,000 of the evicted rows in one slot: the inversion has to count
+    past 16 bits and the merge sums that slot from hundreds of work units."""
+    import torch
+    L, budget, mode = 70000, 300, 2
+    w = synth.tiny(L, 1, 1, budget, 8, mode, seed=31)
+    (q, k, v), (qf, kf, vf), mask, _ = _tensors(w)
+    E = L - budget
+    kept = np.sort(np.unique(synth.uniform_int(synth.stream_key(130), 4 * budget, 0, L - 1))[:budget]).astype(np.int32)
+    assert len(kept) == budget
+    ev = np.setdiff1d(np.arange(L, dtype=np.int32), kept)
+    asg = synth.uniform_int(synth.stream_key(131), E, 0, budget - 1).astype(np.int32)
+    asg[1000:67000] = 17
+    sim = np.clip(synth.normal(synth.stream_key(132), E) * 0.4, -1, 1).astype(np.float32)
+    dev = lambda x: torch.from_numpy(x).cuda()
+    out_k = torch.zeros(1, budget, 128, dtype=torch.bfloat16, device="cuda")
+    out_v = torch.zeros_like(out_k)
+    lay = B.make_layout(None, k)
+    ws = B.alloc_workspace(lay, [L])
+    B.check(B.lookm_merge(k, v, dev(kept), dev(ev), dev(asg), dev(sim), [0, L], [budget], [mode], lay,
+                          0, out_k, out_v, ws))
+    assert B.lookm_device_status(ws) == B.OK
+    rk = orc.merge(kf, 0, kept, ev, asg, sim.astype(np.float64), mode)
+    rv = orc.merge(vf, 0, kept, ev, asg, sim.astype(np.float64), mode)
+    assert merged_close(bf16_to_np(out_k)[0], rk).all() and merged_close(bf16_to_np(out_v)[0], rv).all()
+
+
 def test_merge_single_kept_token_and_bad_index_status(B):
     import torch
     L = 700
