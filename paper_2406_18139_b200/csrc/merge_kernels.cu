@@ -219,6 +219,13 @@ invert_assignment_kernel(const int* __restrict__ assign, const int* __restrict__
     CountT* cnt = reinterpret_cast<CountT*>(inv_smem);                          // [warp][digit]
     int* digit_tot = reinterpret_cast<int*>(inv_smem + (size_t)32 * nd * sizeof(CountT));
     const bool single = (n_pass == 1);
+    // One pass over a segment of at most kInvBatch steps per warp: the count phase already knows
+    // every element's rank among the equal slots of its warp, so the scatter phase needs neither
+    // the ballots nor the running counts again.
+    const bool keep_ranks = single && seg <= 32 * kInvBatch;
+    int local_rank[kInvBatch];
+#pragma unroll
+    for (int q = 0; q < kInvBatch; ++q) local_rank[q] = 0;
 
     // pass p reads (key, value) from src and writes to dst; pass 0 reads assign directly.  With a
     // single pass the sorted position is final, and the entries are written straight away.
@@ -251,6 +258,10 @@ invert_assignment_kernel(const int* __restrict__ assign, const int* __restrict__
                 }
                 const unsigned d = (key[q] >> shift) & dmask;
                 const unsigned peers = same_digit_lanes(d, valid, dbits);
+                if (keep_ranks) {
+                    local_rank[q] = valid ? (int)cnt[warp * nd + d] + __popc(peers & lt_mask) : 0;
+                    __syncwarp();
+                }
                 if (valid && (peers & lt_mask) == 0u) cnt[warp * nd + d] += (CountT)__popc(peers);
                 __syncwarp();
             }
@@ -326,12 +337,16 @@ invert_assignment_kernel(const int* __restrict__ assign, const int* __restrict__
                 const bool valid = i < s_end;
                 if (!pass && key[q] >= (unsigned)B) key[q] = 0u;
                 const unsigned d = (key[q] >> shift) & dmask;
-                const unsigned peers = same_digit_lanes(d, valid, dbits);
                 int off = 0;
-                if (valid) off = digit_tot[d] + cnt[warp * nd + d] + __popc(peers & lt_mask);
-                __syncwarp();
-                if (valid && (peers & lt_mask) == 0u) cnt[warp * nd + d] += (CountT)__popc(peers);
-                __syncwarp();
+                if (keep_ranks) {
+                    if (valid) off = digit_tot[d] + (int)cnt[warp * nd + d] + local_rank[q];
+                } else {
+                    const unsigned peers = same_digit_lanes(d, valid, dbits);
+                    if (valid) off = digit_tot[d] + (int)cnt[warp * nd + d] + __popc(peers & lt_mask);
+                    __syncwarp();
+                    if (valid && (peers & lt_mask) == 0u) cnt[warp * nd + d] += (CountT)__popc(peers);
+                    __syncwarp();
+                }
                 if (valid) {
                     if (single) {
                         if (pe[q] < 0 || pe[q] >= rq.L) { atomicExch(status, (int)LOOKM_ERR_DEVICE_BAD_INDEX); pe[q] = 0; }
