@@ -23,6 +23,7 @@ namespace {
 
 constexpr int kSelThreads = 1024;
 constexpr int kPerThread = 8;
+constexpr int kKeyCache = 8;                         // candidates per thread whose keys stay in registers
 
 __device__ __forceinline__ unsigned order_key(float s) {
     unsigned b = __float_as_uint(s);
@@ -139,9 +140,24 @@ select_kernel(const float* __restrict__ scores, const uint8_t* __restrict__ mask
     const int L = rq.L, B = rq.B, M = rq.M;
     const int N = B - M, nc = L - M;
 
-    // ---- count text candidates ---------------------------------------------------------------
+    // ---- count text candidates; the first kKeyCache * 1024 candidates' keys and classes stay in
+    // registers for the radix passes (the loads would otherwise be repeated in every pass, and
+    // each round trip is paid in full by this latency-bound kernel) -----------------------------
     int cnt = 0;
-    for (int j = threadIdx.x; j < nc; j += kSelThreads) cnt += (msk[j] == 0);
+    unsigned ckey[kKeyCache];
+    unsigned cimg = 0u;                                  // bit q: cached candidate q is an image token
+#pragma unroll
+    for (int q = 0; q < kKeyCache; ++q) {
+        const int j = threadIdx.x + q * kSelThreads;
+        ckey[q] = 0u;
+        if (j < nc) {
+            const bool img = msk[j] != 0;
+            ckey[q] = order_key(s[j]);
+            cimg |= (img ? 1u : 0u) << q;
+            cnt += !img;
+        }
+    }
+    for (int j = threadIdx.x + kKeyCache * kSelThreads; j < nc; j += kSelThreads) cnt += (msk[j] == 0);
     {
         int e0, e1, t0, t1;
         block_scan2(cnt, 0, e0, e1, t0, t1, warp_tot);
@@ -164,7 +180,13 @@ select_kernel(const float* __restrict__ scores, const uint8_t* __restrict__ mask
         for (int shift = 24; shift >= 0; shift -= 8) {
             for (int i = threadIdx.x; i < 256; i += kSelThreads) hist[i] = 0;
             __syncthreads();
-            for (int j = threadIdx.x; j < nc; j += kSelThreads) {
+#pragma unroll
+            for (int q = 0; q < kKeyCache; ++q) {
+                const int j = threadIdx.x + q * kSelThreads;
+                if (j < nc && ((cimg >> q) & 1u) == (unsigned)sel_cls && (ckey[q] & pmask) == prefix)
+                    atomicAdd(&hist[(ckey[q] >> shift) & 255u], 1);
+            }
+            for (int j = threadIdx.x + kKeyCache * kSelThreads; j < nc; j += kSelThreads) {
                 if ((msk[j] != 0) == (sel_cls != 0)) {
                     const unsigned key = order_key(s[j]);
                     if ((key & pmask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1);
