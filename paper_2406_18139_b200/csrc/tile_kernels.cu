@@ -315,7 +315,7 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                 if (KIND == kMatch) {
                     // running arg-max of dot / |kept key| over kept slots, 16 columns at a time with
                     // the next 16 already on their way from TMEM (a load takes about as long as
-                    // the work on 32 columns).  The maximum of 8 columns is taken first; only when it
+                    // the work on 32 columns).  The maximum of the 16 is taken first; only when it
                     // beats the running best is its first column looked up, so a strict comparison
                     // in ascending slot order keeps the lowest slot.
                     auto columns16 = [&](const uint32_t (&r)[16], int c0) {
@@ -334,18 +334,18 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                             for (int c = 0; c < 16; ++c)
                                 if (c0 + c >= col_limit) v[c] = -INFINITY;
                         }
+                        const float m0 = ptx::fmax3(v[0], v[1], v[2]);
+                        const float m1 = ptx::fmax3(v[3], v[4], v[5]);
+                        const float m2 = ptx::fmax3(v[6], v[7], v[8]);
+                        const float m3 = ptx::fmax3(v[9], v[10], v[11]);
+                        const float m4 = ptx::fmax3(v[12], v[13], v[14]);
+                        const float mx = fmaxf(ptx::fmax3(m0, m1, m2), ptx::fmax3(m3, m4, v[15]));
+                        if (mx > best) {
+                            best = mx;
+                            int idx = 15;
 #pragma unroll
-                        for (int h8 = 0; h8 < 2; ++h8) {     // two blocks of 8 columns
-                            const float* u = v + 8 * h8;
-                            const float mx = ptx::fmax3(ptx::fmax3(u[0], u[1], u[2]), ptx::fmax3(u[3], u[4], u[5]),
-                                                        fmaxf(u[6], u[7]));
-                            if (mx > best) {
-                                best = mx;
-                                int idx = 7;
-#pragma unroll
-                                for (int c = 6; c >= 0; --c) if (u[c] == mx) idx = c;
-                                best_slot = t * kTile + c0 + 8 * h8 + idx;
-                            }
+                            for (int c = 14; c >= 0; --c) if (v[c] == mx) idx = c;
+                            best_slot = t * kTile + c0 + idx;
                         }
                     };
                     uint32_t ra[16], rb[16];
