@@ -285,6 +285,8 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
             float acc0 = 0.f, acc1 = 0.f, acc2 = 0.f, acc3 = 0.f;   // sweep 2
             float best = -INFINITY;                          // match
             int best_slot = 0x7fffffff;
+            float lse_next = INFINITY;                       // sweep 2: value for this group's next tile
+            bool have_next = false;
 
             for (int t = 0; t < it.nt; ++t, ++gb) {
                 if ((int)(gb % kGroups) != wg) continue;
@@ -299,7 +301,15 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                     const int qh = it.head * p.group + t % p.group;
                     const int i = ib * kTile + row;          // query column staged by this thread
                     float v = INFINITY;                      // +inf turns the probability into 0
-                    if (i < it.L) v = p.lse[(long long)qh * p.T + it.tok_begin + i] * kLog2e;
+                    if (have_next) v = lse_next;
+                    else if (i < it.L) v = p.lse[(long long)qh * p.T + it.tok_begin + i] * kLog2e;
+                    // without query groups the group's next tile of the item is four query blocks
+                    // further on: fetch its value now, a tile ahead of its use
+                    have_next = (p.group == 1) && (t + kGroups < it.nt);
+                    if (have_next) {
+                        const int i4 = i + kGroups * kTile;
+                        lse_next = (i4 < it.L) ? p.lse[(long long)qh * p.T + it.tok_begin + i4] * kLog2e : INFINITY;
+                    }
                     side[row] = v;
                     diag = (ib == it.blk);
                     ptx::named_barrier_sync(1 + wg, 128);
