@@ -46,7 +46,7 @@ constexpr float kLn2 = 0.6931471805599453f;
 struct __align__(1024) Shared {
     uint8_t a[2][kTileBytes];                    // stationary tiles (double-buffered across items)
     uint8_t b[kStages][kTileBytes];              // streamed tiles
-    float side[kGroups * 4][kTile];              // per epilogue warp: column data of its current tile
+    float side[kGroups][2][kTile];               // per epilogue group, double-buffered column data
     float comb[2][kGroups][2][kTile];            // partial results of the groups, double-buffered
     Req reqs[kReqCache];                         // copy of the request table (when it fits)
     unsigned long long a_full[2], a_empty[2];
@@ -285,57 +285,39 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
             float acc0 = 0.f, acc1 = 0.f, acc2 = 0.f, acc3 = 0.f;   // sweep 2
             float best = -INFINITY;                          // match
             int best_slot = 0x7fffffff;
-            float col_next[4] = {INFINITY, INFINITY, INFINITY, INFINITY};   // sweep 2: values of the next tile
+            float lse_next = INFINITY;                       // sweep 2: value for this group's next tile
             bool have_next = false;
 
             for (int t = 0; t < it.nt; ++t, ++gb) {
                 if ((int)(gb % kGroups) != wg) continue;
                 const int buf = wg;
-                float* side = sh.side[warp - kEpiWarp0];
+                float* side = sh.side[wg][lt & 1];
                 bool diag = false;                           // tile crosses the causal diagonal
                 int col_limit = kTile;                       // match: valid kept slots in the tile
                 if (KIND == kSweep1) {
                     diag = (t == it.blk);
                 } else if (KIND == kSweep2) {
-                    // Every warp stages the tile's 128 column values (log-sum-exp of its queries)
-                    // for itself: four coalesced loads per lane and no barrier across the group.
                     const int ib = it.blk + t / p.group;
                     const int qh = it.head * p.group + t % p.group;
-                    const float* src = p.lse + (long long)qh * p.T + it.tok_begin;
-                    const int i0 = ib * kTile + lane;        // first query column staged by this lane
-                    float v[4];
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        const int i = i0 + 32 * j;
-                        v[j] = INFINITY;                     // +inf turns the probability into 0
-                        if (have_next) v[j] = col_next[j];
-                        else if (i < it.L) v[j] = src[i] * kLog2e;
-                    }
+                    const int i = ib * kTile + row;          // query column staged by this thread
+                    float v = INFINITY;                      // +inf turns the probability into 0
+                    if (have_next) v = lse_next;
+                    else if (i < it.L) v = p.lse[(long long)qh * p.T + it.tok_begin + i] * kLog2e;
                     // without query groups the group's next tile of the item is four query blocks
-                    // further on: fetch its values now, a tile ahead of their use
+                    // further on: fetch its value now, a tile ahead of its use
                     have_next = (p.group == 1) && (t + kGroups < it.nt);
                     if (have_next) {
-#pragma unroll
-                        for (int j = 0; j < 4; ++j) {
-                            const int i = i0 + 32 * j + kGroups * kTile;
-                            col_next[j] = (i < it.L) ? src[i] * kLog2e : INFINITY;
-                        }
+                        const int i4 = i + kGroups * kTile;
+                        lse_next = (i4 < it.L) ? p.lse[(long long)qh * p.T + it.tok_begin + i4] * kLog2e : INFINITY;
                     }
-                    __syncwarp();                            // the lanes are done reading the last tile's values
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) side[lane + 32 * j] = v[j];
-                    __syncwarp();
+                    side[row] = v;
                     diag = (ib == it.blk);
+                    ptx::named_barrier_sync(1 + wg, 128);
                 } else {
-                    const float* src = p.rnorm_kept + it.kept_row0;
-                    __syncwarp();
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        const int slot = t * kTile + lane + 32 * j;
-                        side[lane + 32 * j] = (slot < it.B) ? src[slot] : 0.f;
-                    }
-                    __syncwarp();
+                    const int slot = t * kTile + row;
+                    side[row] = (slot < it.B) ? p.rnorm_kept[it.kept_row0 + slot] : 0.f;
                     col_limit = min(kTile, it.B - t * kTile);
+                    ptx::named_barrier_sync(1 + wg, 128);
                 }
                 ++lt;
                 ptx::mbar_wait(ptx::smem_u32(&sh.t_full[buf]), (gb / kAccum) & 1, abort_flag);
