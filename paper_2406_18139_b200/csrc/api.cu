@@ -34,7 +34,7 @@ struct Plan {
     std::vector<Req> reqs;                  // table order (longest first)
     std::vector<int> out_len;               // caller order
     // workspace offsets (bytes)
-    size_t o_status, o_reqs, o_lse, o_scores, o_rank, o_rnorm_all, o_kept, o_evict, o_kept_keys,
+    size_t o_status, o_reqs, o_lse, o_lse_split, o_scores, o_rank, o_rnorm_all, o_kept, o_evict, o_kept_keys,
         o_rnorm_kept, o_assign, o_sim, o_row_ptr, o_members, o_member_w, o_units, o_slot_cnt, o_parts, o_sort_a, o_sort_b,
         total;
 };
@@ -133,6 +133,7 @@ int build_plan(Plan& pl, const lookm_layout* lay, int n_req, const int* cu_seqle
     pl.o_status = carve(256);
     pl.o_reqs = carve(sizeof(Req) * n_req);
     pl.o_lse = carve(4 * Hq * T);
+    pl.o_lse_split = carve(32 * Hq * T);
     pl.o_scores = carve(4 * Hkv * T);
     pl.o_rank = carve(4 * Hkv * T);
     pl.o_rnorm_all = carve(4 * Hkv * T);
@@ -220,6 +221,21 @@ int make_map_3d(CUtensorMap* map, const void* base, long long tokens, int heads,
     return r == CUDA_SUCCESS ? LOOKM_OK : LOOKM_ERR_CUDA;
 }
 
+// The 16-column companion of the query tensor ([tokens, heads, 16] bf16, 32-byte rows): boxes of
+// 128 tokens of one head with the 32-byte swizzle.
+int make_map_split(CUtensorMap* map, const void* base, long long tokens, int heads) {
+    auto enc = tensor_map_encoder();
+    if (!enc) return LOOKM_ERR_CUDA;
+    cuuint64_t dims[3] = {16, (cuuint64_t)heads, (cuuint64_t)tokens};
+    cuuint64_t strides[2] = {32, (cuuint64_t)heads * 32};
+    cuuint32_t box[3] = {16, 1, (cuuint32_t)kTile};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides,
+                     box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_32B,
+                     CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? LOOKM_OK : LOOKM_ERR_CUDA;
+}
+
 int make_map_2d(CUtensorMap* map, const void* base, long long rows) {
     auto enc = tensor_map_encoder();
     if (!enc) return LOOKM_ERR_CUDA;
@@ -285,17 +301,24 @@ int run_score(const Plan& pl, const DeviceInfo& di, const lookm_layout* lay, con
     CUtensorMap map_q, map_k;
     LOOKM_TRY(make_map_3d(&map_q, q, pl.T, pl.n_q_heads, lay->q_stride_tok, lay->q_stride_head));
     LOOKM_TRY(make_map_3d(&map_k, k, pl.T, pl.n_kv_heads, lay->kv_stride_tok, lay->kv_stride_head));
+    CUtensorMap map_x;
+    unsigned short* split = at<unsigned short>(ws, pl.o_lse_split);
+    LOOKM_TRY(make_map_split(&map_x, split, pl.T, pl.n_q_heads));
     TileParams p = tile_params(pl, ws, lay);
     p.lse = lse;
+    p.lse_split = split;
     p.scores = scores;
     if (!lse_is_input) {
         p.n_items = pl.n_items[kSweep1];
-        LOOKM_CUDA(launch_tile_kernel(kSweep1, map_q, map_k, p, di.sms, st));
+        LOOKM_CUDA(launch_tile_kernel(kSweep1, map_q, map_k, nullptr, p, di.sms, st));
+        ++g_launches;
+    } else {
+        LOOKM_CUDA(launch_lse_split(lse, pl.n_q_heads, pl.T, p.scale_log2, split, st));
         ++g_launches;
     }
     mark_stage(1, st);
     p.n_items = pl.n_items[kSweep2];
-    LOOKM_CUDA(launch_tile_kernel(kSweep2, map_k, map_q, p, di.sms, st));
+    LOOKM_CUDA(launch_tile_kernel(kSweep2, map_k, map_q, &map_x, p, di.sms, st));
     ++g_launches;
     mark_stage(2, st);
     return LOOKM_OK;
@@ -330,7 +353,7 @@ int run_match(const Plan& pl, const DeviceInfo& di, const lookm_layout* lay, con
     p.rnorm_kept = rnorm_kept;
     p.assign = assign;
     p.sim = sim;
-    LOOKM_CUDA(launch_tile_kernel(kMatch, map_k, map_c, p, di.sms, st));
+    LOOKM_CUDA(launch_tile_kernel(kMatch, map_k, map_c, nullptr, p, di.sms, st));
     ++g_launches;
     mark_stage(5, st);
     return LOOKM_OK;

@@ -62,7 +62,9 @@ struct TileParams {
     int n_q_heads, n_kv_heads, group;
     long long T;                 // total packed tokens
     float scale_log2;            // softmax scale * log2(e)
-    float* lse;                  // [n_q_heads, T] natural log (sweep 1 writes, sweep 2 reads)
+    float* lse;                  // [n_q_heads, T] natural log (sweep 1 writes)
+    unsigned short* lse_split;   // [T, n_q_heads, 16] bf16: -lse / scale as three bf16 terms and 13
+                                 // zeros per query row (sweep 1 writes, sweep 2 loads it by TMA)
     float* scores;               // [n_kv_heads, T]
     const int* rank;             // [n_kv_heads, T]      (match)
     const float* rnorm_all;      // [n_kv_heads, T]      (match)
@@ -73,8 +75,14 @@ struct TileParams {
 };
 
 // ---- launchers (each enqueues on `stream` and returns the CUDA error of the launch) -----------
+// map_x: the lse_split tensor (sweep 2 only; NULL otherwise)
 cudaError_t launch_tile_kernel(int kind, const CUtensorMap& map_a, const CUtensorMap& map_b,
-                               const TileParams& p, int num_sms, cudaStream_t stream);
+                               const CUtensorMap* map_x, const TileParams& p, int num_sms,
+                               cudaStream_t stream);
+
+// lse_split from a given lse (for callers that supply their own log-sum-exp)
+cudaError_t launch_lse_split(const float* lse, int n_q_heads, long long T, float scale_log2,
+                             unsigned short* lse_split, cudaStream_t stream);
 
 cudaError_t launch_select(const float* scores, const uint8_t* mask, const Req* reqs, int n_req,
                           int n_kv_heads, long long T, int* kept_idx, int* evict_idx, int* rank,

@@ -22,6 +22,10 @@ __device__ __forceinline__ uint64_t globaltimer_ns() {
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
 }
+// Makes shared-memory writes of this thread visible to the async proxy (TMA, tensor core).
+__device__ __forceinline__ void fence_proxy_async_shared() {
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
 __device__ __forceinline__ void fence_mbar_init() {
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
 }
@@ -115,6 +119,13 @@ __device__ __forceinline__ void tc_fence_after_sync() {
 __device__ __forceinline__ uint64_t umma_desc_sw128(uint32_t smem_addr) {
     const uint32_t lo = ((smem_addr & 0x3FFFFu) >> 4) | (1u << 16);
     const uint32_t hi = (1024u >> 4) | (1u << 14) | (2u << 29);
+    return (static_cast<uint64_t>(hi) << 32) | lo;
+}
+// The same for 32-byte rows with the 32-byte swizzle (a TMA box of 16 bf16 x R rows with
+// SWIZZLE_32B): 8-row groups are 256 bytes apart, layout type 6.
+__device__ __forceinline__ uint64_t umma_desc_sw32(uint32_t smem_addr) {
+    const uint32_t lo = ((smem_addr & 0x3FFFFu) >> 4) | (1u << 16);
+    const uint32_t hi = (256u >> 4) | (1u << 14) | (6u << 29);
     return (static_cast<uint64_t>(hi) << 32) | lo;
 }
 // Instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M x N tile.

@@ -17,12 +17,17 @@
 //   sweep 1: A = 128 queries of one query head, B = key tiles 0..diagonal.  Online softmax
 //            statistics per query row  ->  lse[i] = log sum_{j<=i} exp(s_ij).
 //   sweep 2: A = 128 keys of one KV head, B = query tiles diagonal..last of every query head in
-//            the group.  Thread of key j accumulates sum_i exp(s_ij - lse_i)  ->  A_s[j].
+//            the group.  Thread of key j accumulates sum_i exp(s_ij - lse_i)  ->  A_s[j].  The
+//            subtraction of lse_i is done by the tensor core: sweep 1 leaves -lse_i / scale as
+//            three bf16 terms in a 16-column companion of the query tensor, and a ninth MMA per
+//            tile multiplies it with a constant tile of ones, so the accumulator already holds
+//            s_ij - lse_i / scale and the epilogue needs no per-column data at all.
 //   match  : A = 128 key rows (all positions; kept rows are ignored at the end), B = tiles of the
 //            compacted kept keys.  Thread keeps the largest s_ij / |k_j| and its slot.
 //
 // Work items are laid out heaviest first and dealt to the CTAs in serpentine order; every role
 // walks the same item sequence on its own, so no scheduling state is shared.
+#include <cuda_bf16.h>
 #include <math.h>
 
 #include "internal.h"
@@ -39,6 +44,7 @@ constexpr int kEpiWarp0 = 2;                     // first epilogue warp
 constexpr int kThreads = 64 + kGroups * 128 + 32;   // producer warp, MMA warp, 4 x 4 epilogue warps, second MMA warp
 constexpr int kHalfBytes = kTile * 64 * 2;       // one TMA box: 128 rows x 64 bf16 (128 B rows)
 constexpr int kTileBytes = 2 * kHalfBytes;       // 128 x 128 bf16
+constexpr int kSplitBytes = kTile * 16 * 2;      // 128 rows x 16 bf16 (32-byte rows, 32-byte swizzle)
 constexpr int kReqCache = 32;                    // request-table entries cached in shared memory
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
@@ -46,7 +52,11 @@ constexpr float kLn2 = 0.6931471805599453f;
 struct __align__(1024) Shared {
     uint8_t a[2][kTileBytes];                    // stationary tiles (double-buffered across items)
     uint8_t b[kStages][kTileBytes];              // streamed tiles
-    float side[kGroups][2][kTile];               // per epilogue group, double-buffered column data
+    uint8_t bx[kStages][kSplitBytes];            // sweep 2: the streamed tiles' 16-column companions
+    union {
+        float side[kGroups][2][kTile];           // match: per epilogue group, double-buffered column data
+        uint8_t ax[kSplitBytes];                 // sweep 2: constant ones tile that multiplies bx
+    };
     float comb[2][kGroups][2][kTile];            // partial results of the groups, double-buffered
     Req reqs[kReqCache];                         // copy of the request table (when it fits)
     unsigned long long a_full[2], a_empty[2];
@@ -63,6 +73,32 @@ struct __align__(1024) Shared {
 constexpr int kPolyEvery = 5;
 __device__ __forceinline__ float exp2_mixed(int column, float x) {
     return (column % kPolyEvery == kPolyEvery - 1) ? ptx::ex2_fma(x) : ptx::ex2(x);
+}
+
+// -lse / scale of one query row as three bf16 terms (their sum carries 24 bits) and 13 zeros:
+// the row of the 16-column companion tensor that sweep 2 multiplies with ones.
+__device__ __forceinline__ void store_lse_split(unsigned short* row16, float lse, float scale_log2) {
+    const float u = -lse * (kLog2e / scale_log2);
+    const __nv_bfloat16 hi = __float2bfloat16_rn(u);
+    const float r1 = u - __bfloat162float(hi);
+    const __nv_bfloat16 mid = __float2bfloat16_rn(r1);
+    const __nv_bfloat16 lo = __float2bfloat16_rn(r1 - __bfloat162float(mid));
+    uint4 w0;
+    w0.x = (uint32_t)__bfloat16_as_ushort(hi) | ((uint32_t)__bfloat16_as_ushort(mid) << 16);
+    w0.y = (uint32_t)__bfloat16_as_ushort(lo);
+    w0.z = 0u;
+    w0.w = 0u;
+    uint4* dst = reinterpret_cast<uint4*>(row16);
+    dst[0] = w0;
+    dst[1] = make_uint4(0u, 0u, 0u, 0u);
+}
+
+__global__ void lse_split_kernel(const float* __restrict__ lse, int n_q_heads, long long T,
+                                 float scale_log2, unsigned short* __restrict__ lse_split) {
+    const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;   // over [head][token]
+    if (i >= T * n_q_heads) return;
+    const long long h = i / T, tok = i % T;
+    store_lse_split(lse_split + (tok * n_q_heads + h) * 16, lse[i], scale_log2);
 }
 
 struct Item {
@@ -113,7 +149,7 @@ __device__ __forceinline__ int item_of_round(int round, int cta, int n_cta) {
 template <int KIND>
 __global__ void __launch_bounds__(kThreads, 1)
 tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-            const TileParams p) {
+            const __grid_constant__ CUtensorMap map_x, const TileParams p) {
     extern __shared__ uint8_t smem_raw[];
     Shared& sh = *reinterpret_cast<Shared*>(
         (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
@@ -142,6 +178,16 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         sh.abort_flag = 0;
         ptx::fence_mbar_init();
     }
+    if (KIND == kSweep2 && threadIdx.x < kTile) {
+        // ones tile: row r = (1, 1, 1, 0, ... 0) in bf16; with the 32-byte swizzle the two 16-byte
+        // halves of a row trade places in rows 4-7 of every group of eight
+        const int r = threadIdx.x;
+        const int first = (r >> 2) & 1;
+        uint4* row = reinterpret_cast<uint4*>(sh.ax + r * 32);
+        row[first] = make_uint4(0x3F803F80u, 0x00003F80u, 0u, 0u);
+        row[first ^ 1] = make_uint4(0u, 0u, 0u, 0u);
+        ptx::fence_proxy_async_shared();         // the tensor core reads it through the async proxy
+    }
     // everything above touches only this CTA's shared memory; from here on global memory written
     // by the kernel before this one is read
     grid_dependency_wait();
@@ -166,6 +212,7 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         if (lane == 0) {
             ptx::prefetch_tensormap(&map_a);
             ptx::prefetch_tensormap(&map_b);
+            if (KIND == kSweep2) ptx::prefetch_tensormap(&map_x);
             uint32_t gb = 0;                         // running streamed-tile index
             int n = 0;                               // items done by this CTA
             for (int round = 0;; ++round, ++n) {
@@ -185,7 +232,7 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                     const int s = gb % kStages;
                     ptx::mbar_wait(ptx::smem_u32(&sh.b_empty[s]), ((gb / kStages) & 1) ^ 1, abort_flag);
                     const uint32_t bbar = ptx::smem_u32(&sh.b_full[s]);
-                    ptx::mbar_arrive_expect_tx(bbar, kTileBytes);
+                    ptx::mbar_arrive_expect_tx(bbar, KIND == kSweep2 ? kTileBytes + kSplitBytes : kTileBytes);
                     const uint32_t bdst = ptx::smem_u32(&sh.b[s][0]);
                     if (KIND == kSweep1) {
                         const int row = it.tok_begin + t * kTile;
@@ -197,6 +244,7 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                         const int h = it.head * p.group + t % p.group;
                         ptx::tma_load_3d(bdst, &map_b, 0, h, row, bbar);
                         ptx::tma_load_3d(bdst + kHalfBytes, &map_b, 64, h, row, bbar);
+                        ptx::tma_load_3d(ptx::smem_u32(&sh.bx[s][0]), &map_x, 0, h, row, bbar);
                     } else {
                         const int row = (int)(it.kept_row0 + (long long)t * kTile);
                         ptx::tma_load_2d(bdst, &map_b, 0, row, bbar);
@@ -251,6 +299,9 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                         ptx::umma_bf16(d_tmem, ptx::umma_desc_sw128(a_addr + off),
                                        ptx::umma_desc_sw128(b_addr + off), idesc, kk > 0);
                     }
+                    if (KIND == kSweep2)                 // accumulator += ones x (-lse / scale)^T
+                        ptx::umma_bf16(d_tmem, ptx::umma_desc_sw32(ptx::smem_u32(&sh.ax[0])),
+                                       ptx::umma_desc_sw32(ptx::smem_u32(&sh.bx[s][0])), idesc, 1u);
                     ptx::umma_commit(ptx::smem_u32(&sh.b_empty[s]));
                     ptx::umma_commit(ptx::smem_u32(&sh.t_full[buf]));
                     issued = true;
@@ -285,34 +336,23 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
             float acc0 = 0.f, acc1 = 0.f, acc2 = 0.f, acc3 = 0.f;   // sweep 2
             float best = -INFINITY;                          // match
             int best_slot = 0x7fffffff;
-            float lse_next = INFINITY;                       // sweep 2: value for this group's next tile
-            bool have_next = false;
 
             for (int t = 0; t < it.nt; ++t, ++gb) {
                 if ((int)(gb % kGroups) != wg) continue;
                 const int buf = wg;
                 float* side = sh.side[wg][lt & 1];
                 bool diag = false;                           // tile crosses the causal diagonal
-                int col_limit = kTile;                       // match: valid kept slots in the tile
+                int col_limit = kTile;                       // valid columns of the tile (match, sweep 2)
+                int diag_from = 0;                           // sweep 2: first column this row may use
                 if (KIND == kSweep1) {
                     diag = (t == it.blk);
                 } else if (KIND == kSweep2) {
                     const int ib = it.blk + t / p.group;
-                    const int qh = it.head * p.group + t % p.group;
-                    const int i = ib * kTile + row;          // query column staged by this thread
-                    float v = INFINITY;                      // +inf turns the probability into 0
-                    if (have_next) v = lse_next;
-                    else if (i < it.L) v = p.lse[(long long)qh * p.T + it.tok_begin + i] * kLog2e;
-                    // without query groups the group's next tile of the item is four query blocks
-                    // further on: fetch its value now, a tile ahead of its use
-                    have_next = (p.group == 1) && (t + kGroups < it.nt);
-                    if (have_next) {
-                        const int i4 = i + kGroups * kTile;
-                        lse_next = (i4 < it.L) ? p.lse[(long long)qh * p.T + it.tok_begin + i4] * kLog2e : INFINITY;
-                    }
-                    side[row] = v;
-                    diag = (ib == it.blk);
-                    ptx::named_barrier_sync(1 + wg, 128);
+                    // columns to mask: below the diagonal in the item's first query block, and past
+                    // the end of the request in its last one (rows of the next request or zeros)
+                    col_limit = min(kTile, it.L - ib * kTile);
+                    diag = (ib == it.blk) || (col_limit < kTile);
+                    diag_from = (ib == it.blk) ? row : 0;
                 } else {
                     const int slot = t * kTile + row;
                     side[row] = (slot < it.B) ? p.rnorm_kept[it.kept_row0 + slot] : 0.f;
@@ -426,30 +466,28 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                             m_run = mx;
                         }
                     } else if (KIND == kSweep2) {
-                        // probabilities of key `pos` under query columns c0..c0+31
-                        const float4* sd = reinterpret_cast<const float4*>(side + c0);
+                        // probabilities of key `pos` under query columns c0..c0+31: the accumulator
+                        // holds s_ij - lse_i / scale
                         if (diag) {
 #pragma unroll
                             for (int c4 = 0; c4 < 8; ++c4) {
-                                const float4 l4 = sd[c4];
                                 const int c = c0 + c4 * 4;
-                                const float e0 = exp2_mixed(c4 * 4 + 0, fmaf(__uint_as_float(raw[c4 * 4 + 0]), c2, -l4.x));
-                                const float e1 = exp2_mixed(c4 * 4 + 1, fmaf(__uint_as_float(raw[c4 * 4 + 1]), c2, -l4.y));
-                                const float e2 = exp2_mixed(c4 * 4 + 2, fmaf(__uint_as_float(raw[c4 * 4 + 2]), c2, -l4.z));
-                                const float e3 = exp2_mixed(c4 * 4 + 3, fmaf(__uint_as_float(raw[c4 * 4 + 3]), c2, -l4.w));
-                                acc0 += (c + 0 >= row) ? e0 : 0.f;
-                                acc1 += (c + 1 >= row) ? e1 : 0.f;
-                                acc2 += (c + 2 >= row) ? e2 : 0.f;
-                                acc3 += (c + 3 >= row) ? e3 : 0.f;
+                                const float e0 = exp2_mixed(c4 * 4 + 0, __uint_as_float(raw[c4 * 4 + 0]) * c2);
+                                const float e1 = exp2_mixed(c4 * 4 + 1, __uint_as_float(raw[c4 * 4 + 1]) * c2);
+                                const float e2 = exp2_mixed(c4 * 4 + 2, __uint_as_float(raw[c4 * 4 + 2]) * c2);
+                                const float e3 = exp2_mixed(c4 * 4 + 3, __uint_as_float(raw[c4 * 4 + 3]) * c2);
+                                acc0 += (c + 0 >= diag_from && c + 0 < col_limit) ? e0 : 0.f;
+                                acc1 += (c + 1 >= diag_from && c + 1 < col_limit) ? e1 : 0.f;
+                                acc2 += (c + 2 >= diag_from && c + 2 < col_limit) ? e2 : 0.f;
+                                acc3 += (c + 3 >= diag_from && c + 3 < col_limit) ? e3 : 0.f;
                             }
                         } else {
 #pragma unroll
                             for (int c4 = 0; c4 < 8; ++c4) {
-                                const float4 l4 = sd[c4];
-                                acc0 += exp2_mixed(c4 * 4 + 0, fmaf(__uint_as_float(raw[c4 * 4 + 0]), c2, -l4.x));
-                                acc1 += exp2_mixed(c4 * 4 + 1, fmaf(__uint_as_float(raw[c4 * 4 + 1]), c2, -l4.y));
-                                acc2 += exp2_mixed(c4 * 4 + 2, fmaf(__uint_as_float(raw[c4 * 4 + 2]), c2, -l4.z));
-                                acc3 += exp2_mixed(c4 * 4 + 3, fmaf(__uint_as_float(raw[c4 * 4 + 3]), c2, -l4.w));
+                                acc0 += exp2_mixed(c4 * 4 + 0, __uint_as_float(raw[c4 * 4 + 0]) * c2);
+                                acc1 += exp2_mixed(c4 * 4 + 1, __uint_as_float(raw[c4 * 4 + 1]) * c2);
+                                acc2 += exp2_mixed(c4 * 4 + 2, __uint_as_float(raw[c4 * 4 + 2]) * c2);
+                                acc3 += exp2_mixed(c4 * 4 + 3, __uint_as_float(raw[c4 * 4 + 3]) * c2);
                             }
                         }
                     }
@@ -489,7 +527,10 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
 #pragma unroll
                         for (int g = 1; g < kGroups; ++g) l += lg[g] * ptx::ex2((mg[g] - m) * c2);
                         // natural-log log-sum-exp of the scaled logits
-                        p.lse[(long long)it.head * p.T + it.tok_begin + pos] = (m * c2 + ptx::lg2(l)) * kLn2;
+                        const float lse = (m * c2 + ptx::lg2(l)) * kLn2;
+                        p.lse[(long long)it.head * p.T + it.tok_begin + pos] = lse;
+                        store_lse_split(p.lse_split + ((long long)(it.tok_begin + pos) * p.n_q_heads + it.head) * 16,
+                                        lse, c2);
                     } else if (KIND == kSweep2) {
                         const float own = (acc0 + acc1) + (acc2 + acc3);
                         float a = (wg == 0) ? own : cb[0][0][row];
@@ -531,20 +572,30 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
 }  // namespace
 
 cudaError_t launch_tile_kernel(int kind, const CUtensorMap& map_a, const CUtensorMap& map_b,
-                               const TileParams& p, int num_sms, cudaStream_t stream) {
+                               const CUtensorMap* map_x, const TileParams& p, int num_sms,
+                               cudaStream_t stream) {
     if (p.n_items <= 0) return cudaSuccess;
     const int smem = (int)sizeof(Shared) + 1024;
     const int grid = p.n_items < num_sms ? p.n_items : num_sms;
+    const CUtensorMap& mx = map_x ? *map_x : map_b;      // only sweep 2 uses it
     cudaError_t err;
 #define LOOKM_LAUNCH(K)                                                                          \
     err = cudaFuncSetAttribute(tile_kernel<K>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem); \
     if (err != cudaSuccess) return err;                                                          \
-    err = launch_chained(tile_kernel<K>, dim3(grid), dim3(kThreads), (size_t)smem, stream, map_a, map_b, p);
+    err = launch_chained(tile_kernel<K>, dim3(grid), dim3(kThreads), (size_t)smem, stream, map_a, map_b, mx, p);
     if (kind == kSweep1) { LOOKM_LAUNCH(kSweep1) }
     else if (kind == kSweep2) { LOOKM_LAUNCH(kSweep2) }
     else { LOOKM_LAUNCH(kMatch) }
 #undef LOOKM_LAUNCH
     return err;
+}
+
+cudaError_t launch_lse_split(const float* lse, int n_q_heads, long long T, float scale_log2,
+                             unsigned short* lse_split, cudaStream_t stream) {
+    const long long n = T * n_q_heads;
+    if (n <= 0) return cudaSuccess;
+    lse_split_kernel<<<(unsigned)((n + 255) / 256), 256, 0, stream>>>(lse, n_q_heads, T, scale_log2, lse_split);
+    return cudaGetLastError();
 }
 
 }  // namespace lookm
