@@ -53,7 +53,7 @@ def test_scores_and_lse_match_oracle(B, L, Hq, Hkv):
     scores2 = torch.zeros_like(scores)
     B.check(B.lookm_score(q, k, [0, L], lay, scores2, lse, True, ws))
     assert torch.equal(scores, scores2)
-    assert B.lookm_last_launch_count() == 2                    # table writer + sweep 2
+    assert B.lookm_last_launch_count() == 3                    # table writer, lse companion, sweep 2
 
 
 def test_scores_custom_scale_and_strided_heads(B):
