@@ -216,9 +216,10 @@ __device__ __forceinline__ float ex2(float x) {
 // unit of the softmax epilogues): x = n + f with n the nearest integer (taken from the low mantissa
 // bits after adding 1.5 * 2^23) and f in [-1/2, 1/2], 2^f by a degree-5 minimax polynomial
 // (relative error 2.4e-7 in fp32), n added to the exponent field.  Arguments below -125 give
-// 2^-125 (about 2.4e-38) instead of a denormal or zero; NaN is not handled.
+// 2^-125 (about 2.4e-38) instead of a denormal or zero, arguments above 127 give 2^127 (the
+// exponent field must not overflow); NaN is not handled.
 __device__ __forceinline__ float ex2_fma(float x) {
-    x = fmaxf(x, -125.f);
+    x = fminf(fmaxf(x, -125.f), 127.f);
     const float r = x + 12582912.f;
     const float f = x - (r - 12582912.f);
     float p = 1.327647245e-03f;

@@ -47,6 +47,7 @@ constexpr int kTileBytes = 2 * kHalfBytes;       // 128 x 128 bf16
 constexpr int kSplitBytes = kTile * 16 * 2;      // 128 rows x 16 bf16 (32-byte rows, 32-byte swizzle)
 constexpr int kReqCache = 32;                    // request-table entries cached in shared memory
 constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kReferenceSlack = 1.152921504606847e18f;   // 2^60: largest chunk sum kept against a stale reference
 constexpr float kLn2 = 0.6931471805599453f;
 
 struct __align__(1024) Shared {
@@ -433,21 +434,18 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                     }
                     const int c0 = ch * 32;
                     if (KIND == kSweep1) {
-                        // online softmax statistics of row `pos` over key columns c0..c0+31
-                        float mx = m_run;
+                        // softmax statistics of row `pos` over key columns c0..c0+31: l_run is the
+                        // sum of exp2(x - m_run), where m_run is a REFERENCE, not necessarily the
+                        // maximum so far
                         if (diag) {
+                            // diagonal tile (the last of the item): exact running maximum
+                            float mx = m_run;
 #pragma unroll
                             for (int c = 0; c < 32; ++c)
                                 if (c0 + c <= row) mx = fmaxf(mx, __uint_as_float(raw[c]));
-                        } else {
-#pragma unroll
-                            for (int c = 0; c < 32; c += 2)
-                                mx = ptx::fmax3(mx, __uint_as_float(raw[c]), __uint_as_float(raw[c + 1]));
-                        }
-                        if (mx != -INFINITY) {               // false only above the diagonal
-                            const float mc = mx * c2;
-                            float s0 = 0.f, s1 = 0.f;
-                            if (diag) {
+                            if (mx != -INFINITY) {           // false only above the diagonal
+                                const float mc = mx * c2;
+                                float s0 = 0.f, s1 = 0.f;
 #pragma unroll
                                 for (int c = 0; c < 32; c += 2) {
                                     const float e0 = exp2_mixed(c, fmaf(__uint_as_float(raw[c]), c2, -mc));
@@ -455,15 +453,46 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                                     s0 += (c0 + c <= row) ? e0 : 0.f;
                                     s1 += (c0 + c + 1 <= row) ? e1 : 0.f;
                                 }
-                            } else {
+                                l_run = l_run * ptx::ex2(m_run * c2 - mc) + (s0 + s1);
+                                m_run = mx;
+                            }
+                        } else {
+                            // Full tiles: no maximum is taken.  The reference is the maximum of the
+                            // row's first 32 columns; later logits may exceed it as long as the
+                            // chunk's sum stays below 2^60 (fp32 has the range, and the relative
+                            // precision does not depend on the reference).  When it does not, or
+                            // overflows, the chunk is redone against its true maximum.
+                            float ref = m_run;
+                            if (ref == -INFINITY) {
+#pragma unroll
+                                for (int c = 0; c < 32; c += 2)
+                                    ref = ptx::fmax3(ref, __uint_as_float(raw[c]), __uint_as_float(raw[c + 1]));
+                            }
+                            float mc = ref * c2;
+                            float s0 = 0.f, s1 = 0.f;
+#pragma unroll
+                            for (int c = 0; c < 32; c += 2) {
+                                s0 += exp2_mixed(c, fmaf(__uint_as_float(raw[c]), c2, -mc));
+                                s1 += exp2_mixed(c + 1, fmaf(__uint_as_float(raw[c + 1]), c2, -mc));
+                            }
+                            if (!(s0 + s1 < kReferenceSlack)) {
+                                float mx = ref;
+#pragma unroll
+                                for (int c = 0; c < 32; c += 2)
+                                    mx = ptx::fmax3(mx, __uint_as_float(raw[c]), __uint_as_float(raw[c + 1]));
+                                mc = mx * c2;
+                                s0 = 0.f;
+                                s1 = 0.f;
 #pragma unroll
                                 for (int c = 0; c < 32; c += 2) {
                                     s0 += exp2_mixed(c, fmaf(__uint_as_float(raw[c]), c2, -mc));
                                     s1 += exp2_mixed(c + 1, fmaf(__uint_as_float(raw[c + 1]), c2, -mc));
                                 }
+                                l_run *= ptx::ex2(ref * c2 - mc);
+                                ref = mx;
                             }
-                            l_run = l_run * ptx::ex2(m_run * c2 - mc) + (s0 + s1);
-                            m_run = mx;
+                            l_run += s0 + s1;
+                            m_run = ref;
                         }
                     } else if (KIND == kSweep2) {
                         // probabilities of key `pos` under query columns c0..c0+31: the accumulator

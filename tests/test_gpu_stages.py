@@ -73,6 +73,33 @@ def test_scores_custom_scale_and_strided_heads(B):
     assert np.all(np.abs(got - A) <= 2e-5 * A)
 
 
+def test_scores_logits_that_grow_along_the_prompt(B):
+    """Logits that rise by far more than 2^60 (and past fp32's exp range) from the first keys of a
+    row to its last ones: sweep 1 keeps the maximum of a row's first 32 keys as its reference and
+    must notice when later keys leave it behind; rows also end at every distance from a tile edge."""
+    import torch
+    L, H = 700, 2
+    qn = synth.normal(synth.stream_key(140), L * H * 128).reshape(L, H, 128).astype(np.float32) * 0.25
+    kn = synth.normal(synth.stream_key(141), L * H * 128).reshape(L, H, 128).astype(np.float32) * 0.25
+    qn[:, :, 0] = 4.0
+    kn[:, 0, 0] = 8.0 * np.arange(L) / L                    # head 0: rising
+    kn[:, 1, 0] = 8.0 * (1.0 - np.arange(L) / L)            # head 1: falling (reference stays the maximum)
+    qb, kb = synth.f32_to_bf16_bits(qn), synth.f32_to_bf16_bits(kn)
+    qf, kf = synth.bf16_to_f32(qb), synth.bf16_to_f32(kb)
+    q, k = to_dev(qb), to_dev(kb)
+    lay = B.make_layout(q, k, softmax_scale=4.0)
+    ws = B.alloc_workspace(lay, [L])
+    scores = torch.zeros(H, L, dtype=torch.float32, device="cuda")
+    lse = torch.zeros(H, L, dtype=torch.float32, device="cuda")
+    B.check(B.lookm_score(q, k, [0, L], lay, scores, lse, False, ws))
+    assert B.lookm_device_status(ws) == B.OK
+    A, lse_o = orc.scores(qf, kf, scale=4.0, want_lse=True)
+    assert np.allclose(lse.cpu().numpy().reshape(H, 1, L), lse_o, rtol=1e-6, atol=2e-5)
+    got = scores.cpu().numpy().astype(np.float64)
+    assert np.all(np.abs(got - A) <= 1e-3 * A)
+    assert np.all(np.abs(got - A) <= 1e-4 * A)              # exponent arguments reach 130: 1e-5 relative
+
+
 def test_scores_packed_batch_equals_separate_requests(B):
     import torch
     lens = [200, 131, 1, 400]
