@@ -96,8 +96,9 @@ def test_scores_logits_that_grow_along_the_prompt(B):
     A, lse_o = orc.scores(qf, kf, scale=4.0, want_lse=True)
     assert np.allclose(lse.cpu().numpy().reshape(H, 1, L), lse_o, rtol=1e-6, atol=2e-5)
     got = scores.cpu().numpy().astype(np.float64)
-    assert np.all(np.abs(got - A) <= 1e-3 * A)
-    assert np.all(np.abs(got - A) <= 1e-4 * A)              # exponent arguments reach 130: 1e-5 relative
+    # scores below fp32's normal range (the oracle goes down to 1e-57 here) flush to zero
+    assert np.all(np.abs(got - A) <= 1e-4 * A + 1e-30)      # exponent arguments reach 130: 1e-5 relative
+    assert np.allclose(got.sum(axis=1), L, rtol=1e-5)
 
 
 def test_scores_packed_batch_equals_separate_requests(B):
