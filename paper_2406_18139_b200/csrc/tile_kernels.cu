@@ -462,36 +462,27 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                             // chunk's sum stays below 2^60 (fp32 has the range, and the relative
                             // precision does not depend on the reference).  When it does not, or
                             // overflows, the chunk is redone against its true maximum.
-                            float ref = m_run;
-                            if (ref == -INFINITY) {
-#pragma unroll
-                                for (int c = 0; c < 32; c += 2)
-                                    ref = ptx::fmax3(ref, __uint_as_float(raw[c]), __uint_as_float(raw[c + 1]));
-                            }
-                            float mc = ref * c2;
-                            float s0 = 0.f, s1 = 0.f;
-#pragma unroll
-                            for (int c = 0; c < 32; c += 2) {
-                                s0 += exp2_mixed(c, fmaf(__uint_as_float(raw[c]), c2, -mc));
-                                s1 += exp2_mixed(c + 1, fmaf(__uint_as_float(raw[c + 1]), c2, -mc));
-                            }
-                            if (!(s0 + s1 < kReferenceSlack)) {
-                                float mx = ref;
-#pragma unroll
-                                for (int c = 0; c < 32; c += 2)
-                                    mx = ptx::fmax3(mx, __uint_as_float(raw[c]), __uint_as_float(raw[c + 1]));
-                                mc = mx * c2;
-                                s0 = 0.f;
-                                s1 = 0.f;
+                            float ref = m_run;           // -inf at the row's first chunk: the sum
+                            float sum;                   // overflows and the second round sets it
+#pragma unroll 1
+                            for (int round2 = 0;; ++round2) {
+                                const float mc = ref * c2;
+                                float s0 = 0.f, s1 = 0.f;
 #pragma unroll
                                 for (int c = 0; c < 32; c += 2) {
                                     s0 += exp2_mixed(c, fmaf(__uint_as_float(raw[c]), c2, -mc));
                                     s1 += exp2_mixed(c + 1, fmaf(__uint_as_float(raw[c + 1]), c2, -mc));
                                 }
-                                l_run *= ptx::ex2(ref * c2 - mc);
+                                sum = s0 + s1;
+                                if (sum < kReferenceSlack || round2) break;
+                                float mx = ref;
+#pragma unroll
+                                for (int c = 0; c < 32; c += 2)
+                                    mx = ptx::fmax3(mx, __uint_as_float(raw[c]), __uint_as_float(raw[c + 1]));
+                                l_run *= ptx::ex2(ref * c2 - mx * c2);
                                 ref = mx;
                             }
-                            l_run += s0 + s1;
+                            l_run += sum;
                             m_run = ref;
                         }
                     } else if (KIND == kSweep2) {
