@@ -71,7 +71,7 @@ struct __align__(1024) Shared {
 
 // The softmax epilogues are bound by the special-function unit (16 ex2 per clock and SM), so one
 // column in kPolyEvery is exponentiated on the FMA pipe instead.
-constexpr int kPolyEvery = 5;
+constexpr int kPolyEvery = 6;
 __device__ __forceinline__ float exp2_mixed(int column, float x) {
     return (column % kPolyEvery == kPolyEvery - 1) ? ptx::ex2_fma(x) : ptx::ex2(x);
 }
