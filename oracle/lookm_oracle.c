@@ -12,8 +12,9 @@
  * Tensors are addressed as base pointer + token stride (in elements), feature index contiguous.
  *
  * Pinned by tests/test_oracle_*.py: closed forms (uniform attention -> harmonic numbers, the
- * two-token sigmoid form, single-kept-token merges), invariants (row sums, kept count, window,
- * text survival, sum preservation) and brute force on tiny inputs.  No function is unpinned.
+ * two-token sigmoid form, single-kept-token merges, the decode step's uniform mean and a
+ * three-row hand case), invariants (row sums, kept count, window, text survival, sum
+ * preservation, shift invariance) and brute force on tiny inputs.  No function is unpinned.
  */
 #include <math.h>
 #include <stdint.h>
@@ -94,6 +95,10 @@ int lookm_oracle_lse_rows(const float *q, long long q_stride_tok, const float *k
  * text score: all scores are positive, so any boosted score exceeds any unboosted one), then
  * larger A_s first, then lower position first.  T_p is never added numerically.
  *
+ * text_prior = 0 leaves Eq. 5 out: the N best are taken by A_s alone (Eq. 8 on the raw scores;
+ * the rows of the paper's main-results table that merge without the text prior), ties still to
+ * the lower position.
+ *
  * mask[j] = 1 for an image token, 0 for text.  B and M are clamped: B <= L, M <= B.
  * kept[] receives the kept positions in ascending order (the N selected, then the window);
  * evicted[] the others in ascending order.  Returns the kept count (= min(B, L)), or -1.
@@ -108,7 +113,7 @@ static int cand_before(const cand_t *a, const cand_t *b)
 }
 
 int lookm_oracle_select(const double *scores, const uint8_t *mask, int L, int B, int M,
-                        int *kept, int *evicted)
+                        int text_prior, int *kept, int *evicted)
 {
     if (L <= 0 || B <= 0 || M < 0) return -1;
     if (B > L) B = L;
@@ -117,7 +122,7 @@ int lookm_oracle_select(const double *scores, const uint8_t *mask, int L, int B,
     cand_t *c = (cand_t *)malloc(sizeof(cand_t) * (size_t)(n_cand > 0 ? n_cand : 1));
     uint8_t *keep = (uint8_t *)calloc((size_t)L, 1);
     if (!c || !keep) { free(c); free(keep); return -1; }
-    for (int j = 0; j < n_cand; ++j) { c[j].is_text = mask[j] ? 0 : 1; c[j].score = scores[j]; c[j].pos = j; }
+    for (int j = 0; j < n_cand; ++j) { c[j].is_text = (text_prior && !mask[j]) ? 1 : 0; c[j].score = scores[j]; c[j].pos = j; }
     /* insertion of the N best by repeated selection: O(N * L), obviously a full ordering */
     for (int r = 0; r < N; ++r) {
         int best = r;
@@ -190,6 +195,7 @@ void lookm_oracle_argmax_rows(const double *sim_matrix, int n_evicted, int n_kep
  *   mode 0 averaged : (x_c + sum_e x_e) / (n + 1)
  *   mode 1 pivotal  : (x_c + 1/2 sum_e (x_e + x_c)) / (n + 1)
  *   mode 2 weighted : (x_c + sum_e sim[e] x_e) / (n + 1)
+ *   mode 3 none     : x_c  (eviction alone, Eq. 6-7: the evicted rows are dropped, not merged)
  * All sums use the original rows.  out is [n_kept, d] in fp64.
  * ------------------------------------------------------------------------------------------ */
 int lookm_oracle_merge(const float *x, long long x_stride_tok, int d, const int *kept, int n_kept,
@@ -202,7 +208,7 @@ int lookm_oracle_merge(const float *x, long long x_stride_tok, int d, const int 
         const float *xc = x + (long long)kept[c] * x_stride_tok;
         for (int t = 0; t < d; ++t) out[(long long)c * d + t] = (double)xc[t];
     }
-    for (int e = 0; e < n_evicted; ++e) {
+    for (int e = 0; e < n_evicted && mode != 3; ++e) {
         int c = assign[e];
         const float *xe = x + (long long)evicted[e] * x_stride_tok;
         const float *xc = x + (long long)kept[c] * x_stride_tok;
@@ -218,5 +224,40 @@ int lookm_oracle_merge(const float *x, long long x_stride_tok, int d, const int 
     for (int c = 0; c < n_kept; ++c)
         for (int t = 0; t < d; ++t) out[(long long)c * d + t] /= (double)(count[c] + 1);
     free(count);
+    return 0;
+}
+
+/* ------------------------------------------------------------------------------------------
+ * The step after the path: one token-generation step over a cache (Section 3.1, Eq. 2-3).
+ * The new token's key and value rows are appended to the cache first (Eq. 2); the caller passes
+ * the cache WITH that row, n rows in all.  Then, for each of the n_group query heads that share
+ * this KV head,  out_g = softmax(q_g K^T * scale) V  over all n rows (Eq. 3; no mask: every cached
+ * row precedes the new token).  out is [n_group, d] in fp64.  Returns 0, or -1 without memory.
+ * ------------------------------------------------------------------------------------------ */
+int lookm_oracle_decode_head(const float *q, long long q_stride_head, int n_group, const float *k,
+                             long long k_stride_row, const float *v, long long v_stride_row, int n,
+                             int d, double scale, double *out)
+{
+    double *p = (double *)malloc(sizeof(double) * (size_t)(n > 0 ? n : 1));
+    if (!p) return -1;
+    for (int g = 0; g < n_group; ++g) {
+        const float *qg = q + (long long)g * q_stride_head;
+        double row_max = -INFINITY;
+        for (int j = 0; j < n; ++j) {
+            const float *kj = k + (long long)j * k_stride_row;
+            double dot = 0.0;
+            for (int c = 0; c < d; ++c) dot += (double)qg[c] * (double)kj[c];
+            p[j] = dot * scale;
+            if (p[j] > row_max) row_max = p[j];
+        }
+        double denom = 0.0;
+        for (int j = 0; j < n; ++j) { p[j] = exp(p[j] - row_max); denom += p[j]; }
+        for (int c = 0; c < d; ++c) {
+            double acc = 0.0;
+            for (int j = 0; j < n; ++j) acc += p[j] * (double)v[(long long)j * v_stride_row + c];
+            out[(long long)g * d + c] = acc / denom;
+        }
+    }
+    free(p);
     return 0;
 }

@@ -28,7 +28,7 @@ _SO = os.path.join(_HERE, "_lookm_oracle.so")
 _lib = None
 _lock = threading.Lock()
 
-MERGE_AVERAGE, MERGE_PIVOTAL, MERGE_WEIGHTED = 0, 1, 2
+MERGE_AVERAGE, MERGE_PIVOTAL, MERGE_WEIGHTED, MERGE_NONE = 0, 1, 2, 3
 
 
 def build(force: bool = False) -> str:
@@ -58,7 +58,7 @@ def _lib_locked():
         L.lookm_oracle_scores_head.restype = C.c_int
         L.lookm_oracle_lse_rows.argtypes = [fp, ll, fp, ll, C.c_int, C.c_double, ip, C.c_int, dp]
         L.lookm_oracle_lse_rows.restype = C.c_int
-        L.lookm_oracle_select.argtypes = [dp, u8p, C.c_int, C.c_int, C.c_int, ip, ip]
+        L.lookm_oracle_select.argtypes = [dp, u8p, C.c_int, C.c_int, C.c_int, C.c_int, ip, ip]
         L.lookm_oracle_select.restype = C.c_int
         L.lookm_oracle_match.argtypes = [fp, ll, C.c_int, ip, C.c_int, ip, C.c_int, ip, dp, dp]
         L.lookm_oracle_match.restype = None
@@ -67,6 +67,9 @@ def _lib_locked():
         L.lookm_oracle_merge.argtypes = [fp, ll, C.c_int, ip, C.c_int, ip, C.c_int, ip, dp,
                                          C.c_int, dp]
         L.lookm_oracle_merge.restype = C.c_int
+        L.lookm_oracle_decode_head.argtypes = [fp, ll, C.c_int, fp, ll, fp, ll, C.c_int, C.c_int,
+                                               C.c_double, dp]
+        L.lookm_oracle_decode_head.restype = C.c_int
         _lib = L
     return _lib
 
@@ -153,8 +156,10 @@ def lse_rows(q, k, q_head: int, kv_head: int, rows, scale: Optional[float] = Non
     return out
 
 
-def select(score_row, mask, budget: int, window: int):
-    """Window + text prior + Top-N for one head: (kept, evicted) ascending int32 position arrays."""
+def select(score_row, mask, budget: int, window: int, text_prior: bool = True):
+    """Window + text prior + Top-N for one head: (kept, evicted) ascending int32 position arrays.
+
+    text_prior=False ranks the candidates by score alone (Eq. 8 without the boost of Eq. 5)."""
     s = np.ascontiguousarray(score_row, dtype=np.float64)
     m = np.ascontiguousarray(mask, dtype=np.uint8)
     L = s.shape[0]
@@ -163,7 +168,7 @@ def select(score_row, mask, budget: int, window: int):
     kept = np.zeros(nk, dtype=np.int32)
     ev = np.zeros(L - nk, dtype=np.int32)
     rc = lib().lookm_oracle_select(_p(s, C.c_double), _p(m, C.c_uint8), L, budget, window,
-                                   _p(kept, C.c_int), _p(ev, C.c_int))
+                                   1 if text_prior else 0, _p(kept, C.c_int), _p(ev, C.c_int))
     if rc != nk:
         raise ValueError("oracle select rejected its arguments")
     return kept, ev
@@ -219,8 +224,11 @@ def merge(x, kv_head: int, kept, evicted, assign, sim, mode: int) -> np.ndarray:
 
 def compress_layer(q, k, v, mask, budget: int, window: int, mode: int,
                    scale: Optional[float] = None, kv_heads: Optional[Sequence[int]] = None,
-                   threads: int = 1, score_dtype=np.float64):
+                   threads: int = 1, score_dtype=np.float64, text_prior: bool = True):
     """Compress one request's layer.  Returns a dict of per-head results for `kv_heads`.
+
+    mode MERGE_NONE evicts without merging (no matching is done: `assign` and `sim` are empty);
+    text_prior=False selects by score alone.
 
     score_dtype=np.float32 rounds the scores to fp32 before selection, and the similarities
     before weighted merging are kept in fp64; this is what a comparison with a kernel that
@@ -236,10 +244,15 @@ def compress_layer(q, k, v, mask, budget: int, window: int, mode: int,
     def one(idx):
         h = heads[idx]
         srow = A[idx].astype(score_dtype).astype(np.float64)
-        kept, ev = select(srow, mask, budget, window)
-        assign, sim = match(k, h, kept, ev)
-        ok = merge(k, h, kept, ev, assign, sim, mode)
-        ov = merge(v, h, kept, ev, assign, sim, mode)
+        kept, ev = select(srow, mask, budget, window, text_prior=text_prior)
+        if mode == MERGE_NONE:
+            assign, sim = np.zeros(0, dtype=np.int32), np.zeros(0)
+            ev_m = ev[:0]
+        else:
+            assign, sim = match(k, h, kept, ev)
+            ev_m = ev
+        ok = merge(k, h, kept, ev_m, assign, sim, mode)
+        ov = merge(v, h, kept, ev_m, assign, sim, mode)
         return kept, ev, assign, sim, ok, ov
 
     for kept, ev, assign, sim, ok, ov in _pool_map(one, range(len(heads)), threads):
@@ -251,12 +264,44 @@ def compress_layer(q, k, v, mask, budget: int, window: int, mode: int,
 
 def compress_varlen(q, k, v, mask, cu_seqlens, budgets, windows, modes,
                     scale: Optional[float] = None, kv_heads: Optional[Sequence[int]] = None,
-                    threads: int = 1, score_dtype=np.float64):
+                    threads: int = 1, score_dtype=np.float64, text_prior: bool = True):
     """Packed batch: every request compressed on its own slice of the token axis."""
     out = []
     for r in range(len(cu_seqlens) - 1):
         a, b = int(cu_seqlens[r]), int(cu_seqlens[r + 1])
         out.append(compress_layer(q[a:b], k[a:b], v[a:b], mask[a:b], int(budgets[r]),
                                   int(windows[r]), int(modes[r]), scale=scale, kv_heads=kv_heads,
-                                  threads=threads, score_dtype=score_dtype))
+                                  threads=threads, score_dtype=score_dtype, text_prior=text_prior))
     return out
+
+
+# ---------------------------------------------------------------------------------------------
+# the step after the path: token generation over a cache (Section 3.1, Eq. 2-3)
+# ---------------------------------------------------------------------------------------------
+
+def decode_step(q_t, k_new, v_new, cache_k, cache_v, scale: Optional[float] = None):
+    """One generation step of one layer.
+
+    q_t [Hq, d]; k_new, v_new [Hkv, d]; cache_k, cache_v [Hkv, n, d] (float32 arrays holding the
+    cached rows).  The new rows are appended (Eq. 2), then every query head attends over its KV
+    head's n + 1 rows (Eq. 3).  Returns (out [Hq, d] float64, cache_k', cache_v' [Hkv, n + 1, d]).
+    """
+    q_t = np.ascontiguousarray(q_t, dtype=np.float32)
+    ck = np.concatenate([np.asarray(cache_k, dtype=np.float32),
+                         np.asarray(k_new, dtype=np.float32)[:, None, :]], axis=1)
+    cv = np.concatenate([np.asarray(cache_v, dtype=np.float32),
+                         np.asarray(v_new, dtype=np.float32)[:, None, :]], axis=1)
+    ck, cv = np.ascontiguousarray(ck), np.ascontiguousarray(cv)
+    Hq, d = q_t.shape
+    Hkv, n, _ = ck.shape
+    assert Hq % Hkv == 0
+    G = Hq // Hkv
+    scale = 1.0 / math.sqrt(d) if scale is None else float(scale)
+    out = np.zeros((Hq, d), dtype=np.float64)
+    for h in range(Hkv):
+        rc = lib().lookm_oracle_decode_head(_p(q_t[h * G:], C.c_float), d, G, _p(ck[h], C.c_float), d,
+                                            _p(cv[h], C.c_float), d, n, d, scale,
+                                            _p(out[h * G:], C.c_double))
+        if rc != 0:
+            raise MemoryError("oracle decode")
+    return out, ck, cv
