@@ -56,7 +56,9 @@ typedef enum {
 typedef enum {
     LOOKM_MERGE_AVERAGE = 0,          /* Eq. 10 */
     LOOKM_MERGE_PIVOTAL = 1,          /* Eq. 11 */
-    LOOKM_MERGE_WEIGHTED = 2          /* Eq. 12 */
+    LOOKM_MERGE_WEIGHTED = 2,         /* Eq. 12 */
+    LOOKM_MERGE_NONE = 3              /* eviction alone (Eq. 6-7): kept rows are copied, evicted rows
+                                         dropped; no matching is done for such a request */
 } lookm_merge_mode;
 
 /* Shapes and strides (in elements) of Q [tokens, n_q_heads, head_dim] and of K and V
@@ -99,6 +101,39 @@ int lookm_compress_varlen(const void* q, const void* k, const void* v, const uin
                           int* out_cu_seqlens_host, void* workspace, size_t workspace_bytes,
                           void* cuda_stream);
 
+/* Options of the whole-path calls below; a NULL pointer or an all-zero struct selects the
+ * behaviour of lookm_compress_layer / lookm_compress_varlen.
+ *   flags            LOOKM_OPT_NO_TEXT_PRIOR: leave the boost of Eq. 5 out and rank the candidates
+ *                    by A_s alone (Eq. 8 on the raw scores: the paper's merging rows without the
+ *                    text prior).  modality_mask is then not read and may be NULL.
+ *   lse              device [n_q_heads, total_tokens] fp32, natural-log row log-sum-exp of the
+ *                    prompt's causal attention, e.g. as the caller's prefill attention kernel
+ *                    left it (Eq. 4 takes its scores from that very attention).  When not NULL the
+ *                    first score sweep is skipped.  It must belong to the same q, k and scale.
+ *   out_stride_head  lookm_compress_layer_opt only: elements between two heads of out_k / out_v,
+ *                    so that the compressed rows can be written into a cache with room for
+ *                    generated tokens ([n_kv_heads, capacity, 128]: capacity * 128).  0 selects
+ *                    the dense out_len * 128; otherwise a multiple of 8, at least out_len * 128. */
+#define LOOKM_OPT_NO_TEXT_PRIOR 1u
+typedef struct {
+    unsigned flags;
+    const float* lse;
+    long long out_stride_head;
+} lookm_options;
+
+/* lookm_compress_layer / lookm_compress_varlen with options (Section 3.2-3.3, Eq. 4-12). */
+int lookm_compress_layer_opt(const void* q, const void* k, const void* v, const uint8_t* modality_mask,
+                             int seq_len, int budget, int recent_window, int merge_mode,
+                             const lookm_layout* layout, const lookm_options* options, void* out_k,
+                             void* out_v, int* out_len_host, void* workspace, size_t workspace_bytes,
+                             void* cuda_stream);
+int lookm_compress_varlen_opt(const void* q, const void* k, const void* v, const uint8_t* modality_mask,
+                              const int* cu_seqlens_host, int n_requests, const int* budgets_host,
+                              const int* windows_host, const int* merge_modes_host,
+                              const lookm_layout* layout, const lookm_options* options, void* out_k,
+                              void* out_v, int* out_cu_seqlens_host, void* workspace,
+                              size_t workspace_bytes, void* cuda_stream);
+
 /* Step 1 alone (Eq. 4): scores[h, t] = sum over the query heads of KV head h and over the rows
  * i >= t of the same request of softmax_row_i(q_i . k * scale)[t].
  *   scores  [n_kv_heads, total_tokens] fp32
@@ -112,6 +147,8 @@ int lookm_score(const void* q, const void* k, const int* cu_seqlens_host, int n_
 
 /* The selection alone (Eq. 5-8), fed with given scores [n_kv_heads, total_tokens] (fp32; the
  * method's scores are positive, other finite values are ordered numerically).
+ *   modality_mask  NULL switches the text prior off: every candidate is ranked by its score alone
+ *               (Eq. 8 without Eq. 5)
  *   kept_idx    kept positions, ascending (layout above)
  *   evict_idx   evicted positions, ascending
  *   rank        [n_kv_heads, total_tokens]: evicted token -> its index in the evicted list,
@@ -136,6 +173,8 @@ int lookm_match_from_sim(const float* sim_matrix, const int* cu_seqlens_host, in
                          void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /* The merging alone (Eq. 10-12 and the compaction of Eq. 6-7), fed with given lists.
+ * Requests whose mode is LOOKM_MERGE_NONE only have their kept rows copied; assign and sim may be
+ * NULL when every request of the call has that mode.
  * varlen_output = 0: out [n_kv_heads, out_len, 128] (requires n_requests == 1);
  * varlen_output = 1: out [sum_r out_len_r, n_kv_heads, 128]. */
 int lookm_merge(const void* k, const void* v, const int* kept_idx, const int* evict_idx,

@@ -18,9 +18,11 @@ _lib = None
 
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE_TOO_SMALL, ERR_CUDA, ERR_DEVICE_TIMEOUT, \
     ERR_DEVICE_BAD_INDEX = range(7)
-MERGE_AVERAGE, MERGE_PIVOTAL, MERGE_WEIGHTED = 0, 1, 2
+MERGE_AVERAGE, MERGE_PIVOTAL, MERGE_WEIGHTED, MERGE_NONE = 0, 1, 2, 3
+OPT_NO_TEXT_PRIOR = 1
 
-EXPORTS = ["lookm_workspace_size", "lookm_workspace_layout", "lookm_compress_layer", "lookm_compress_varlen", "lookm_score",
+EXPORTS = ["lookm_workspace_size", "lookm_workspace_layout", "lookm_compress_layer", "lookm_compress_varlen",
+           "lookm_compress_layer_opt", "lookm_compress_varlen_opt", "lookm_score",
            "lookm_select", "lookm_match", "lookm_match_from_sim", "lookm_merge",
            "lookm_set_stage_events", "lookm_merge_noalloc", "lookm_noalloc_status", "lookm_device_status", "lookm_last_launch_count", "lookm_strerror"]
 N_STAGE_EVENTS = 8
@@ -30,6 +32,10 @@ STAGE_NAMES = ["score_sweep1", "score_sweep2", "select_norms", "gather", "match"
 class WorkspaceOffsets(C.Structure):
     _fields_ = [(n, C.c_size_t) for n in ("status", "lse", "scores", "rank", "kept_idx", "evict_idx",
                                           "assign", "sim")]
+
+
+class Options(C.Structure):
+    _fields_ = [("flags", C.c_uint), ("lse", C.c_void_p), ("out_stride_head", C.c_longlong)]
 
 
 class Layout(C.Structure):
@@ -57,6 +63,11 @@ def lib():
                                            vp, vp, ip, vp, sz, vp]
         L.lookm_compress_varlen.argtypes = [vp, vp, vp, vp, ip, C.c_int, ip, ip, ip, lp, vp, vp, ip,
                                             vp, sz, vp]
+        op = C.POINTER(Options)
+        L.lookm_compress_layer_opt.argtypes = [vp, vp, vp, vp, C.c_int, C.c_int, C.c_int, C.c_int, lp, op,
+                                               vp, vp, ip, vp, sz, vp]
+        L.lookm_compress_varlen_opt.argtypes = [vp, vp, vp, vp, ip, C.c_int, ip, ip, ip, lp, op, vp, vp, ip,
+                                                vp, sz, vp]
         L.lookm_score.argtypes = [vp, vp, ip, C.c_int, lp, vp, vp, C.c_int, vp, sz, vp]
         L.lookm_select.argtypes = [vp, vp, ip, C.c_int, ip, ip, C.c_int, vp, vp, vp, vp, sz, vp]
         L.lookm_match.argtypes = [vp, vp, vp, ip, C.c_int, ip, lp, vp, vp, vp, sz, vp]
@@ -73,7 +84,8 @@ def lib():
         L.lookm_last_launch_count.argtypes = []
         L.lookm_strerror.argtypes = [C.c_int]
         L.lookm_strerror.restype = C.c_char_p
-        for name in ("lookm_compress_layer", "lookm_compress_varlen", "lookm_score", "lookm_select",
+        for name in ("lookm_compress_layer", "lookm_compress_varlen", "lookm_compress_layer_opt",
+                     "lookm_compress_varlen_opt", "lookm_score", "lookm_select",
                      "lookm_match", "lookm_match_from_sim", "lookm_merge", "lookm_device_status",
                      "lookm_last_launch_count"):
             getattr(L, name).restype = C.c_int
@@ -161,6 +173,13 @@ def read_intermediates(workspace, layout: Layout, seq_lens: Sequence[int], budge
     return scores, per_request
 
 
+def make_options(no_text_prior: bool = False, lse=None, out_stride_head: int = 0) -> Options:
+    """Options of the *_opt calls; `lse` is a float32 CUDA tensor [n_q_heads, total_tokens] or None
+    (the caller keeps it alive until the call's work has run)."""
+    return Options(OPT_NO_TEXT_PRIOR if no_text_prior else 0, None if lse is None else lse.data_ptr(),
+                   int(out_stride_head))
+
+
 def lookm_compress_layer(q, k, v, modality_mask, seq_len, budget, recent_window, merge_mode, layout,
                          out_k, out_v, workspace, stream=None):
     """Returns (status, out_len)."""
@@ -169,6 +188,18 @@ def lookm_compress_layer(q, k, v, modality_mask, seq_len, budget, recent_window,
                                     int(budget), int(recent_window), int(merge_mode), C.byref(layout),
                                     _ptr(out_k), _ptr(out_v), C.byref(out_len), _ptr(workspace),
                                     workspace.numel() * workspace.element_size(), _stream(stream))
+    return st, out_len.value
+
+
+def lookm_compress_layer_opt(q, k, v, modality_mask, seq_len, budget, recent_window, merge_mode, layout,
+                             options, out_k, out_v, workspace, stream=None):
+    """Returns (status, out_len).  options: an Options (see make_options) or None."""
+    out_len = C.c_int(0)
+    st = lib().lookm_compress_layer_opt(_ptr(q), _ptr(k), _ptr(v), _ptr(modality_mask), int(seq_len),
+                                        int(budget), int(recent_window), int(merge_mode), C.byref(layout),
+                                        None if options is None else C.byref(options), _ptr(out_k),
+                                        _ptr(out_v), C.byref(out_len), _ptr(workspace),
+                                        workspace.numel() * workspace.element_size(), _stream(stream))
     return st, out_len.value
 
 
@@ -181,6 +212,19 @@ def lookm_compress_varlen(q, k, v, modality_mask, cu_seqlens, budgets, windows, 
                                      n, _ints(budgets), _ints(windows), _ints(merge_modes),
                                      C.byref(layout), _ptr(out_k), _ptr(out_v), out_cu, _ptr(workspace),
                                      workspace.numel() * workspace.element_size(), _stream(stream))
+    return st, list(out_cu)
+
+
+def lookm_compress_varlen_opt(q, k, v, modality_mask, cu_seqlens, budgets, windows, merge_modes, layout,
+                              options, out_k, out_v, workspace, stream=None):
+    """Returns (status, out_cu_seqlens list).  options: an Options (see make_options) or None."""
+    n = len(cu_seqlens) - 1
+    out_cu = (C.c_int * (n + 1))()
+    st = lib().lookm_compress_varlen_opt(_ptr(q), _ptr(k), _ptr(v), _ptr(modality_mask), _ints(cu_seqlens),
+                                         n, _ints(budgets), _ints(windows), _ints(merge_modes),
+                                         C.byref(layout), None if options is None else C.byref(options),
+                                         _ptr(out_k), _ptr(out_v), out_cu, _ptr(workspace),
+                                         workspace.numel() * workspace.element_size(), _stream(stream))
     return st, list(out_cu)
 
 

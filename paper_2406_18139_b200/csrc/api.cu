@@ -3,6 +3,7 @@
 #include <algorithm>
 #include <cmath>
 #include <cstring>
+#include <initializer_list>
 #include <mutex>
 #include <vector>
 
@@ -28,6 +29,8 @@ struct Plan {
     int n_req = 0, n_q_heads = 0, n_kv_heads = 0, group = 1;
     long long T = 0, sum_B = 0, sum_E = 0, sum_EB = 0;
     int max_L = 0, max_E = 0, max_B = 0;
+    int n_none = 0;                         // requests with LOOKM_MERGE_NONE
+    long long out_stride_head = 0;          // elements between heads of a single-prompt output
     int n_items[3] = {0, 0, 0};
     long long total_slots = 0;              // n_kv_heads * sum_B
     long long total_units = 0;              // merge work units
@@ -64,7 +67,8 @@ int build_plan(Plan& pl, const lookm_layout* lay, int n_req, const int* cu_seqle
         const int budget = budgets ? budgets[r] : (int)L;
         const int window = windows ? windows[r] : 0;
         const int mode = modes ? modes[r] : 0;
-        if (budget <= 0 || window < 0 || mode < 0 || mode > 2) return LOOKM_ERR_INVALID_ARG;
+        if (budget <= 0 || window < 0 || mode < 0 || mode > LOOKM_MERGE_NONE) return LOOKM_ERR_INVALID_ARG;
+        if (mode == LOOKM_MERGE_NONE) ++pl.n_none;
         Req& q = pl.reqs[r];
         q.tok_begin = (int)begin;
         q.L = (int)L;
@@ -113,11 +117,12 @@ int build_plan(Plan& pl, const lookm_layout* lay, int n_req, const int* cu_seqle
         q.slot_begin = (int)slots;
         q.unit_begin = (int)units;
         q.unit_entries = unit_entries;
-        const long long n_units = (q.L + unit_entries - 1) / unit_entries;
+        const bool merges = q.mode != LOOKM_MERGE_NONE;
+        const long long n_units = merges ? (q.L + unit_entries - 1) / unit_entries : 0;
         units += (long long)pl.n_kv_heads * n_units;
         it0 += (long long)q.nblk * pl.n_q_heads;
         it1 += (long long)q.nblk * pl.n_kv_heads;
-        it2 += q.E > 0 ? (long long)q.nblk * pl.n_kv_heads : 0;
+        it2 += (q.E > 0 && merges) ? (long long)q.nblk * pl.n_kv_heads : 0;
         slots += (long long)q.B * pl.n_kv_heads;
     }
     pl.total_units = units;
@@ -364,42 +369,85 @@ int run_merge(const Plan& pl, const lookm_layout* lay, const void* k, const void
               int varlen_output, void* out_k, void* out_v, void* ws, cudaStream_t st) {
     const Req* reqs = at<Req>(ws, pl.o_reqs);
     int* status = at<int>(ws, pl.o_status);
-    // counter width and widest digit over the requests of the call
-    const bool wide = pl.max_E > kInvWideCountsAbove;
-    int digit_bits = 1;
-    for (const Req& r : pl.reqs) {
-        int n_pass, dbits;
-        invert_digits(r.B, wide ? kInvDigitBits32 : kInvDigitBits16, n_pass, dbits);
-        digit_bits = std::max(digit_bits, dbits);
+    if (pl.n_none < pl.n_req) {
+        // counter width and widest digit over the requests of the call
+        const bool wide = pl.max_E > kInvWideCountsAbove;
+        int digit_bits = 1;
+        for (const Req& r : pl.reqs) {
+            int n_pass, dbits;
+            invert_digits(r.B, wide ? kInvDigitBits32 : kInvDigitBits16, n_pass, dbits);
+            digit_bits = std::max(digit_bits, dbits);
+        }
+        LOOKM_CUDA(launch_invert_assignment(assign, kept_idx, evict_idx, sim, reqs, pl.n_req, pl.n_kv_heads,
+                                            pl.T, wide, digit_bits, at<int>(ws, pl.o_row_ptr), at<int>(ws, pl.o_members),
+                                            at<float>(ws, pl.o_member_w), at<int4>(ws, pl.o_units),
+                                            at<int>(ws, pl.o_slot_cnt), at<unsigned>(ws, pl.o_sort_a),
+                                            at<unsigned>(ws, pl.o_sort_b), status, st));
+        ++g_launches;
     }
-    LOOKM_CUDA(launch_invert_assignment(assign, kept_idx, evict_idx, sim, reqs, pl.n_req, pl.n_kv_heads,
-                                        pl.T, wide, digit_bits, at<int>(ws, pl.o_row_ptr), at<int>(ws, pl.o_members),
-                                        at<float>(ws, pl.o_member_w), at<int4>(ws, pl.o_units),
-                                        at<int>(ws, pl.o_slot_cnt), at<unsigned>(ws, pl.o_sort_a),
-                                        at<unsigned>(ws, pl.o_sort_b), status, st));
-    ++g_launches;
     mark_stage(6, st);
-    DeviceInfo di;
-    LOOKM_TRY(device_info(di));
-    LOOKM_CUDA(launch_merge(k, v, lay->kv_stride_tok, lay->kv_stride_head, reqs, pl.n_req,
-                            pl.n_kv_heads, pl.T, pl.total_units, at<int>(ws, pl.o_row_ptr),
-                            at<int>(ws, pl.o_members), at<float>(ws, pl.o_member_w),
-                            at<int4>(ws, pl.o_units), at<int>(ws, pl.o_slot_cnt),
-                            at<float>(ws, pl.o_parts), varlen_output, out_k, out_v, status, di.sms, st));
-    ++g_launches;
+    if (pl.n_none < pl.n_req) {
+        DeviceInfo di;
+        LOOKM_TRY(device_info(di));
+        LOOKM_CUDA(launch_merge(k, v, lay->kv_stride_tok, lay->kv_stride_head, reqs, pl.n_req,
+                                pl.n_kv_heads, pl.T, pl.total_units, at<int>(ws, pl.o_row_ptr),
+                                at<int>(ws, pl.o_members), at<float>(ws, pl.o_member_w),
+                                at<int4>(ws, pl.o_units), at<int>(ws, pl.o_slot_cnt),
+                                at<float>(ws, pl.o_parts), varlen_output, pl.out_stride_head, out_k,
+                                out_v, status, di.sms, st));
+        ++g_launches;
+    }
+    if (pl.n_none > 0) {
+        // eviction alone: the kept rows of those requests go straight to the output
+        LOOKM_CUDA(launch_compact_kept(k, v, lay->kv_stride_tok, lay->kv_stride_head, reqs, pl.n_req,
+                                       pl.n_kv_heads, pl.total_slots, kept_idx, varlen_output,
+                                       pl.out_stride_head, out_k, out_v, status, st));
+        ++g_launches;
+    }
     mark_stage(7, st);
+    return LOOKM_OK;
+}
+
+// Output pointers are written with 16-byte stores, index and weight lists read as 32-bit words.
+int check_out_ptrs(const void* out_k, const void* out_v) {
+    if ((reinterpret_cast<uintptr_t>(out_k) & 15u) || (reinterpret_cast<uintptr_t>(out_v) & 15u))
+        return LOOKM_ERR_INVALID_ARG;
+    return LOOKM_OK;
+}
+int check_word_ptrs(std::initializer_list<const void*> ptrs) {
+    for (const void* p : ptrs)
+        if (reinterpret_cast<uintptr_t>(p) & 3u) return LOOKM_ERR_INVALID_ARG;
+    return LOOKM_OK;
+}
+
+// Stride between the heads of a single-prompt output (0 = dense).
+int set_out_stride(Plan& pl, int varlen_output, long long out_stride_head) {
+    pl.out_stride_head = 0;
+    if (varlen_output) return out_stride_head ? LOOKM_ERR_INVALID_ARG : LOOKM_OK;
+    const long long dense = (long long)pl.out_len[0] * kHeadDim;
+    if (out_stride_head == 0) { pl.out_stride_head = dense; return LOOKM_OK; }
+    if (out_stride_head % 8 || out_stride_head < dense) return LOOKM_ERR_INVALID_ARG;
+    pl.out_stride_head = out_stride_head;
     return LOOKM_OK;
 }
 
 int compress_common(const void* q, const void* k, const void* v, const uint8_t* mask,
                     const int* cu_seqlens, int n_req, const int* budgets, const int* windows,
-                    const int* modes, const lookm_layout* lay, int varlen_output, void* out_k,
-                    void* out_v, int* out_cu, void* ws, size_t ws_bytes, void* stream) {
-    if (!q || !k || !v || !mask || !out_k || !out_v || !budgets || !windows || !modes)
+                    const int* modes, const lookm_layout* lay, const lookm_options* opt,
+                    int varlen_output, void* out_k, void* out_v, int* out_cu, void* ws,
+                    size_t ws_bytes, void* stream) {
+    const unsigned flags = opt ? opt->flags : 0u;
+    const float* lse_in = opt ? opt->lse : nullptr;
+    if (flags & ~LOOKM_OPT_NO_TEXT_PRIOR) return LOOKM_ERR_INVALID_ARG;
+    const bool text_prior = !(flags & LOOKM_OPT_NO_TEXT_PRIOR);
+    if (!q || !k || !v || (!mask && text_prior) || !out_k || !out_v || !budgets || !windows || !modes)
         return LOOKM_ERR_INVALID_ARG;
     Plan pl;
     LOOKM_TRY(build_plan(pl, lay, n_req, cu_seqlens, nullptr, budgets, windows, modes));
     LOOKM_TRY(check_layout_ptrs(lay, q, k, v));
+    LOOKM_TRY(check_out_ptrs(out_k, out_v));
+    LOOKM_TRY(check_word_ptrs({lse_in}));
+    LOOKM_TRY(set_out_stride(pl, varlen_output, opt ? opt->out_stride_head : 0));
     LOOKM_TRY(check_workspace(pl, ws, ws_bytes));
     DeviceInfo di;
     LOOKM_TRY(device_info(di));
@@ -416,11 +464,15 @@ int compress_common(const void* q, const void* k, const void* v, const uint8_t* 
     int* rank = at<int>(ws, pl.o_rank);
     int* assign = at<int>(ws, pl.o_assign);
     float* sim = at<float>(ws, pl.o_sim);
-    LOOKM_TRY(run_score(pl, di, lay, q, k, scores, at<float>(ws, pl.o_lse), false, ws, st));
+    // a caller's log-sum-exp (read only) replaces the first sweep
+    float* lse = lse_in ? const_cast<float*>(lse_in) : at<float>(ws, pl.o_lse);
+    LOOKM_TRY(run_score(pl, di, lay, q, k, scores, lse, lse_in != nullptr, ws, st));
     // the selection launch also computes the key norms that the matching needs
-    LOOKM_CUDA(launch_select(scores, mask, at<Req>(ws, pl.o_reqs), pl.n_req, pl.n_kv_heads, pl.T,
-                             kept, evict, rank, k, lay->kv_stride_tok, lay->kv_stride_head,
-                             at<float>(ws, pl.o_rnorm_all), di.sms, st));
+    const bool need_match = pl.n_items[kMatch] > 0;
+    LOOKM_CUDA(launch_select(scores, text_prior ? mask : nullptr, at<Req>(ws, pl.o_reqs), pl.n_req,
+                             pl.n_kv_heads, pl.T, kept, evict, rank, need_match ? k : nullptr,
+                             lay->kv_stride_tok, lay->kv_stride_head, at<float>(ws, pl.o_rnorm_all),
+                             di.sms, st));
     ++g_launches;
     mark_stage(3, st);
     LOOKM_TRY(run_match(pl, di, lay, k, kept, rank, assign, sim, ws, true, st));
@@ -460,18 +512,40 @@ int lookm_workspace_layout(const lookm_layout* layout, int n_requests, const int
     return LOOKM_OK;
 }
 
-int lookm_compress_layer(const void* q, const void* k, const void* v, const uint8_t* modality_mask,
-                         int seq_len, int budget, int recent_window, int merge_mode,
-                         const lookm_layout* layout, void* out_k, void* out_v, int* out_len_host,
-                         void* workspace, size_t workspace_bytes, void* cuda_stream) {
+int lookm_compress_layer_opt(const void* q, const void* k, const void* v, const uint8_t* modality_mask,
+                             int seq_len, int budget, int recent_window, int merge_mode,
+                             const lookm_layout* layout, const lookm_options* options, void* out_k,
+                             void* out_v, int* out_len_host, void* workspace, size_t workspace_bytes,
+                             void* cuda_stream) {
     if (seq_len <= 0) return LOOKM_ERR_INVALID_ARG;
     const int cu[2] = {0, seq_len};
     int out_cu[2] = {0, 0};
     const int st = compress_common(q, k, v, modality_mask, cu, 1, &budget, &recent_window, &merge_mode,
-                                   layout, 0, out_k, out_v, out_cu, workspace, workspace_bytes,
+                                   layout, options, 0, out_k, out_v, out_cu, workspace, workspace_bytes,
                                    cuda_stream);
     if (st == LOOKM_OK && out_len_host) *out_len_host = out_cu[1];
     return st;
+}
+
+int lookm_compress_layer(const void* q, const void* k, const void* v, const uint8_t* modality_mask,
+                         int seq_len, int budget, int recent_window, int merge_mode,
+                         const lookm_layout* layout, void* out_k, void* out_v, int* out_len_host,
+                         void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    return lookm_compress_layer_opt(q, k, v, modality_mask, seq_len, budget, recent_window, merge_mode,
+                                    layout, nullptr, out_k, out_v, out_len_host, workspace,
+                                    workspace_bytes, cuda_stream);
+}
+
+int lookm_compress_varlen_opt(const void* q, const void* k, const void* v, const uint8_t* modality_mask,
+                              const int* cu_seqlens_host, int n_requests, const int* budgets_host,
+                              const int* windows_host, const int* merge_modes_host,
+                              const lookm_layout* layout, const lookm_options* options, void* out_k,
+                              void* out_v, int* out_cu_seqlens_host, void* workspace,
+                              size_t workspace_bytes, void* cuda_stream) {
+    if (!cu_seqlens_host) return LOOKM_ERR_INVALID_ARG;
+    return compress_common(q, k, v, modality_mask, cu_seqlens_host, n_requests, budgets_host,
+                           windows_host, merge_modes_host, layout, options, 1, out_k, out_v,
+                           out_cu_seqlens_host, workspace, workspace_bytes, cuda_stream);
 }
 
 int lookm_compress_varlen(const void* q, const void* k, const void* v, const uint8_t* modality_mask,
@@ -480,16 +554,16 @@ int lookm_compress_varlen(const void* q, const void* k, const void* v, const uin
                           const lookm_layout* layout, void* out_k, void* out_v,
                           int* out_cu_seqlens_host, void* workspace, size_t workspace_bytes,
                           void* cuda_stream) {
-    if (!cu_seqlens_host) return LOOKM_ERR_INVALID_ARG;
-    return compress_common(q, k, v, modality_mask, cu_seqlens_host, n_requests, budgets_host,
-                           windows_host, merge_modes_host, layout, 1, out_k, out_v,
-                           out_cu_seqlens_host, workspace, workspace_bytes, cuda_stream);
+    return lookm_compress_varlen_opt(q, k, v, modality_mask, cu_seqlens_host, n_requests, budgets_host,
+                                     windows_host, merge_modes_host, layout, nullptr, out_k, out_v,
+                                     out_cu_seqlens_host, workspace, workspace_bytes, cuda_stream);
 }
 
 int lookm_score(const void* q, const void* k, const int* cu_seqlens_host, int n_requests,
                 const lookm_layout* layout, float* scores, float* lse, int lse_is_input,
                 void* workspace, size_t workspace_bytes, void* cuda_stream) {
     if (!q || !k || !cu_seqlens_host || !scores || (lse_is_input && !lse)) return LOOKM_ERR_INVALID_ARG;
+    LOOKM_TRY(check_word_ptrs({scores, lse}));
     Plan pl;
     LOOKM_TRY(build_plan(pl, layout, n_requests, cu_seqlens_host, nullptr, nullptr, nullptr, nullptr));
     LOOKM_TRY(check_layout_ptrs(layout, q, k, nullptr));
@@ -506,9 +580,9 @@ int lookm_select(const float* scores, const uint8_t* modality_mask, const int* c
                  int n_requests, const int* budgets_host, const int* windows_host, int n_kv_heads,
                  int* kept_idx, int* evict_idx, int* rank, void* workspace, size_t workspace_bytes,
                  void* cuda_stream) {
-    if (!scores || !modality_mask || !cu_seqlens_host || !budgets_host || !windows_host || !kept_idx ||
-        !evict_idx)
+    if (!scores || !cu_seqlens_host || !budgets_host || !windows_host || !kept_idx || !evict_idx)
         return LOOKM_ERR_INVALID_ARG;
+    LOOKM_TRY(check_word_ptrs({scores, kept_idx, evict_idx, rank}));
     lookm_layout lay;
     std::memset(&lay, 0, sizeof(lay));
     lay.n_q_heads = lay.n_kv_heads = n_kv_heads;
@@ -529,6 +603,7 @@ int lookm_match(const void* k, const int* kept_idx, const int* evict_idx, const 
                 float* sim, void* workspace, size_t workspace_bytes, void* cuda_stream) {
     if (!k || !kept_idx || !evict_idx || !cu_seqlens_host || !budgets_host || !assign || !sim)
         return LOOKM_ERR_INVALID_ARG;
+    LOOKM_TRY(check_word_ptrs({kept_idx, evict_idx, assign, sim}));
     Plan pl;
     LOOKM_TRY(build_plan(pl, layout, n_requests, cu_seqlens_host, nullptr, budgets_host, nullptr, nullptr));
     LOOKM_TRY(check_layout_ptrs(layout, nullptr, k, nullptr));
@@ -550,6 +625,7 @@ int lookm_match_from_sim(const float* sim_matrix, const int* cu_seqlens_host, in
                          const int* budgets_host, int n_kv_heads, int* assign, float* sim,
                          void* workspace, size_t workspace_bytes, void* cuda_stream) {
     if (!sim_matrix || !cu_seqlens_host || !budgets_host || !assign || !sim) return LOOKM_ERR_INVALID_ARG;
+    LOOKM_TRY(check_word_ptrs({sim_matrix, assign, sim}));
     lookm_layout lay;
     std::memset(&lay, 0, sizeof(lay));
     lay.n_q_heads = lay.n_kv_heads = n_kv_heads;
@@ -570,14 +646,18 @@ int lookm_merge(const void* k, const void* v, const int* kept_idx, const int* ev
                 const int* budgets_host, const int* merge_modes_host, const lookm_layout* layout,
                 int varlen_output, void* out_k, void* out_v, void* workspace,
                 size_t workspace_bytes, void* cuda_stream) {
-    if (!k || !v || !kept_idx || !evict_idx || !assign || !sim || !cu_seqlens_host || !budgets_host ||
-        !merge_modes_host || !out_k || !out_v)
+    if (!k || !v || !kept_idx || !evict_idx || !cu_seqlens_host || !budgets_host || !merge_modes_host ||
+        !out_k || !out_v)
         return LOOKM_ERR_INVALID_ARG;
     if (!varlen_output && n_requests != 1) return LOOKM_ERR_INVALID_ARG;
     Plan pl;
     LOOKM_TRY(build_plan(pl, layout, n_requests, cu_seqlens_host, nullptr, budgets_host, nullptr,
                          merge_modes_host));
+    if ((!assign || !sim) && pl.n_none < pl.n_req) return LOOKM_ERR_INVALID_ARG;
     LOOKM_TRY(check_layout_ptrs(layout, nullptr, k, v));
+    LOOKM_TRY(check_out_ptrs(out_k, out_v));
+    LOOKM_TRY(check_word_ptrs({kept_idx, evict_idx, assign, sim}));
+    LOOKM_TRY(set_out_stride(pl, varlen_output, 0));
     LOOKM_TRY(check_workspace(pl, workspace, workspace_bytes));
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     LOOKM_TRY(begin_call(pl, workspace, st));
@@ -663,6 +743,9 @@ extern "C" int lookm_merge_noalloc(const void* k, const void* v, const int* kept
     LOOKM_TRY(build_plan(pl, layout, n_requests, cu_seqlens_host, nullptr, budgets_host, nullptr,
                          merge_modes_host));
     LOOKM_TRY(check_layout_ptrs(layout, nullptr, k, v));
+    LOOKM_TRY(check_out_ptrs(out_k, out_v));
+    LOOKM_TRY(check_word_ptrs({kept_idx, evict_idx, assign, sim}));
+    LOOKM_TRY(set_out_stride(pl, varlen_output, 0));
     // compact carving of just what the merge needs: 28 bytes per (KV head, token), 4 per kept row,
     // the per-unit records and the table
     const size_t units = (size_t)pl.n_kv_heads * (size_t)pl.T;

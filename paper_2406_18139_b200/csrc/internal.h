@@ -37,7 +37,8 @@ struct Req {
     int B;                // kept rows  = min(budget, L)
     int M;                // recent window, clamped to B
     int E;                // evicted rows = L - B
-    int mode;             // lookm_merge_mode
+    int mode;             // lookm_merge_mode; LOOKM_MERGE_NONE requests have no match items and no
+                          // merge work units
     int nblk;             // ceil(L / kTile)
     int out_begin;        // sum of B over the requests before this one (caller order)
     long long kept_off;   // n_kv_heads * out_begin          (start of this request's kept lists)
@@ -124,8 +125,16 @@ cudaError_t launch_merge(const void* k, const void* v, long long stride_tok, lon
                          const Req* reqs, int n_req, int n_kv_heads, long long T,
                          long long total_units, const int* row_ptr, const int* ent_pos,
                          const float* ent_w, const int4* unit_first, int* slot_cnt, float* parts,
-                         int varlen_output, void* out_k, void* out_v, int* status, int num_sms,
-                         cudaStream_t stream);
+                         int varlen_output, long long out_stride_head, void* out_k, void* out_v,
+                         int* status, int num_sms, cudaStream_t stream);
+
+// Kept K and V rows of the requests whose mode is LOOKM_MERGE_NONE copied to the output cache
+// (eviction alone, Eq. 6-7); requests with another mode are left to the merge kernel.
+cudaError_t launch_compact_kept(const void* k, const void* v, long long stride_tok,
+                                long long stride_head, const Req* reqs, int n_req, int n_kv_heads,
+                                long long total_kept_rows, const int* kept_idx, int varlen_output,
+                                long long out_stride_head, void* out_k, void* out_v, int* status,
+                                cudaStream_t stream);
 
 // Launch with programmatic stream serialisation: the grid may be set up while the kernel before it
 // in the stream drains.  Every kernel launched this way starts with grid_dependency_wait(), which

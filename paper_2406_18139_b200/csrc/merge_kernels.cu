@@ -83,6 +83,7 @@ gather_kept_kernel(const __nv_bfloat16* __restrict__ k, long long stride_tok, lo
     const long long g = (long long)blockIdx.x * 16 + half;
     if (g >= total_rows) return;
     const Req& rq = find_req_by_slot(reqs, n_req, g);
+    if (rq.mode == LOOKM_MERGE_NONE) return;             // nothing is matched against its kept keys
     const long long u = g - rq.slot_begin;
     const int h = (int)(u / rq.B), slot = (int)(u % rq.B);
     const long long dst = rq.kept_off + (long long)h * rq.B + slot;
@@ -92,6 +93,34 @@ gather_kept_kernel(const __nv_bfloat16* __restrict__ k, long long stride_tok, lo
     const uint4 u4 = *reinterpret_cast<const uint4*>(k + tok * stride_tok + h * stride_head + l16 * 8);
     *reinterpret_cast<uint4*>(kept_keys + dst * kHeadDim + l16 * 8) = u4;
     if (l16 == 0) rnorm_kept[dst] = rnorm_all[(long long)h * T + tok];
+}
+
+// ---------------------------------------------------------------------------------------------
+// Eviction alone (Eq. 6-7): kept K and V rows of the requests with LOOKM_MERGE_NONE copied to the
+// output cache, one warp per row (lanes 0-15 the K row, 16-31 the V row).
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+compact_kept_kernel(const __nv_bfloat16* __restrict__ k, const __nv_bfloat16* __restrict__ v,
+                    long long stride_tok, long long stride_head, const Req* __restrict__ reqs, int n_req,
+                    int n_kv_heads, long long total_rows, const int* __restrict__ kept_idx,
+                    int varlen_output, long long out_stride_head, __nv_bfloat16* __restrict__ out_k,
+                    __nv_bfloat16* __restrict__ out_v, int* status) {
+    grid_dependency_wait();
+    const int lane = threadIdx.x & 31, l16 = lane & 15;
+    const long long g = (long long)blockIdx.x * 8 + (threadIdx.x >> 5);
+    if (g >= total_rows) return;
+    const Req& rq = find_req_by_slot(reqs, n_req, g);
+    if (rq.mode != LOOKM_MERGE_NONE) return;
+    const long long u = g - rq.slot_begin;
+    const int h = (int)(u / rq.B), slot = (int)(u % rq.B);
+    int pos = kept_idx[rq.kept_off + (long long)h * rq.B + slot];
+    if (pos < 0 || pos >= rq.L) { if (lane == 0) atomicExch(status, (int)LOOKM_ERR_DEVICE_BAD_INDEX); pos = 0; }
+    const __nv_bfloat16* src = (lane < 16 ? k : v) + (rq.tok_begin + (long long)pos) * stride_tok +
+                               (long long)h * stride_head + l16 * 8;
+    long long dst;
+    if (varlen_output) dst = (((long long)rq.out_begin + slot) * n_kv_heads + h) * kHeadDim;
+    else dst = (long long)h * out_stride_head + (long long)slot * kHeadDim;
+    *reinterpret_cast<uint4*>((lane < 16 ? out_k : out_v) + dst + l16 * 8) = *reinterpret_cast<const uint4*>(src);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -188,6 +217,7 @@ invert_assignment_kernel(const int* __restrict__ assign, const int* __restrict__
     __shared__ int warp_sums[32];
     grid_dependency_wait();
     const Req rq = reqs[blockIdx.y];
+    if (rq.mode == LOOKM_MERGE_NONE) return;             // its kept rows are copied, nothing is merged
     const int h = blockIdx.x;
     const int E = rq.E, B = rq.B;
     const long long ev_base = rq.ev_off + (long long)h * E;
@@ -454,8 +484,8 @@ merge_kernel(const __nv_bfloat16* __restrict__ k, const __nv_bfloat16* __restric
              int n_kv_heads, long long T, long long total_units, const int* __restrict__ row_ptr,
              const int* __restrict__ ent_pos, const float* __restrict__ ent_w,
              const int4* __restrict__ unit_first, int* __restrict__ slot_cnt, float* __restrict__ parts,
-             int varlen_output, __nv_bfloat16* __restrict__ out_k, __nv_bfloat16* __restrict__ out_v,
-             int* status) {
+             int varlen_output, long long out_stride_head, __nv_bfloat16* __restrict__ out_k,
+             __nv_bfloat16* __restrict__ out_v, int* status) {
     extern __shared__ uint8_t merge_smem_raw[];
     MergeShared& sh = *reinterpret_cast<MergeShared*>(
         (reinterpret_cast<uintptr_t>(merge_smem_raw) + 127) & ~static_cast<uintptr_t>(127));
@@ -543,10 +573,10 @@ merge_kernel(const __nv_bfloat16* __restrict__ k, const __nv_bfloat16* __restric
                 for (int i = 0; i < 8; ++i) o.v[i] = fmaf(wc, xc.v[i], wm * sum[i]) * inv;
                 result = pack8(o);
             }
-            long long row;
-            if (varlen_output) row = ((long long)rq.out_begin + c) * n_kv_heads + h;
-            else row = (long long)h * B + c;
-            *reinterpret_cast<uint4*>(dst_base + row * kHeadDim + l16 * 8) = result;
+            long long at;
+            if (varlen_output) at = (((long long)rq.out_begin + c) * n_kv_heads + h) * kHeadDim;
+            else at = (long long)h * out_stride_head + (long long)c * kHeadDim;
+            *reinterpret_cast<uint4*>(dst_base + at + l16 * 8) = result;
         };
         // ends the running piece: a whole slot is written out; a piece of a slot that other units
         // share goes to this unit's record (announced after the loop)
@@ -747,8 +777,8 @@ cudaError_t launch_merge(const void* k, const void* v, long long stride_tok, lon
                          const Req* reqs, int n_req, int n_kv_heads, long long T,
                          long long total_units, const int* row_ptr, const int* ent_pos,
                          const float* ent_w, const int4* unit_first, int* slot_cnt, float* parts,
-                         int varlen_output, void* out_k, void* out_v, int* status, int num_sms,
-                         cudaStream_t stream) {
+                         int varlen_output, long long out_stride_head, void* out_k, void* out_v,
+                         int* status, int num_sms, cudaStream_t stream) {
     if (total_units <= 0) return cudaSuccess;
     if (stride_tok <= 0 || stride_tok >= (1ll << 31)) return cudaErrorInvalidValue;   // byte stride kept in 32 bits
     const int smem = (int)sizeof(MergeShared) + 128;
@@ -759,7 +789,21 @@ cudaError_t launch_merge(const void* k, const void* v, long long stride_tok, lon
     return launch_chained(merge_kernel, dim3((unsigned)blocks), dim3(kMergeWarps * 32), (size_t)smem, stream,
                           (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, stride_tok, stride_head, reqs,
                           n_req, n_kv_heads, T, total_units, row_ptr, ent_pos, ent_w, unit_first, slot_cnt,
-                          parts, varlen_output, (__nv_bfloat16*)out_k, (__nv_bfloat16*)out_v, status);
+                          parts, varlen_output, out_stride_head, (__nv_bfloat16*)out_k, (__nv_bfloat16*)out_v,
+                          status);
+}
+
+cudaError_t launch_compact_kept(const void* k, const void* v, long long stride_tok,
+                                long long stride_head, const Req* reqs, int n_req, int n_kv_heads,
+                                long long total_kept_rows, const int* kept_idx, int varlen_output,
+                                long long out_stride_head, void* out_k, void* out_v, int* status,
+                                cudaStream_t stream) {
+    if (total_kept_rows <= 0) return cudaSuccess;
+    const long long blocks = (total_kept_rows + 7) / 8;
+    return launch_chained(compact_kept_kernel, dim3((unsigned)blocks), dim3(256), 0, stream,
+                          (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, stride_tok, stride_head, reqs,
+                          n_req, n_kv_heads, total_kept_rows, kept_idx, varlen_output, out_stride_head,
+                          (__nv_bfloat16*)out_k, (__nv_bfloat16*)out_v, status);
 }
 
 cudaError_t launch_argmax_rows(const float* sim_matrix, const Req* reqs, int n_req,

@@ -5,6 +5,8 @@
 // (is_text, score, lower position).  With n_text text candidates and N slots:
 //   n_text <= N : all text candidates are kept and the best N - n_text image candidates;
 //   n_text >  N : the best N text candidates are kept and no image candidate.
+// Without a mask (text prior off: Eq. 8 on the raw scores) every candidate is in the text class,
+// which reduces to a plain Top-N by score.
 // Either way one class is kept wholesale or not at all and the other needs an exact top-k, done
 // by a 4-pass radix select on an order-preserving 32-bit key; ties at the threshold go to the
 // lowest positions.  A final ordered pass writes the kept and evicted lists in ascending position.
@@ -136,7 +138,8 @@ select_kernel(const float* __restrict__ scores, const uint8_t* __restrict__ mask
     const Req rq = reqs[blockIdx.x / n_kv_heads];
     const int h = blockIdx.x % n_kv_heads;
     const float* s = scores + (long long)h * T + rq.tok_begin;
-    const uint8_t* msk = mask + rq.tok_begin;
+    const uint8_t* msk = mask ? mask + rq.tok_begin : nullptr;
+    auto is_image = [msk](int j) { return msk != nullptr && msk[j] != 0; };
     const int L = rq.L, B = rq.B, M = rq.M;
     const int N = B - M, nc = L - M;
 
@@ -151,13 +154,13 @@ select_kernel(const float* __restrict__ scores, const uint8_t* __restrict__ mask
         const int j = threadIdx.x + q * kSelThreads;
         ckey[q] = 0u;
         if (j < nc) {
-            const bool img = msk[j] != 0;
+            const bool img = is_image(j);
             ckey[q] = order_key(s[j]);
             cimg |= (img ? 1u : 0u) << q;
             cnt += !img;
         }
     }
-    for (int j = threadIdx.x + kKeyCache * kSelThreads; j < nc; j += kSelThreads) cnt += (msk[j] == 0);
+    for (int j = threadIdx.x + kKeyCache * kSelThreads; j < nc; j += kSelThreads) cnt += !is_image(j);
     {
         int e0, e1, t0, t1;
         block_scan2(cnt, 0, e0, e1, t0, t1, warp_tot);
@@ -187,7 +190,7 @@ select_kernel(const float* __restrict__ scores, const uint8_t* __restrict__ mask
                     atomicAdd(&hist[(ckey[q] >> shift) & 255u], 1);
             }
             for (int j = threadIdx.x + kKeyCache * kSelThreads; j < nc; j += kSelThreads) {
-                if ((msk[j] != 0) == (sel_cls != 0)) {
+                if (is_image(j) == (sel_cls != 0)) {
                     const unsigned key = order_key(s[j]);
                     if ((key & pmask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1);
                 }
@@ -246,7 +249,7 @@ select_kernel(const float* __restrict__ scores, const uint8_t* __restrict__ mask
                 if (j >= nc) {
                     keep[q] = 1;
                 } else {
-                    const int cls = (msk[j] != 0);
+                    const int cls = is_image(j);
                     if (cls != sel_cls) {
                         keep[q] = other_kept;
                     } else if (take_all) {

@@ -50,7 +50,8 @@ def test_host_side_argument_errors_need_no_device():
     assert lib.lookm_compress_layer(*args(L=0)) == B.ERR_INVALID_ARG
     assert lib.lookm_compress_layer(*args(B=0)) == B.ERR_INVALID_ARG
     assert lib.lookm_compress_layer(*args(M=-1)) == B.ERR_INVALID_ARG
-    assert lib.lookm_compress_layer(*args(mode=3)) == B.ERR_INVALID_ARG
+    assert lib.lookm_compress_layer(*args(mode=4)) == B.ERR_INVALID_ARG
+    assert lib.lookm_compress_layer(*args(mode=-1)) == B.ERR_INVALID_ARG
     assert lib.lookm_compress_layer(*args(lay=_layout(d=64))) == B.ERR_UNSUPPORTED
     assert lib.lookm_compress_layer(*args(q=C.c_void_p(264))) == B.ERR_INVALID_ARG   # 8-byte aligned only
     bad = _layout()
@@ -60,3 +61,47 @@ def test_host_side_argument_errors_need_no_device():
     assert lib.lookm_compress_layer(*args(ws=C.c_void_p(128))) == B.ERR_INVALID_ARG   # workspace alignment
     assert out_len.value == -1
     assert lib.lookm_device_status(None, None) == B.ERR_INVALID_ARG
+
+
+def test_misaligned_outputs_lists_and_bad_options_are_rejected_on_the_host():
+    lib = B.lib()
+    lay = _layout()
+    out_len = C.c_int(-1)
+    fake, odd16, odd4 = C.c_void_p(256), C.c_void_p(264), C.c_void_p(258)
+    # outputs are written with 16-byte stores
+    base = [fake, fake, fake, fake, 100, 20, 4, 0, C.byref(lay)]
+    tail = [C.byref(out_len), fake, 1 << 40, None]
+    assert lib.lookm_compress_layer(*base, odd16, fake, *tail) == B.ERR_INVALID_ARG
+    assert lib.lookm_compress_layer(*base, fake, odd16, *tail) == B.ERR_INVALID_ARG
+    # options: unknown flag bits, a misaligned log-sum-exp, a head stride below the dense one,
+    # a missing mask while the text prior is on
+    def opt_call(opt, mask=fake):
+        return lib.lookm_compress_layer_opt(fake, fake, fake, mask, 100, 20, 4, 0, C.byref(lay),
+                                            C.byref(opt), fake, fake, *tail)
+    assert opt_call(B.Options(2, None, 0)) == B.ERR_INVALID_ARG
+    assert opt_call(B.Options(0, 258, 0)) == B.ERR_INVALID_ARG
+    assert opt_call(B.Options(0, None, 20 * 128 - 8)) == B.ERR_INVALID_ARG
+    assert opt_call(B.Options(0, None, 20 * 128 + 4)) == B.ERR_INVALID_ARG
+    assert opt_call(B.Options(0, None, 0), mask=None) == B.ERR_INVALID_ARG
+    cu = (C.c_int * 2)(0, 100)
+    one = lambda v: (C.c_int * 1)(v)
+    # a varlen call takes no head stride
+    assert lib.lookm_compress_varlen_opt(fake, fake, fake, fake, cu, 1, one(20), one(4), one(0), C.byref(lay),
+                                         C.byref(B.Options(0, None, 4096)), fake, fake, None, fake, 1 << 40,
+                                         None) == B.ERR_INVALID_ARG
+    # index and weight lists are read as 32-bit words
+    merge = lambda kept=fake, sim=fake, outk=fake, mode=0: lib.lookm_merge(
+        fake, fake, kept, fake, fake, sim, cu, 1, one(20), one(mode), C.byref(lay), 0, outk, fake, fake, 1 << 40, None)
+    assert merge(kept=odd4) == B.ERR_INVALID_ARG
+    assert merge(sim=odd4) == B.ERR_INVALID_ARG
+    assert merge(outk=odd16) == B.ERR_INVALID_ARG
+    assert merge(sim=None) == B.ERR_INVALID_ARG                       # weights are needed to merge ...
+    noalloc = lambda kept=fake, outk=fake: lib.lookm_merge_noalloc(
+        fake, fake, kept, fake, fake, fake, cu, 1, one(20), one(0), C.byref(lay), 0, outk, fake, None)
+    assert noalloc(kept=odd4) == B.ERR_INVALID_ARG
+    assert noalloc(outk=odd16) == B.ERR_INVALID_ARG
+    sel = lambda scores=fake, kept=fake: lib.lookm_select(scores, fake, cu, 1, one(20), one(4), 32, kept, fake,
+                                                          None, fake, 1 << 40, None)
+    assert sel(scores=odd4) == B.ERR_INVALID_ARG
+    assert sel(kept=odd4) == B.ERR_INVALID_ARG
+    assert out_len.value == -1

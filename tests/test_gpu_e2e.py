@@ -23,11 +23,16 @@ def B():
     return binding
 
 
-def check_head(kf, vf, mask, h, budget, window, mode, A_h, kept_g, ev_g, asg_g, gk, gv, stats):
-    """Compare one head's GPU result (lists + merged rows) with the oracle; returns nothing."""
+def check_head(kf, vf, mask, h, budget, window, mode, A_h, kept_g, ev_g, asg_g, gk, gv, stats,
+               text_prior=True):
+    """Compare one head's GPU result (lists + merged rows) with the oracle; returns nothing.
+
+    mode 3 (eviction alone) has no assignment: the merged rows must then equal the kept rows."""
     L = len(mask)
+    if not text_prior:
+        mask = np.zeros_like(mask)                  # one class: the near-tie rule below needs no prior
     s32 = A_h.astype(np.float32).astype(np.float64)
-    kept_o, ev_o = orc.select(s32, mask, budget, window)
+    kept_o, ev_o = orc.select(s32, mask, budget, window, text_prior=text_prior)
     if not np.array_equal(kept_g, kept_o):
         only_g = np.setdiff1d(kept_g, kept_o)
         only_o = np.setdiff1d(kept_o, kept_g)
@@ -40,6 +45,10 @@ def check_head(kf, vf, mask, h, budget, window, mode, A_h, kept_g, ev_g, asg_g, 
         stats["kept_near_ties"] += 1
         kept_o, ev_o = kept_g, ev_g                 # downstream comparison on the GPU's lists
     assert np.array_equal(ev_g, ev_o)
+    if mode == 3:
+        assert np.array_equal(gk, kf[kept_o, h].astype(np.float64))
+        assert np.array_equal(gv, vf[kept_o, h].astype(np.float64))
+        return
     asg_o, sim_o, S = orc.match(kf, h, kept_o, ev_o, want_matrix=True)
     bad = np.where(asg_g != asg_o)[0]
     for e in bad:
