@@ -183,6 +183,54 @@ int lookm_merge(const void* k, const void* v, const int* kept_idx, const int* ev
                 int varlen_output, void* out_k, void* out_v, void* workspace,
                 size_t workspace_bytes, void* cuda_stream);
 
+/* ---- the step after the path: token generation over the compressed cache ----------------------
+ *
+ * One generation step of one layer (Section 3.1 "Token Generation", Eq. 2-3): the new token's key
+ * and value rows are appended to the cache (Eq. 2), then every query head attends over all rows of
+ * its KV head, the new one included:  out = softmax(q K^T * scale) V  (Eq. 3; no mask, every cached
+ * row precedes the new token; nothing is evicted any more).  The cache is the output of the calls
+ * above (rows after compression) or an uncompressed cache; bf16, head_dim 128.
+ *
+ * Row t of KV head h of request r lives at element
+ *     (cache_begin[r] + t) * cache_stride_row + h * cache_stride_head
+ * of cache_k / cache_v, which covers [n_kv_heads, capacity, 128] caches (stride_row = 128,
+ * stride_head = capacity * 128; see lookm_options.out_stride_head) and packed
+ * [rows, n_kv_heads, 128] caches (stride_row = n_kv_heads * 128, stride_head = 128).  Strides are
+ * multiples of 8 elements, base pointers 16-byte aligned.  The caller guarantees room for row
+ * cache_len (the appended one).  softmax_scale = 0 selects 1/sqrt(head_dim). */
+typedef struct {
+    int n_q_heads, n_kv_heads, head_dim;
+    long long cache_stride_row, cache_stride_head;
+    float softmax_scale;
+} lookm_cache_layout;
+
+/* Bytes of workspace (256-byte aligned) a generation step over caches of these lengths needs
+ * (partial results of the cache splits and their arrival counters); it grows with n_requests and
+ * n_q_heads, not with the cache lengths.  Returns 0 on invalid arguments. */
+size_t lookm_decode_workspace_size(const lookm_cache_layout* layout, int n_requests,
+                                   const int* cache_lens_host);
+
+/* One step for one request.
+ *   q             [n_q_heads, 128] bf16: the new token's query rows
+ *   k_new, v_new  [n_kv_heads, 128] bf16: its key and value rows; written to cache row cache_len
+ *                 (they must not lie inside the cache)
+ *   cache_k/_v    read (rows 0 .. cache_len - 1) and extended by one row; cache_len >= 0
+ *   out           [n_q_heads, 128] fp32
+ * Asynchronous on cuda_stream like every other call; calls that share a workspace must not overlap
+ * on the GPU.  Results do not depend on timing (fixed order of additions). */
+int lookm_decode_step(const void* q, const void* k_new, const void* v_new, void* cache_k,
+                      void* cache_v, int cache_len, const lookm_cache_layout* layout, float* out,
+                      void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* One step for a batch of requests with their own caches and lengths.
+ *   q [n_requests, n_q_heads, 128], k_new / v_new [n_requests, n_kv_heads, 128] bf16,
+ *   out [n_requests, n_q_heads, 128] fp32; cache_begin_host / cache_lens_host: n_requests entries. */
+int lookm_decode_step_varlen(const void* q, const void* k_new, const void* v_new, void* cache_k,
+                             void* cache_v, const long long* cache_begin_host,
+                             const int* cache_lens_host, int n_requests,
+                             const lookm_cache_layout* layout, float* out, void* workspace,
+                             size_t workspace_bytes, void* cuda_stream);
+
 /* Byte offsets, inside the workspace, of the intermediate results a whole-path call leaves behind
  * (layouts as described at the top: scores [n_kv_heads, T] fp32, lse [n_q_heads, T] fp32,
  * rank [n_kv_heads, T] i32, kept/evicted/assign lists i32, sim fp32).  They stay valid until

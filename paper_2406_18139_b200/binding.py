@@ -24,6 +24,7 @@ OPT_NO_TEXT_PRIOR = 1
 EXPORTS = ["lookm_workspace_size", "lookm_workspace_layout", "lookm_compress_layer", "lookm_compress_varlen",
            "lookm_compress_layer_opt", "lookm_compress_varlen_opt", "lookm_score",
            "lookm_select", "lookm_match", "lookm_match_from_sim", "lookm_merge",
+           "lookm_decode_workspace_size", "lookm_decode_step", "lookm_decode_step_varlen",
            "lookm_set_stage_events", "lookm_merge_noalloc", "lookm_noalloc_status", "lookm_device_status", "lookm_last_launch_count", "lookm_strerror"]
 N_STAGE_EVENTS = 8
 STAGE_NAMES = ["score_sweep1", "score_sweep2", "select_norms", "gather", "match", "invert", "merge"]
@@ -36,6 +37,12 @@ class WorkspaceOffsets(C.Structure):
 
 class Options(C.Structure):
     _fields_ = [("flags", C.c_uint), ("lse", C.c_void_p), ("out_stride_head", C.c_longlong)]
+
+
+class CacheLayout(C.Structure):
+    _fields_ = [("n_q_heads", C.c_int), ("n_kv_heads", C.c_int), ("head_dim", C.c_int),
+                ("cache_stride_row", C.c_longlong), ("cache_stride_head", C.c_longlong),
+                ("softmax_scale", C.c_float)]
 
 
 class Layout(C.Structure):
@@ -68,6 +75,14 @@ def lib():
                                                vp, vp, ip, vp, sz, vp]
         L.lookm_compress_varlen_opt.argtypes = [vp, vp, vp, vp, ip, C.c_int, ip, ip, ip, lp, op, vp, vp, ip,
                                                 vp, sz, vp]
+        cp = C.POINTER(CacheLayout)
+        L.lookm_decode_workspace_size.argtypes = [cp, C.c_int, ip]
+        L.lookm_decode_workspace_size.restype = sz
+        L.lookm_decode_step.argtypes = [vp, vp, vp, vp, vp, C.c_int, cp, vp, vp, sz, vp]
+        L.lookm_decode_step.restype = C.c_int
+        L.lookm_decode_step_varlen.argtypes = [vp, vp, vp, vp, vp, C.POINTER(C.c_longlong), ip, C.c_int, cp,
+                                               vp, vp, sz, vp]
+        L.lookm_decode_step_varlen.restype = C.c_int
         L.lookm_score.argtypes = [vp, vp, ip, C.c_int, lp, vp, vp, C.c_int, vp, sz, vp]
         L.lookm_select.argtypes = [vp, vp, ip, C.c_int, ip, ip, C.c_int, vp, vp, vp, vp, sz, vp]
         L.lookm_match.argtypes = [vp, vp, vp, ip, C.c_int, ip, lp, vp, vp, vp, sz, vp]
@@ -277,6 +292,34 @@ def lookm_merge_noalloc(k, v, kept_idx, evict_idx, assign, sim, cu_seqlens, budg
 
 def lookm_noalloc_status(stream=None) -> int:
     return lib().lookm_noalloc_status(_stream(stream))
+
+
+def lookm_decode_workspace_size(layout: CacheLayout, cache_lens: Sequence[int]) -> int:
+    return int(lib().lookm_decode_workspace_size(C.byref(layout), len(cache_lens), _ints(cache_lens)))
+
+
+def alloc_decode_workspace(layout: CacheLayout, n_requests: int = 1, device="cuda"):
+    import torch
+    n = lookm_decode_workspace_size(layout, [0] * n_requests)
+    if n == 0:
+        raise ValueError("lookm_decode_workspace_size rejected the layout")
+    return torch.empty(n, dtype=torch.uint8, device=device)
+
+
+def lookm_decode_step(q, k_new, v_new, cache_k, cache_v, cache_len, layout: CacheLayout, out, workspace,
+                      stream=None):
+    return lib().lookm_decode_step(_ptr(q), _ptr(k_new), _ptr(v_new), _ptr(cache_k), _ptr(cache_v),
+                                   int(cache_len), C.byref(layout), _ptr(out), _ptr(workspace),
+                                   workspace.numel() * workspace.element_size(), _stream(stream))
+
+
+def lookm_decode_step_varlen(q, k_new, v_new, cache_k, cache_v, cache_begin, cache_lens, layout: CacheLayout,
+                             out, workspace, stream=None):
+    begins = (C.c_longlong * len(cache_begin))(*[int(b) for b in cache_begin])
+    return lib().lookm_decode_step_varlen(_ptr(q), _ptr(k_new), _ptr(v_new), _ptr(cache_k), _ptr(cache_v),
+                                          begins, _ints(cache_lens), len(cache_lens), C.byref(layout),
+                                          _ptr(out), _ptr(workspace),
+                                          workspace.numel() * workspace.element_size(), _stream(stream))
 
 
 _stage_event_array = None

@@ -778,3 +778,142 @@ extern "C" int lookm_noalloc_status(void* cuda_stream) {
     LOOKM_TRY(noalloc_scratch_ptr(&scratch));
     return lookm_device_status(scratch, cuda_stream);
 }
+
+// ------------------------------------------------------------------------------------------------
+// Generation step over a cache (Section 3.1, Eq. 2-3): host planner of decode_kernel.cu.
+// ------------------------------------------------------------------------------------------------
+namespace {
+
+struct DecodePlan {
+    int n_req = 0, gt = 1, n_pass = 1, rows_per_split = 64;
+    std::vector<DecodeReq> reqs;            // caller order
+    size_t o_arrivals = 0, o_parts = 0, total = 0;
+};
+
+int decode_sms() {
+    DeviceInfo di;
+    return (device_info(di) == LOOKM_OK && di.sms > 0) ? di.sms : 148;
+}
+
+// lens may be NULL (sizing only).  The workspace is sized for the largest number of splits any
+// lengths can produce, so a cache may grow from step to step under one workspace.
+int build_decode_plan(DecodePlan& dp, const lookm_cache_layout* lay, int n_req, const long long* begins,
+                      const int* lens) {
+    if (!lay || n_req <= 0) return LOOKM_ERR_INVALID_ARG;
+    if (lay->head_dim != kHeadDim) return LOOKM_ERR_UNSUPPORTED;
+    if (lay->n_kv_heads <= 0 || lay->n_q_heads <= 0 || lay->n_q_heads % lay->n_kv_heads)
+        return LOOKM_ERR_INVALID_ARG;
+    if (lay->n_q_heads > 65535 || n_req > (1 << 20)) return LOOKM_ERR_UNSUPPORTED;
+    if (lay->cache_stride_row <= 0 || lay->cache_stride_head <= 0 || lay->cache_stride_row % 8 ||
+        lay->cache_stride_head % 8)
+        return LOOKM_ERR_INVALID_ARG;
+    if (!(lay->softmax_scale >= 0.f) || !std::isfinite(lay->softmax_scale)) return LOOKM_ERR_INVALID_ARG;
+    const int group = lay->n_q_heads / lay->n_kv_heads;
+    dp.n_req = n_req;
+    dp.gt = group % 8 == 0 ? 8 : group % 4 == 0 ? 4 : group % 2 == 0 ? 2 : 1;
+    dp.n_pass = group / dp.gt;
+    const long long units = (long long)lay->n_kv_heads * dp.n_pass;      // (KV head, pass) per request
+    const long long target_ctas = 4ll * decode_sms();
+    long long total_rows = 0;
+    if (lens) {
+        for (int r = 0; r < n_req; ++r) {
+            if (lens[r] < 0 || lens[r] >= (1 << 30) || (begins && begins[r] < 0)) return LOOKM_ERR_INVALID_ARG;
+            total_rows += ((long long)lens[r] + 1) * units;
+        }
+    }
+    long long s = (total_rows + target_ctas - 1) / target_ctas;
+    s = std::max<long long>(64, (s + 63) / 64 * 64);
+    if (s >= (1ll << 31)) return LOOKM_ERR_UNSUPPORTED;
+    dp.rows_per_split = (int)s;
+    // at most target_ctas + one ragged split per (request, KV head, pass)
+    const long long max_splits = target_ctas + (long long)n_req * units;
+    if (max_splits * dp.gt >= (1ll << 31)) return LOOKM_ERR_UNSUPPORTED;
+    if (lens) {
+        dp.reqs.resize(n_req);
+        long long parts = 0, arrivals = 0;
+        for (int r = 0; r < n_req; ++r) {
+            DecodeReq& q = dp.reqs[r];
+            q.begin = begins ? begins[r] : 0;
+            q.len = lens[r];
+            q.index = r;
+            q.n_splits = (int)(((long long)lens[r] + 1 + s - 1) / s);
+            q.cta_begin = 0;
+            q.part_begin = (int)parts;
+            q.arrival_begin = (int)arrivals;
+            parts += (long long)q.n_splits * units * dp.gt;
+            arrivals += units;
+        }
+    }
+    size_t o = 0;
+    auto carve = [&](size_t bytes) { size_t at = o; o = align_up(o + bytes, 256); return at; };
+    dp.o_arrivals = carve(4 * (size_t)n_req * (size_t)units);
+    dp.o_parts = carve(4 * (size_t)(kHeadDim + 2) * (size_t)max_splits * (size_t)dp.gt);
+    dp.total = o;
+    return LOOKM_OK;
+}
+
+int decode_common(const void* q, const void* k_new, const void* v_new, void* cache_k, void* cache_v,
+                  const long long* begins, const int* lens, int n_req, const lookm_cache_layout* lay,
+                  float* out, void* ws, size_t ws_bytes, void* stream) {
+    if (!q || !k_new || !v_new || !cache_k || !cache_v || !lens || !out) return LOOKM_ERR_INVALID_ARG;
+    for (const void* p : {q, k_new, v_new, (const void*)cache_k, (const void*)cache_v})
+        if (reinterpret_cast<uintptr_t>(p) & 15u) return LOOKM_ERR_INVALID_ARG;
+    LOOKM_TRY(check_word_ptrs({out}));
+    DecodePlan dp;
+    LOOKM_TRY(build_decode_plan(dp, lay, n_req, begins, lens));
+    if (!ws || (reinterpret_cast<uintptr_t>(ws) & 255u)) return LOOKM_ERR_INVALID_ARG;
+    if (ws_bytes < dp.total) return LOOKM_ERR_WORKSPACE_TOO_SMALL;
+    DeviceInfo di;
+    LOOKM_TRY(device_info(di));
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    g_launches = 0;
+    const float scale = lay->softmax_scale > 0.f ? lay->softmax_scale : 1.0f / std::sqrt((float)lay->head_dim);
+    int* arrivals = at<int>(ws, dp.o_arrivals);
+    const long long units = (long long)lay->n_kv_heads * dp.n_pass;
+    LOOKM_CUDA(cudaMemsetAsync(arrivals, 0, 4 * (size_t)n_req * (size_t)units, st));
+    for (int base = 0; base < n_req; base += kDecodeChunk) {
+        DecodeBatch batch;
+        std::memset(&batch, 0, sizeof(batch));
+        batch.n_req = std::min(kDecodeChunk, n_req - base);
+        long long ctas = 0;
+        for (int i = 0; i < batch.n_req; ++i) {
+            batch.r[i] = dp.reqs[base + i];
+            batch.r[i].cta_begin = (int)ctas;
+            ctas += (long long)batch.r[i].n_splits * units;
+        }
+        if (ctas >= (1ll << 31)) return LOOKM_ERR_UNSUPPORTED;
+        LOOKM_CUDA(launch_decode(batch, (int)ctas, dp.gt, q, k_new, v_new, cache_k, cache_v,
+                                 lay->cache_stride_row, lay->cache_stride_head, lay->n_q_heads,
+                                 lay->n_kv_heads, dp.rows_per_split, scale * 1.4426950408889634f,
+                                 at<float>(ws, dp.o_parts), arrivals, out, st));
+        ++g_launches;
+    }
+    return LOOKM_OK;
+}
+
+}  // namespace
+
+extern "C" size_t lookm_decode_workspace_size(const lookm_cache_layout* layout, int n_requests,
+                                              const int* cache_lens_host) {
+    DecodePlan dp;
+    if (build_decode_plan(dp, layout, n_requests, nullptr, cache_lens_host) != LOOKM_OK) return 0;
+    return dp.total;
+}
+
+extern "C" int lookm_decode_step(const void* q, const void* k_new, const void* v_new, void* cache_k,
+                                 void* cache_v, int cache_len, const lookm_cache_layout* layout,
+                                 float* out, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    const long long begin = 0;
+    return decode_common(q, k_new, v_new, cache_k, cache_v, &begin, &cache_len, 1, layout, out, workspace,
+                         workspace_bytes, cuda_stream);
+}
+
+extern "C" int lookm_decode_step_varlen(const void* q, const void* k_new, const void* v_new, void* cache_k,
+                                        void* cache_v, const long long* cache_begin_host,
+                                        const int* cache_lens_host, int n_requests,
+                                        const lookm_cache_layout* layout, float* out, void* workspace,
+                                        size_t workspace_bytes, void* cuda_stream) {
+    if (!cache_begin_host) return LOOKM_ERR_INVALID_ARG;
+    return decode_common(q, k_new, v_new, cache_k, cache_v, cache_begin_host, cache_lens_host, n_requests,
+                         layout, out, workspace, workspace_bytes, cuda_stream);
+}

@@ -136,6 +136,28 @@ cudaError_t launch_compact_kept(const void* k, const void* v, long long stride_t
                                 long long out_stride_head, void* out_k, void* out_v, int* status,
                                 cudaStream_t stream);
 
+// ---- generation step over a cache (decode_kernel.cu) --------------------------------------------
+// One request of a decode call as the kernel sees it; a launch carries up to kDecodeChunk of them
+// by value (no table in device memory, no copy that would synchronise the host).
+struct DecodeReq {
+    long long begin;      // first cache row of the request
+    int len;              // cached rows before the step
+    int index;            // position of the request in the caller's q / k_new / v_new / out arrays
+    int n_splits;         // CTAs per (KV head, pass)
+    int cta_begin;        // first CTA of the request in this launch
+    int part_begin;       // first partial-result record of the request in the workspace
+    int arrival_begin;    // first arrival counter of the request
+};
+constexpr int kDecodeChunk = 96;
+struct DecodeBatch { int n_req; int pad; DecodeReq r[kDecodeChunk]; };
+
+// gt: query heads handled per pass over the rows (1, 2, 4 or 8; divides the group size)
+cudaError_t launch_decode(const DecodeBatch& batch, int total_ctas, int gt, const void* q,
+                          const void* k_new, const void* v_new, void* cache_k, void* cache_v,
+                          long long stride_row, long long stride_head, int n_q_heads, int n_kv_heads,
+                          int rows_per_split, float scale_log2, float* parts, int* arrivals,
+                          float* out, cudaStream_t stream);
+
 // Launch with programmatic stream serialisation: the grid may be set up while the kernel before it
 // in the stream drains.  Every kernel launched this way starts with grid_dependency_wait(), which
 // returns once that kernel has completed and its writes are visible (a no-op for plain launches).

@@ -105,3 +105,23 @@ def test_misaligned_outputs_lists_and_bad_options_are_rejected_on_the_host():
     assert sel(scores=odd4) == B.ERR_INVALID_ARG
     assert sel(kept=odd4) == B.ERR_INVALID_ARG
     assert out_len.value == -1
+
+
+def test_decode_step_host_side_argument_errors():
+    lib = B.lib()
+    lay = B.CacheLayout(32, 8, 128, 128, 4096, 0.0)
+    fake = C.c_void_p(256)
+    call = lambda **kw: lib.lookm_decode_step(kw.get("q", fake), fake, fake, kw.get("ck", fake), fake,
+                                              kw.get("n", 10), C.byref(kw.get("lay", lay)), fake,
+                                              kw.get("ws", fake), kw.get("wsb", 1 << 30), None)
+    assert call(q=None) == B.ERR_INVALID_ARG
+    assert call(n=-1) == B.ERR_INVALID_ARG
+    assert call(ck=C.c_void_p(264)) == B.ERR_INVALID_ARG
+    assert call(lay=B.CacheLayout(32, 8, 64, 64, 4096, 0.0)) == B.ERR_UNSUPPORTED
+    assert call(lay=B.CacheLayout(32, 5, 128, 128, 4096, 0.0)) == B.ERR_INVALID_ARG
+    assert call(lay=B.CacheLayout(32, 8, 128, 130, 4096, 0.0)) == B.ERR_INVALID_ARG
+    assert call(wsb=16) == B.ERR_WORKSPACE_TOO_SMALL
+    assert call(ws=C.c_void_p(8)) == B.ERR_INVALID_ARG
+    assert B.lookm_decode_workspace_size(B.CacheLayout(32, 8, 64, 64, 4096, 0.0), [10]) == 0
+    n1 = B.lookm_decode_workspace_size(lay, [10])
+    assert n1 > 0 and n1 % 256 == 0 and B.lookm_decode_workspace_size(lay, [1 << 20]) == n1
