@@ -1,9 +1,10 @@
 """Benchmark of the LOOK-M prefill-time KV-cache compression path on B200.
 
-A step is one pass of the whole path (score -> select -> match -> merge/compact) over one layer
-of the 8192-token, 32-head LLaVA-1.5-7B-shaped synthetic prompt (budget 20 %, window 32, merge
-mode cycling averaged / pivotal / weighted).  The metric is prompt tokens x KV heads compressed
-per second.  One JSON line is printed by rank 0.
+A step is one pass of the whole path (score -> select -> match -> merge/compact) over the 32
+layers of the 8192-token, 32-head LLaVA-1.5-7B-shaped synthetic prompt (budget 20 %, window 32,
+merge mode cycling averaged / pivotal / weighted from layer to layer), one lookm_compress_layer
+call per layer.  The metric is prompt tokens x KV heads compressed per second.  One JSON line is
+printed by rank 0.
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
 
@@ -12,6 +13,7 @@ With N > 1 (launched by torch.distributed.run) every rank compresses its own rep
 workload (layers with different seeds); there is no data-path collective.
 """
 import argparse
+import hashlib
 import json
 import os
 import sys
@@ -28,15 +30,42 @@ from paper_2406_18139_b200 import synth  # noqa: E402
 
 METRIC = "prompt tokens*heads compressed/s per layer at 8K prompt"
 UNIT = "token*heads/s"
-N_INPUT_SETS = 3          # distinct layers rotated through, 192 MiB each (> the 126 MB L2)
+N_INPUT_SETS = 3          # distinct layers' inputs rotated through, 192 MiB each (> the 126 MB L2)
+SUSTAINED_ABOVE_S = 0.5   # a timed region at least this long is in the power-capped regime
+TRAFFIC_FILE = os.path.join(ROOT, "profiles", "tile_kernels_dram_traffic.txt")
+TILE_SOURCES = [os.path.join(ROOT, "paper_2406_18139_b200", "csrc", f) for f in ("tile_kernels.cu", "ptx.cuh")]
 
 
 def measured_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
         p = json.load(open(path))
-        return {"hbm_gbs": p["hbm_gbs"], "tflops": p["bf16_tflops_sustained"], "source": "measured"}
-    return {"hbm_gbs": 6650.0, "tflops": 1400.0, "source": "fallback"}
+        return {"hbm_gbs": p["hbm_gbs"], "tflops_burst": p["bf16_tflops"],
+                "tflops_sustained": p["bf16_tflops_sustained"], "source": "measured"}
+    return {"hbm_gbs": 6650.0, "tflops_burst": 1590.0, "tflops_sustained": 1400.0, "source": "fallback"}
+
+
+def tile_source_hash():
+    h = hashlib.sha256()
+    for path in TILE_SOURCES:
+        h.update(open(path, "rb").read())
+    return h.hexdigest()
+
+
+def captured_traffic():
+    """DRAM bytes per launch of the sweep kernels from the committed ncu capture, or None when the
+    kernel sources have changed since it was taken (the file records their hash)."""
+    if not os.path.exists(TRAFFIC_FILE):
+        return None
+    rec = {}
+    for line in open(TRAFFIC_FILE):
+        if ":" in line and not line.startswith("#"):
+            key, val = line.split(":", 1)
+            rec[key.strip()] = val.strip()
+    if rec.get("sha256_of_tile_sources") != tile_source_hash():
+        return None
+    return {"score_sweep1": float(rec["score_sweep1_bytes"]), "score_sweep2": float(rec["score_sweep2_bytes"]),
+            "tokens": float(rec["case_tokens"]), "heads": float(rec["case_heads"])}
 
 
 def workload(args=None):
@@ -149,9 +178,12 @@ def cpu_baseline(w, bits):
     cores = orc.default_threads()
     heads = list(range(min(cores, w.n_kv_heads)))
     sec, units = oracle_sample(w, heads, cores, bits)
+    sec1, units1 = oracle_sample(w, [0], 1, bits)
     return {"value": units / sec, "unit": UNIT, "cores": min(cores, len(heads)), "kind": "oracle",
-            "sample": "whole path on %d of %d KV heads of one 8192-token layer, one head per thread, %.1f s"
-                      % (len(heads), w.n_kv_heads, sec)}
+            "sample": "whole path on %d of %d KV heads of one %d-token layer, one head per thread, %.1f s"
+                      % (len(heads), w.n_kv_heads, w.requests[0].seq_len, sec),
+            "single_thread": {"value": units1 / sec1, "unit": UNIT, "cores": 1,
+                              "sample": "whole path on 1 KV head of the same layer, %.1f s" % sec1}}
 
 
 def run_reference(args):
@@ -177,8 +209,8 @@ def run_reference(args):
         step(i)
     sec = time.perf_counter() - t0
     value = args.steps * req.seq_len * len(heads) / sec
-    sample = "whole path on %d of %d KV heads of one 8192-token layer per step, one head per thread" % (
-        len(heads), w.n_kv_heads)
+    sample = "whole path on %d of %d KV heads of one %d-token layer per step, one head per thread" % (
+        len(heads), w.n_kv_heads, req.seq_len)
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * sec / args.steps,
@@ -211,6 +243,7 @@ def run_ours(args):
     w = workload(args)
     req = w.requests[0]
     L, Hq, Hkv, budget, window = req.seq_len, w.n_q_heads, w.n_kv_heads, req.budget, req.window
+    n_layers = args.layers or w.n_layers
     dev = lambda bits: torch.from_numpy(bits.view(np.int16)).cuda().view(torch.bfloat16)
     host_sets, dev_sets, first_bits = [], [], None
     for layer in rank_layers(rank):
@@ -226,9 +259,12 @@ def run_ours(args):
     out_k = torch.zeros(Hkv, budget, 128, dtype=torch.bfloat16, device="cuda")
     out_v = torch.zeros_like(out_k)
 
-    def step(i, tensors=None):
-        q, k, v = tensors if tensors is not None else dev_sets[i % N_INPUT_SETS]
-        st, _ = B.lookm_compress_layer(q, k, v, mask, L, budget, window, i % 3, lay, out_k, out_v, ws)
+    def layer_call(j, options=None, win=window, tensors=None, outs=None, msk=None):
+        """Layer j of the model: input set j mod 3, merge mode j mod 3."""
+        q, k, v = tensors if tensors is not None else dev_sets[j % N_INPUT_SETS]
+        ok, ov = outs if outs is not None else (out_k, out_v)
+        st, _ = B.lookm_compress_layer_opt(q, k, v, mask if msk is None else msk, L, budget, win, j % 3, lay,
+                                           options, ok, ov, ws)
         if st != B.OK:
             raise RuntimeError("lookm_compress_layer: " + B.lookm_strerror(st))
         return B.lookm_last_launch_count()
@@ -239,54 +275,164 @@ def run_ours(args):
             dist.barrier()
             torch.cuda.synchronize()
 
+    def new_events(n):
+        evs = [torch.cuda.Event(enable_timing=True) for _ in range(n)]
+        for e in evs:
+            e.record()
+        return evs
+
+    def timed_steps(n_steps, call):
+        """n_steps passes over the model's layers; returns (total ms, per-step ms list)."""
+        marks = new_events(n_steps + 1)
+        fence()
+        marks[0].record()
+        for i in range(n_steps):
+            for l in range(n_layers):
+                call(i * n_layers + l)
+            marks[i + 1].record()
+        fence()
+        per = [marks[i].elapsed_time(marks[i + 1]) for i in range(n_steps)]
+        return marks[0].elapsed_time(marks[n_steps]), per
+
     # ---- device-resident timing ------------------------------------------------------------------
     # Inside the timed region only the events around the two score sweeps (the dominant kernels)
-    # are recorded; every further event between two kernels costs about 2 us.  The full per-stage
-    # breakdown comes from a second, untimed pass below.
+    # are recorded; every further event between two kernels costs about 2 us.  The other stages
+    # come from a second pass of the same length below, i.e. in the same clock regime.
     n_ev = B.N_STAGE_EVENTS
-    stage_events = [[torch.cuda.Event(enable_timing=True) if s < 3 else None for s in range(n_ev)]
-                    for _ in range(args.steps)]
-    for evs in stage_events:
-        for e in evs:
-            if e is not None:
-                e.record()
+    n_calls = args.steps * n_layers
+    sweep_events = [new_events(3) + [None] * (n_ev - 3) for _ in range(n_calls)]
     for i in range(args.warmup):
-        step(i)
+        for l in range(n_layers):
+            layer_call(i * n_layers + l)
     B.check(B.lookm_device_status(ws))
     sampler = ClockSampler(physical_gpu_index(local_rank))
-    t_begin, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    launches = 0
-    fence()
+    launches = [0]
+
+    def main_call(j):
+        B.lookm_set_stage_events(sweep_events[j])
+        launches[0] += layer_call(j)
+
     sampler.start()
-    t_begin.record()
-    for i in range(args.steps):
-        B.lookm_set_stage_events(stage_events[i])
-        launches += step(i)
-    t_end.record()
-    fence()
+    ms_total, step_ms = timed_steps(args.steps, main_call)
     clocks = sampler.stop()
     B.lookm_set_stage_events(None)
     B.check(B.lookm_device_status(ws))
-    ms_total = t_begin.elapsed_time(t_end)
 
-    # ---- per-stage breakdown: same steps again with every stage event recorded (not timed) -----
-    n_detail = max(3, min(args.steps, 20))
-    detail_events = [[torch.cuda.Event(enable_timing=True) for _ in range(n_ev)] for _ in range(n_detail)]
-    for evs in detail_events:
-        for e in evs:
-            e.record()
-    fence()
-    for i in range(n_detail):
-        B.lookm_set_stage_events(detail_events[i])
-        step(i)
-    fence()
+    # ---- per-stage breakdown: the same steps again with every stage event recorded ---------------
+    n_detail_steps = max(1, min(args.steps, 10))
+    detail_events = [new_events(n_ev) for _ in range(n_detail_steps * n_layers)]
+
+    def detail_call(j):
+        B.lookm_set_stage_events(detail_events[j])
+        layer_call(j)
+
+    timed_steps(n_detail_steps, detail_call)
     B.lookm_set_stage_events(None)
 
+    # ---- variants of the path, each over the same steps (per-layer times, same regime) -----------
+    extra_steps = max(1, min(args.steps, 10))
+    # (a) the caller supplies the row log-sum-exp (as a prefill attention kernel leaves it), so the
+    #     first sweep is skipped: one lse tensor per input set, taken from a plain run
+    off = B.lookm_workspace_layout(lay, [L])
+    lse_sets = []
+    for s in range(N_INPUT_SETS):
+        layer_call(s)
+        torch.cuda.synchronize()
+        lse_sets.append(ws[off.lse:off.lse + 4 * Hq * L].view(torch.float32).clone())
+    lse_opts = [B.make_options(lse=t) for t in lse_sets]
+    ms_lse, _ = timed_steps(extra_steps, lambda j: layer_call(j, options=lse_opts[j % N_INPUT_SETS]))
+    # (b) the paper's own window rule: recent = important = 10 % of the prompt
+    win10 = int(0.1 * L)
+    ms_win, _ = timed_steps(extra_steps, lambda j: layer_call(j, win=win10))
+    # (c) eviction alone (no matching, no merging) and (d) no text prior
+    none_mode = lambda j: B.lookm_compress_layer(*dev_sets[j % N_INPUT_SETS], mask, L, budget, window,
+                                                 B.MERGE_NONE, lay, out_k, out_v, ws)
+    ms_none, _ = timed_steps(extra_steps, none_mode)
+    no_prior = B.make_options(no_text_prior=True)
+    ms_noprior, _ = timed_steps(extra_steps, lambda j: layer_call(j, options=no_prior))
+    B.check(B.lookm_device_status(ws))
+    # (e) all layers of the model in ONE launch sequence: the layers' tensors packed along the token
+    #     axis and handed to lookm_compress_varlen as n_layers requests
+    ms_batched = None
+    if n_layers > 1 and not args.no_batched:
+        cat = lambda i: torch.cat([dev_sets[l % N_INPUT_SETS][i] for l in range(n_layers)])
+        bq, bk, bv = cat(0), cat(1), cat(2)
+        bmask = mask.repeat(n_layers)
+        bws = B.alloc_workspace(lay, [L] * n_layers)
+        bok = torch.zeros(n_layers * budget, Hkv, 128, dtype=torch.bfloat16, device="cuda")
+        bov = torch.zeros_like(bok)
+        cu = [i * L for i in range(n_layers + 1)]
+        bargs = ([budget] * n_layers, [window] * n_layers, [l % 3 for l in range(n_layers)])
+
+        def batched():
+            st, _ = B.lookm_compress_varlen(bq, bk, bv, bmask, cu, *bargs, lay, bok, bov, bws)
+            if st != B.OK:
+                raise RuntimeError("lookm_compress_varlen: " + B.lookm_strerror(st))
+
+        for _ in range(2):
+            batched()
+        b0, b1 = new_events(2)
+        fence()
+        b0.record()
+        for _ in range(extra_steps):
+            batched()
+        b1.record()
+        fence()
+        B.check(B.lookm_device_status(bws))
+        ms_batched = b0.elapsed_time(b1) / extra_steps
+        del bq, bk, bv, bws, bok, bov
+
+    # ---- the step after the path: generation over the cache at the paper's three budgets ---------
+    # One token = one lookm_decode_step per layer over that layer's own cache (random bf16 rows, a
+    # cache per layer so that nothing is reused from L2 beyond what a real model would reuse).
+    decode = {}
+    if not args.no_decode:
+        tok_steps = 12
+        gen = torch.Generator(device="cuda")
+        gen.manual_seed(1234 + rank)
+        dq = torch.randn(Hq, 128, device="cuda", generator=gen).to(torch.bfloat16)
+        dkn = torch.randn(Hkv, 128, device="cuda", generator=gen).to(torch.bfloat16)
+        dvn = torch.randn(Hkv, 128, device="cuda", generator=gen).to(torch.bfloat16)
+        dout = torch.zeros(Hq, 128, dtype=torch.float32, device="cuda")
+        for ratio in (1.0, 0.2, 0.05):
+            n0 = int(ratio * L)
+            cap = n0 + tok_steps + 4
+            clay = B.CacheLayout(Hq, Hkv, 128, 128, cap * 128, 0.0)
+            dws = B.alloc_decode_workspace(clay)
+            caches = [(torch.randn(Hkv, cap, 128, device="cuda", generator=gen).to(torch.bfloat16),
+                       torch.randn(Hkv, cap, 128, device="cuda", generator=gen).to(torch.bfloat16))
+                      for _ in range(n_layers)]
+
+            def token(t):
+                for ck, cv in caches:
+                    st = B.lookm_decode_step(dq, dkn, dvn, ck, cv, n0 + t, clay, dout, dws)
+                    if st != B.OK:
+                        raise RuntimeError("lookm_decode_step: " + B.lookm_strerror(st))
+
+            for t in range(3):
+                token(t)
+            d0, d1 = new_events(2)
+            fence()
+            d0.record()
+            for t in range(3, tok_steps):
+                token(t)
+            d1.record()
+            fence()
+            ms_tok = d0.elapsed_time(d1) / (tok_steps - 3)
+            n_mid = n0 + (3 + tok_steps) // 2 + 1
+            bytes_layer = 2.0 * n_mid * 128 * 2 * Hkv
+            decode["%g%%" % (100 * ratio)] = {
+                "cache_rows": n0, "ms_per_token_all_layers": round(ms_tok, 4),
+                "us_per_layer": round(1e3 * ms_tok / n_layers, 2),
+                "gbs": round(bytes_layer * n_layers / (ms_tok * 1e-3) / 1e9, 1),
+                "kv_cache_gib_all_layers": round(2.0 * n0 * 128 * 2 * Hkv * n_layers / 2 ** 30, 3)}
+            del caches
+
     # ---- end to end through the public call with host buffers -----------------------------------
-    # Every step copies its inputs from pinned host memory, compresses, and copies the compacted
+    # Every layer copies its inputs from pinned host memory, compresses, and copies the compacted
     # cache back.  The three phases run on three streams with two sets of staging buffers, so
-    # the upload of step i + 1 and the download of step i - 1 overlap the kernels of step i (the
-    # PCIe link carries 201 MB up and 27 MB down per step and is the limit).
+    # the upload of layer i + 1 and the download of layer i - 1 overlap the kernels of layer i (the
+    # PCIe link carries 201 MB up and 27 MB down per layer and is the limit).
     n_sets = 2
     stage = [tuple(torch.empty_like(t) for t in dev_sets[0]) + (torch.empty_like(mask),) for _ in range(n_sets)]
     outs = [(torch.zeros_like(out_k), torch.zeros_like(out_v)) for _ in range(n_sets)]
@@ -297,7 +443,7 @@ def run_ours(args):
     run_done = [torch.cuda.Event() for _ in range(n_sets)]
     out_done = [torch.cuda.Event() for _ in range(n_sets)]
 
-    def e2e_step(i):
+    def e2e_layer(i):
         b = i % n_sets
         hq, hk, hv = host_sets[i % N_INPUT_SETS]
         sq, sk, sv, sm = stage[b]
@@ -309,25 +455,23 @@ def run_ours(args):
         with torch.cuda.stream(s_run):
             s_run.wait_event(in_ready[b])
             s_run.wait_event(out_done[b])                # its previous result has left the device
-            st, _ = B.lookm_compress_layer(sq, sk, sv, sm, L, budget, window, i % 3, lay, outs[b][0], outs[b][1], ws)
-            if st != B.OK:
-                raise RuntimeError("lookm_compress_layer: " + B.lookm_strerror(st))
+            layer_call(i, tensors=(sq, sk, sv), outs=outs[b], msk=sm)
             run_done[b].record(s_run)
         with torch.cuda.stream(s_out):
             s_out.wait_event(run_done[b])
             host_out[b][0].copy_(outs[b][0], non_blocking=True); host_out[b][1].copy_(outs[b][1], non_blocking=True)
             out_done[b].record(s_out)
 
-    e2e_steps = max(3, min(args.steps, 20))
+    e2e_steps = max(1, min(args.steps, 5))
     for i in range(2):
-        e2e_step(i)
+        e2e_layer(i)
     e_begin, e_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     fence()
     e_begin.record()
     for st_ in (s_in, s_run, s_out):
         st_.wait_event(e_begin)
-    for i in range(e2e_steps):
-        e2e_step(i)
+    for i in range(e2e_steps * n_layers):
+        e2e_layer(i)
     cur = torch.cuda.current_stream()
     for ev in out_done + run_done + in_ready:
         cur.wait_event(ev)
@@ -335,72 +479,109 @@ def run_ours(args):
     fence()
     e2e_ms = e_begin.elapsed_time(e_end)
     B.check(B.lookm_device_status(ws))
-    # the last step's download must equal what the device holds
-    last = (e2e_steps - 1) % n_sets
+    # the last layer's download must equal what the device holds
+    last = (e2e_steps * n_layers - 1) % n_sets
     if not torch.equal(host_out[last][0], outs[last][0].cpu()):
         raise RuntimeError("end-to-end result differs from the device result")
 
-    ms_total, e2e_ms = max_over_ranks([ms_total, e2e_ms], world, "cuda")
+    ms_total, e2e_ms, step_median = max_over_ranks([ms_total, e2e_ms, float(np.median(step_ms))], world, "cuda")
 
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
         return
 
-    units_per_step = L * Hkv
-    value = job_throughput(world, args.steps, units_per_step, ms_total)
+    # ---- the line --------------------------------------------------------------------------------
+    units_per_layer = L * Hkv
+    units_per_step = units_per_layer * n_layers
+    value = world * units_per_step / (step_median * 1e-3)          # from the median step
+    peaks = measured_peaks()
+    sustained = ms_total >= 1e3 * SUSTAINED_ABOVE_S or "sw_power_cap" in clocks["reasons"]
+    regime = "sustained" if sustained else "burst"
+    tf_peak = peaks["tflops_sustained"] if sustained else peaks["tflops_burst"]
     stage_ms = np.zeros(n_ev - 1)
     for evs in detail_events:
         for s in range(n_ev - 1):
             stage_ms[s] += evs[s].elapsed_time(evs[s + 1])
-    stage_ms /= n_detail
-    # the two sweeps as timed inside the timed region (these feed the roofline)
-    for s in range(2):
-        stage_ms[s] = sum(evs[s].elapsed_time(evs[s + 1]) for evs in stage_events) / args.steps
-    peaks = measured_peaks()
+    stage_ms /= len(detail_events)
+    for s in range(2):                                             # the sweeps as timed in the timed region
+        stage_ms[s] = sum(evs[s].elapsed_time(evs[s + 1]) for evs in sweep_events) / len(sweep_events)
     d = w.head_dim
-    sweep_flops = float(d) * L * (L + 1) * Hq                 # one causal QK^T over all query heads
+    sweep_flops = float(d) * L * (L + 1) * Hq                      # one causal QK^T over all query heads
     match_flops = 2.0 * (L - budget) * budget * d * Hkv
     merge_bytes = float(L + budget) * d * 2 * 2 * Hkv
-    names = B.STAGE_NAMES
-    stages = {}
-    for s, n in enumerate(names):
-        stages[n] = {"ms": round(float(stage_ms[s]), 4)}
+    stages = {n: {"ms": round(float(stage_ms[s]), 4)} for s, n in enumerate(B.STAGE_NAMES)}
+
+    def tensor_fracs(flops, ms):
+        tf = flops / (ms * 1e-3) / 1e12
+        return {"tflops": round(tf, 1), "frac": round(tf / tf_peak, 4),
+                "frac_of_burst": round(tf / peaks["tflops_burst"], 4),
+                "frac_of_sustained": round(tf / peaks["tflops_sustained"], 4)}
+
     for n in ("score_sweep1", "score_sweep2"):
-        tf = sweep_flops / (stages[n]["ms"] * 1e-3) / 1e12
-        stages[n].update({"tflops": round(tf, 1), "frac_of_%s_bf16" % peaks["source"]: round(tf / peaks["tflops"], 4)})
-    tf = match_flops / (stages["match"]["ms"] * 1e-3) / 1e12
-    stages["match"].update({"tflops": round(tf, 1), "frac_of_%s_bf16" % peaks["source"]: round(tf / peaks["tflops"], 4)})
+        stages[n].update(tensor_fracs(sweep_flops, stages[n]["ms"]))
+    stages["match"].update(tensor_fracs(match_flops, stages["match"]["ms"]))
     gbs = merge_bytes / (stages["merge"]["ms"] * 1e-3) / 1e9
-    stages["merge"].update({"gbs": round(gbs, 1), "frac_of_%s_hbm" % peaks["source"]: round(gbs / peaks["hbm_gbs"], 4)})
+    stages["merge"].update({"gbs": round(gbs, 1), "frac": round(gbs / peaks["hbm_gbs"], 4), "target": 0.70,
+                            "target_met": bool(gbs / peaks["hbm_gbs"] >= 0.70)})
     dom = max(("score_sweep1", "score_sweep2"), key=lambda n: stages[n]["ms"])
-    achieved = sweep_flops / (stages[dom]["ms"] * 1e-3) / 1e12
-    # DRAM traffic per launch of the dominant kernel: dram__bytes_read + write of one ncu capture
-    # on the 4096-token x 16-head case (profiles/tile_kernels_4096x16.txt), scaled by tokens x heads
-    # (the kernels read Q and K once from DRAM and re-read tiles from L2, so traffic grows with
-    # the input size).  Must be set to None when the tile kernels change after the capture.
-    captured = {"score_sweep1": 33.594624e6, "score_sweep2": 35.689984e6}
-    traffic = captured[dom] * (L * Hq) / (4096.0 * 16.0)
-    roofline = {"kernel": "tile_kernel<%s>" % dom, "bound": "tensor", "achieved": round(achieved, 2),
-                "peak": peaks["tflops"], "peak_source": peaks["source"] + " (cuBLAS bf16, sustained)",
-                "unit": "TFLOP/s", "frac": round(achieved / peaks["tflops"], 4), "traffic": traffic,
-                "traffic_unit": "bytes per launch (ncu capture of a 4096x16 case, scaled)"}
+    # the tensor pipe's own clock: a 128x128x128 bf16 tile keeps it busy for 512 clocks
+    n_sms = torch.cuda.get_device_properties(local_rank).multi_processor_count
+    nb = (L + 127) // 128
+    tiles_per_sm = Hq * nb * (nb + 1) / 2.0 / n_sms
+    pipe = None
+    if clocks["sm_mhz"]:
+        clocks_per_tile = stages[dom]["ms"] * 1e-3 * clocks["sm_mhz"] * 1e6 / tiles_per_sm
+        pipe = {"clocks_per_tile": round(clocks_per_tile, 1), "ideal_clocks_per_tile": 512,
+                "frac_of_tensor_pipe_at_sampled_clock": round(512.0 / clocks_per_tile, 4),
+                "target": 0.50, "target_met": bool(512.0 / clocks_per_tile >= 0.50)}
+    cap = captured_traffic()
+    traffic = cap[dom] * (L * Hq) / (cap["tokens"] * cap["heads"]) if cap else None
+    roofline = {"kernel": "tile_kernel<%s>" % dom, "bound": "tensor", "achieved": stages[dom]["tflops"],
+                "peak": tf_peak, "peak_source": "%s (cuBLAS bf16, %s: timed region %.2f s, reasons %s)"
+                % (peaks["source"], regime, ms_total * 1e-3, clocks["reasons"]),
+                "unit": "TFLOP/s", "frac": stages[dom]["frac"], "frac_of_burst": stages[dom]["frac_of_burst"],
+                "frac_of_sustained": stages[dom]["frac_of_sustained"], "tensor_pipe": pipe, "traffic": traffic,
+                "traffic_unit": "bytes per launch (ncu capture of a smaller case scaled by tokens x heads; "
+                                "null when the kernel sources changed after the capture)",
+                "others": {"merge": stages["merge"], "match": stages["match"]}}
+    for v in decode.values():
+        v["frac_of_hbm"] = round(v["gbs"] / peaks["hbm_gbs"], 4)
+    if decode:
+        full = decode["100%"]["ms_per_token_all_layers"]
+        for v in decode.values():
+            v["speedup_vs_full_cache"] = round(full / v["ms_per_token_all_layers"], 2)
+        roofline["others"]["decode_full_cache"] = {"gbs": decode["100%"]["gbs"], "frac": decode["100%"]["frac_of_hbm"]}
+    per_layer = lambda ms: {"ms_per_layer": round(ms / (extra_steps * n_layers), 4),
+                            "value": round(units_per_layer / (ms / (extra_steps * n_layers) * 1e-3), 1)}
+    variants = {"lse_supplied": per_layer(ms_lse), "window_rule_10pct": per_layer(ms_win),
+                "evict_only": per_layer(ms_none), "no_text_prior": per_layer(ms_noprior)}
+    if ms_batched is not None:
+        variants["all_layers_one_launch_sequence"] = {"ms_per_layer": round(ms_batched / n_layers, 4),
+                                                      "value": round(units_per_step / (ms_batched * 1e-3), 1)}
     e2e_value = job_throughput(world, e2e_steps, units_per_step, e2e_ms)
-    h2d = sum(t.numel() * t.element_size() for t in host_sets[0]) + mask_host.numel()
-    d2h = (out_k.numel() + out_v.numel()) * 2
+    h2d = (sum(t.numel() * t.element_size() for t in host_sets[0]) + mask_host.numel()) * n_layers
+    d2h = (out_k.numel() + out_v.numel()) * 2 * n_layers
     out = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-        "warmup": args.warmup, "ms_per_step": ms_total / args.steps, "higher_is_better": True,
+        "warmup": args.warmup, "ms_per_step": step_median, "ms_per_step_mean": ms_total / args.steps,
+        "ms_per_layer": step_median / n_layers, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": w.name, "seq_len": L, "n_q_heads": Hq, "n_kv_heads": Hkv, "head_dim": d,
-                   "budget": budget, "window": window, "merge_mode": "average/pivotal/weighted by step",
+        "config": {"workload": w.name, "layers_per_step": n_layers, "seq_len": L, "n_q_heads": Hq,
+                   "n_kv_heads": Hkv, "head_dim": d, "budget": budget, "window": window,
+                   "merge_mode": "average/pivotal/weighted by layer",
                    "l2": "inputs rotate over %d layers of 192 MiB each, larger than L2" % N_INPUT_SETS,
-                   "parallelism": "replicas x%d" % world},
-        "clocks": clocks, "gpu_launches": launches,
+                   "value_from": "median step", "parallelism": "replicas x%d" % world},
+        "clocks": clocks, "gpu_launches": launches[0],
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "steps": e2e_steps, "ms_per_step": e2e_ms / e2e_steps},
         "roofline": roofline, "stages": stages,
-        "stages_note": "sweeps timed inside the timed region; other stages from a second pass with all stage events",
+        "stages_note": "per layer; sweeps timed inside the timed region, other stages from a second pass of "
+                       "%d steps with all stage events (same regime)" % n_detail_steps,
+        "variants": variants, "decode": decode,
+        "decode_note": "synthetic caches; attention over the cache only (Eq. 2-3), 32 layers per token; "
+                       "the paper's table (28.16 / 20.98 / 18.22 ms per token, 1.52 / 0.32 / 0.13 GiB on an "
+                       "RTX 3090) times the whole model",
     }
     if world == 1 and not args.no_cpu_baseline:
         out["cpu_baseline"] = cpu_baseline(w, first_bits)
@@ -416,13 +597,16 @@ def main():
     ap.add_argument("--warmup", type=int, default=None)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-decode", action="store_true")
+    ap.add_argument("--no-batched", action="store_true")
+    ap.add_argument("--layers", type=int, default=0, help="layers per step (default: the model's 32)")
     ap.add_argument("--seq-len", type=int, default=0, help="reduced prompt length (profiling only)")
     ap.add_argument("--heads", type=int, default=0, help="reduced head count (profiling only)")
     args = ap.parse_args()
     if args.steps is None:
-        args.steps = 60 if args.impl == "ours" else 5
+        args.steps = 20 if args.impl == "ours" else 5
     if args.warmup is None:
-        args.warmup = 5 if args.impl == "ours" else 1
+        args.warmup = 3 if args.impl == "ours" else 1
     if args.impl == "ours":
         args.warmup = max(args.warmup, 3)
     if args.impl == "reference":
