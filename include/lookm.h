@@ -19,8 +19,12 @@
  *     B_r = min(budget_r, L_r) and E_r = L_r - B_r, the list of (request r, KV head h) starts at
  *     element  n_kv_heads * sum_{r'<r} B_r' + h * B_r   (kept lists) or
  *              n_kv_heads * sum_{r'<r} E_r' + h * E_r   (evicted, assign and sim arrays).
- *   - Every buffer is owned by the caller.  The library allocates nothing, keeps no state between
- *     calls, never modifies inputs; outputs and workspace must not overlap inputs.  `workspace`
+ *   - Every buffer is owned by the caller.  The library allocates nothing and never modifies
+ *     inputs; outputs and workspace must not overlap inputs.  No result depends on an earlier
+ *     call: the only state kept between calls is per host thread and diagnostic (the event handles
+ *     given to lookm_set_stage_events and the launch count lookm_last_launch_count returns), plus
+ *     per-device facts cached on first use (SM count, kernel attributes, the address of the
+ *     lookm_merge_noalloc scratch).  `workspace`
  *     must be 256-byte aligned and at least lookm_workspace_size() bytes; its first bytes hold
  *     the device status word.  Calls that share a workspace must not overlap on the GPU.
  *   - Work is enqueued on `cuda_stream` (a cudaStream_t; NULL = default stream) and the call
@@ -205,7 +209,7 @@ typedef struct {
 } lookm_cache_layout;
 
 /* Bytes of workspace (256-byte aligned) a generation step over caches of these lengths needs
- * (partial results of the cache splits and their arrival counters); it grows with n_requests and
+ * (partial results of the cache splits); it grows with n_requests and
  * n_q_heads, not with the cache lengths.  Returns 0 on invalid arguments. */
 size_t lookm_decode_workspace_size(const lookm_cache_layout* layout, int n_requests,
                                    const int* cache_lens_host);
@@ -289,6 +293,14 @@ int lookm_set_stage_events(void* const* events_host, int n_events);
  * of `workspace` (LOOKM_OK if no kernel reported a problem since the last call that used this
  * workspace began). */
 int lookm_device_status(void* workspace, void* cuda_stream);
+
+/* Self-test of what happens when a device-side wait runs out (deployment aid; Eq. 4-12 contain no
+ * waits, so the paper has nothing to cite here).  Enqueues one CTA that waits, with the very wait
+ * routine and abort protocol of the tensor-core kernels and a limit of `limit_us` microseconds
+ * (1 .. 100000), on a barrier at which nobody ever arrives.  The wait expires, the CTA returns, and
+ * lookm_device_status(workspace, stream) then reports LOOKM_ERR_DEVICE_TIMEOUT; the CUDA context
+ * stays usable.  workspace: at least 256 bytes, 256-byte aligned (only its status word is used). */
+int lookm_selftest_wait_expiry(int limit_us, void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /* Number of kernels the last call on this host thread enqueued (for launch accounting). */
 int lookm_last_launch_count(void);

@@ -13,7 +13,7 @@ import os
 from typing import Optional, Sequence
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.environ.get("LOOKM_LIB", os.path.join(_HERE, "liblookm.so"))   # LOOKM_LIB: another build of the same library
+LIB_PATH = os.path.join(_HERE, "liblookm.so")     # the in-tree build, nothing else
 _lib = None
 
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE_TOO_SMALL, ERR_CUDA, ERR_DEVICE_TIMEOUT, \
@@ -25,7 +25,7 @@ EXPORTS = ["lookm_workspace_size", "lookm_workspace_layout", "lookm_compress_lay
            "lookm_compress_layer_opt", "lookm_compress_varlen_opt", "lookm_score",
            "lookm_select", "lookm_match", "lookm_match_from_sim", "lookm_merge",
            "lookm_decode_workspace_size", "lookm_decode_step", "lookm_decode_step_varlen",
-           "lookm_set_stage_events", "lookm_merge_noalloc", "lookm_noalloc_status", "lookm_device_status", "lookm_last_launch_count", "lookm_strerror"]
+           "lookm_set_stage_events", "lookm_selftest_wait_expiry", "lookm_merge_noalloc", "lookm_noalloc_status", "lookm_device_status", "lookm_last_launch_count", "lookm_strerror"]
 N_STAGE_EVENTS = 8
 STAGE_NAMES = ["score_sweep1", "score_sweep2", "select_norms", "gather", "match", "invert", "merge"]
 
@@ -91,6 +91,8 @@ def lib():
                                   vp, sz, vp]
         L.lookm_set_stage_events.argtypes = [C.POINTER(C.c_void_p), C.c_int]
         L.lookm_set_stage_events.restype = C.c_int
+        L.lookm_selftest_wait_expiry.argtypes = [C.c_int, vp, sz, vp]
+        L.lookm_selftest_wait_expiry.restype = C.c_int
         L.lookm_merge_noalloc.argtypes = [vp, vp, vp, vp, vp, vp, ip, C.c_int, ip, ip, lp, C.c_int, vp, vp, vp]
         L.lookm_merge_noalloc.restype = C.c_int
         L.lookm_noalloc_status.argtypes = [vp]
@@ -335,6 +337,11 @@ def lookm_set_stage_events(events) -> int:
     arr = (C.c_void_p * len(events))(*[(e.cuda_event if e is not None else None) for e in events])
     _stage_event_array = arr                     # the library keeps the pointer: keep it alive
     return lib().lookm_set_stage_events(arr, len(events))
+
+
+def lookm_selftest_wait_expiry(limit_us: int, workspace, stream=None) -> int:
+    return lib().lookm_selftest_wait_expiry(int(limit_us), _ptr(workspace),
+                                            workspace.numel() * workspace.element_size(), _stream(stream))
 
 
 def lookm_device_status(workspace, stream=None) -> int:

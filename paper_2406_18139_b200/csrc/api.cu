@@ -675,6 +675,20 @@ int lookm_device_status(void* workspace, void* cuda_stream) {
     return word;
 }
 
+int lookm_selftest_wait_expiry(int limit_us, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    if (limit_us < 1 || limit_us > 100000) return LOOKM_ERR_INVALID_ARG;
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u)) return LOOKM_ERR_INVALID_ARG;
+    if (workspace_bytes < 256) return LOOKM_ERR_WORKSPACE_TOO_SMALL;
+    DeviceInfo di;
+    LOOKM_TRY(device_info(di));
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    g_launches = 0;
+    LOOKM_CUDA(cudaMemsetAsync(workspace, 0, 256, st));
+    LOOKM_CUDA(launch_wait_probe(1000ull * (unsigned long long)limit_us, static_cast<int*>(workspace), st));
+    ++g_launches;
+    return LOOKM_OK;
+}
+
 int lookm_last_launch_count(void) { return g_launches; }
 
 int lookm_set_stage_events(void* const* events_host, int n_events) {
@@ -787,7 +801,7 @@ namespace {
 struct DecodePlan {
     int n_req = 0, gt = 1, n_pass = 1, rows_per_split = 64;
     std::vector<DecodeReq> reqs;            // caller order
-    size_t o_arrivals = 0, o_parts = 0, total = 0;
+    size_t o_parts = 0, total = 0;
 };
 
 int decode_sms() {
@@ -813,24 +827,46 @@ int build_decode_plan(DecodePlan& dp, const lookm_cache_layout* lay, int n_req, 
     dp.gt = group % 8 == 0 ? 8 : group % 4 == 0 ? 4 : group % 2 == 0 ? 2 : 1;
     dp.n_pass = group / dp.gt;
     const long long units = (long long)lay->n_kv_heads * dp.n_pass;      // (KV head, pass) per request
-    const long long target_ctas = 4ll * decode_sms();
-    long long total_rows = 0;
+    const int sms = decode_sms();
+    // The grid is one wave: as many CTAs as the GPU holds at a time (a second, partly filled wave
+    // would cost as much as the first).  Rows per split: the smallest count with which the splits
+    // of all requests fit into that wave.
+    long long s = 16;
     if (lens) {
+        const int per_sm = decode_ctas_per_sm(dp.gt);
+        const long long wave = (long long)sms * (per_sm > 0 ? per_sm : 2);
+        long long total_rows = 0;
         for (int r = 0; r < n_req; ++r) {
             if (lens[r] < 0 || lens[r] >= (1 << 30) || (begins && begins[r] < 0)) return LOOKM_ERR_INVALID_ARG;
             total_rows += ((long long)lens[r] + 1) * units;
         }
+        auto ctas_with = [&](long long rows) {
+            long long c = 0;
+            for (int r = 0; r < n_req; ++r) c += (((long long)lens[r] + rows) / rows) * units;
+            return c;
+        };
+        s = std::max<long long>(16, (total_rows + wave - 1) / wave);
+        if (ctas_with(s) > wave) {
+            // smallest count in (s, longest cache + 1] that fits (the CTA count never grows with
+            // it); with the upper end every request is a single split, the least there can be
+            long long lo = s, hi = s;
+            for (int r = 0; r < n_req; ++r) hi = std::max<long long>(hi, (long long)lens[r] + 1);
+            while (lo < hi) {
+                const long long mid = lo + (hi - lo) / 2;
+                if (ctas_with(mid) > wave) lo = mid + 1; else hi = mid;
+            }
+            s = lo;
+        }
     }
-    long long s = (total_rows + target_ctas - 1) / target_ctas;
-    s = std::max<long long>(64, (s + 63) / 64 * 64);
     if (s >= (1ll << 31)) return LOOKM_ERR_UNSUPPORTED;
     dp.rows_per_split = (int)s;
-    // at most target_ctas + one ragged split per (request, KV head, pass)
-    const long long max_splits = target_ctas + (long long)n_req * units;
+    // at most one wave of the fullest kernel, or one (short) split per (request, KV head, pass)
+    // when the batch alone has more units than a wave holds
+    const long long max_splits = (long long)kDecodeMaxCtasPerSm * sms + (long long)n_req * units;
     if (max_splits * dp.gt >= (1ll << 31)) return LOOKM_ERR_UNSUPPORTED;
     if (lens) {
         dp.reqs.resize(n_req);
-        long long parts = 0, arrivals = 0;
+        long long parts = 0;
         for (int r = 0; r < n_req; ++r) {
             DecodeReq& q = dp.reqs[r];
             q.begin = begins ? begins[r] : 0;
@@ -839,14 +875,12 @@ int build_decode_plan(DecodePlan& dp, const lookm_cache_layout* lay, int n_req, 
             q.n_splits = (int)(((long long)lens[r] + 1 + s - 1) / s);
             q.cta_begin = 0;
             q.part_begin = (int)parts;
-            q.arrival_begin = (int)arrivals;
+            q.pad = 0;
             parts += (long long)q.n_splits * units * dp.gt;
-            arrivals += units;
         }
     }
     size_t o = 0;
     auto carve = [&](size_t bytes) { size_t at = o; o = align_up(o + bytes, 256); return at; };
-    dp.o_arrivals = carve(4 * (size_t)n_req * (size_t)units);
     dp.o_parts = carve(4 * (size_t)(kHeadDim + 2) * (size_t)max_splits * (size_t)dp.gt);
     dp.total = o;
     return LOOKM_OK;
@@ -868,25 +902,30 @@ int decode_common(const void* q, const void* k_new, const void* v_new, void* cac
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     g_launches = 0;
     const float scale = lay->softmax_scale > 0.f ? lay->softmax_scale : 1.0f / std::sqrt((float)lay->head_dim);
-    int* arrivals = at<int>(ws, dp.o_arrivals);
     const long long units = (long long)lay->n_kv_heads * dp.n_pass;
-    LOOKM_CUDA(cudaMemsetAsync(arrivals, 0, 4 * (size_t)n_req * (size_t)units, st));
     for (int base = 0; base < n_req; base += kDecodeChunk) {
         DecodeBatch batch;
         std::memset(&batch, 0, sizeof(batch));
         batch.n_req = std::min(kDecodeChunk, n_req - base);
         long long ctas = 0;
+        bool split = false;
         for (int i = 0; i < batch.n_req; ++i) {
             batch.r[i] = dp.reqs[base + i];
             batch.r[i].cta_begin = (int)ctas;
             ctas += (long long)batch.r[i].n_splits * units;
+            split = split || batch.r[i].n_splits > 1;
         }
         if (ctas >= (1ll << 31)) return LOOKM_ERR_UNSUPPORTED;
         LOOKM_CUDA(launch_decode(batch, (int)ctas, dp.gt, q, k_new, v_new, cache_k, cache_v,
                                  lay->cache_stride_row, lay->cache_stride_head, lay->n_q_heads,
                                  lay->n_kv_heads, dp.rows_per_split, scale * 1.4426950408889634f,
-                                 at<float>(ws, dp.o_parts), arrivals, out, st));
+                                 at<float>(ws, dp.o_parts), out, st));
         ++g_launches;
+        if (split) {
+            LOOKM_CUDA(launch_decode_combine(batch, dp.gt, lay->n_q_heads, lay->n_kv_heads,
+                                             scale * 1.4426950408889634f, at<float>(ws, dp.o_parts), out, st));
+            ++g_launches;
+        }
     }
     return LOOKM_OK;
 }

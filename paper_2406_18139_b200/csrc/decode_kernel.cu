@@ -6,14 +6,16 @@
 // The step is bound by HBM bandwidth: every cached K and V row (256 bytes each) is read exactly
 // once per step, whatever the number of query heads in the group, and nothing else of any size
 // moves.  The rows of a (request, KV head) are cut into splits of `rows_per_split` rows (chosen
-// per call so that the grid fills the GPU a few times over); a CTA of 8 warps takes one split:
-// half a warp owns a row (16 bytes per lane), four rows per half-warp are in flight at a time, the
-// dot products are reduced with four shuffles, and each half-warp keeps its own running softmax
-// statistics (reference maximum, sum, weighted V sum) for every query head of the group in
-// registers.  Half-warps and warps are combined through shared memory in a fixed order; with more
-// than one split the CTA leaves its partial result in the workspace and the CTA that arrives last
-// at the (request, KV head) adds the splits in split order.  No CTA waits for another and the
-// order of additions never depends on timing, so results are reproducible bit for bit.
+// per call so that the grid is one wave of resident CTAs); a CTA of 8 warps takes one split: half a
+// warp owns a row (16 bytes per lane).  Rows travel global -> shared memory with 16-byte cp.async
+// copies into a ring private to each warp (a step = four K and four V rows per half-warp; the
+// steps ahead are in flight while one is worked on, and every lane reads back exactly the bytes it
+// copied, so cp.async.wait_group is all the synchronisation there is).  The dot products are
+// reduced with four shuffles, and each half-warp keeps its own running softmax statistics
+// (reference maximum, sum, weighted V sum) for every query head of the group in registers.  Half-warps and warps are combined through shared memory in a fixed order; with more
+// than one split the CTA leaves its partial result in the workspace and a second kernel, chained
+// behind the first, adds the splits in split order.  No CTA waits for another and the order of
+// additions never depends on timing, so results are reproducible bit for bit.
 #include <cuda_bf16.h>
 #include <math.h>
 
@@ -22,10 +24,20 @@
 namespace lookm {
 namespace {
 
-constexpr int kDecThreads = 256;
+constexpr int kDecThreads = kDecodeThreads;
 constexpr int kDecWarps = kDecThreads / 32;
 constexpr int kDecHalfWarps = 2 * kDecWarps;         // rows a CTA has in hand at once
-constexpr int kDecFlight = 4;                        // rows in flight per half-warp
+#ifndef LOOKM_DEC_FLIGHT
+#define LOOKM_DEC_FLIGHT 4
+#endif
+#ifndef LOOKM_DEC_RING
+#define LOOKM_DEC_RING 4
+#endif
+constexpr int kDecFlight = LOOKM_DEC_FLIGHT;         // rows per half-warp and step
+constexpr int kDecRing = LOOKM_DEC_RING;             // steps in the ring of a warp (all but one in flight)
+constexpr int kDecRowBytes = kHeadDim * 2;
+constexpr int kDecStepBytes = 2 * kDecFlight * 2 * kDecRowBytes;   // per warp: [half][row][K|V][256 B]
+constexpr int kDecRingBytes = kDecWarps * kDecRing * kDecStepBytes;
 
 __device__ __forceinline__ void unpack_bf16x8(const uint4& u, float (&x)[8]) {
     const unsigned w[4] = {u.x, u.y, u.z, u.w};
@@ -47,7 +59,6 @@ struct DecShared {
     float m[kDecWarps][GT];                          // [warp][query head of the pass]
     float l[kDecWarps][GT];
     float o[kDecWarps][GT][kHeadDim];
-    int last;
 };
 
 // GT query heads of the group are handled per pass over the rows (GT divides the group size).
@@ -57,9 +68,9 @@ decode_kernel(const __grid_constant__ DecodeBatch batch, const __nv_bfloat16* __
               const __nv_bfloat16* __restrict__ k_new, const __nv_bfloat16* __restrict__ v_new,
               __nv_bfloat16* __restrict__ cache_k, __nv_bfloat16* __restrict__ cache_v,
               long long stride_row, long long stride_head, int n_q_heads, int n_kv_heads, int group,
-              int rows_per_split, float scale_log2, float* __restrict__ parts, int* __restrict__ arrivals,
-              float* __restrict__ out) {
+              int rows_per_split, float scale_log2, float* __restrict__ parts, float* __restrict__ out) {
     __shared__ DecShared<GT> sh;
+    extern __shared__ __align__(128) uint8_t dec_ring[];         // [warp][ring step][half][row][K|V][256 B]
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int hw = threadIdx.x >> 4, l16 = lane & 15;
 
@@ -107,31 +118,60 @@ decode_kernel(const __grid_constant__ DecodeBatch batch, const __nv_bfloat16* __
         for (int i = 0; i < 8; ++i) o[g][i] = 0.f;
     }
 
-    // the loop bound does not depend on the half-warp, so both halves of a warp reach the shuffles
-    for (int base = row0; base < row1; base += kDecHalfWarps * kDecFlight) {
+    // The appended row (Eq. 2) is read from k_new / v_new by whoever owns it; the CTA that owns it
+    // on the group's first pass also writes it into the cache (nobody reads cache row `len` in this
+    // step, so the write races with nothing).
+    if (pass == 0 && rq.len >= row0 && rq.len < row1 && warp == 0) {
+        const __nv_bfloat16* src = lane < 16 ? nk : nv;
+        __nv_bfloat16* dst = (lane < 16 ? cache_k : cache_v) + rq.begin * stride_row + head_off +
+                             (long long)rq.len * stride_row;
+        *reinterpret_cast<uint4*>(dst) = __ldg(reinterpret_cast<const uint4*>(src));
+    }
+
+    // Copies of one step: K and V of kDecFlight rows per half-warp, 16 bytes per lane and row,
+    // straight into this warp's ring.  Rows past the split are zero-filled (a copy of 0 source
+    // bytes), so that they contribute exact zeros.  One commit group per step, also past the end.
+    const uint32_t ring0 = (uint32_t)__cvta_generic_to_shared(dec_ring) + warp * (kDecRing * kDecStepBytes) +
+                           ((lane >> 4) * kDecFlight * 2) * kDecRowBytes + l16 * 16;
+    auto issue = [&](int step) {
+        const int base = row0 + step * (kDecHalfWarps * kDecFlight);
+        const uint32_t dst = ring0 + (uint32_t)(step % kDecRing) * kDecStepBytes;
+        if (base < row1) {
+#pragma unroll
+            for (int f = 0; f < kDecFlight; ++f) {
+                const int row = base + f * kDecHalfWarps + hw;
+                const bool is_new = (row == rq.len);
+                const bool valid = row < row1;
+                const __nv_bfloat16* kp = (is_new || !valid) ? nk : ck + (long long)row * stride_row;
+                const __nv_bfloat16* vp = (is_new || !valid) ? nv : cv + (long long)row * stride_row;
+                const int nbytes = valid ? 16 : 0;
+                asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;"
+                             ::"r"(dst + (2 * f) * kDecRowBytes), "l"(kp), "r"(nbytes) : "memory");
+                asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;"
+                             ::"r"(dst + (2 * f + 1) * kDecRowBytes), "l"(vp), "r"(nbytes) : "memory");
+            }
+        }
+        asm volatile("cp.async.commit_group;" ::: "memory");
+    };
+    // Softmax statistics and weighted V sums of one step's rows (online softmax against the running
+    // maximum of this half-warp).
+    auto consume = [&](int step) {
+        const int base = row0 + step * (kDecHalfWarps * kDecFlight);
+        const uint32_t src = ring0 + (uint32_t)(step % kDecRing) * kDecStepBytes;
         uint4 ku[kDecFlight], vu[kDecFlight];
-        bool valid[kDecFlight];
 #pragma unroll
         for (int f = 0; f < kDecFlight; ++f) {
-            const int row = base + f * kDecHalfWarps + hw;
-            valid[f] = row < row1;
-            ku[f] = make_uint4(0u, 0u, 0u, 0u);
-            vu[f] = make_uint4(0u, 0u, 0u, 0u);
-            if (valid[f]) {
-                const bool is_new = (row == rq.len);             // Eq. 2: the appended row
-                const __nv_bfloat16* kp = is_new ? nk : ck + (long long)row * stride_row;
-                const __nv_bfloat16* vp = is_new ? nv : cv + (long long)row * stride_row;
-                ku[f] = __ldg(reinterpret_cast<const uint4*>(kp));
-                vu[f] = __ldg(reinterpret_cast<const uint4*>(vp));
-                if (is_new && pass == 0) {                       // the cache grows by this row
-                    *reinterpret_cast<uint4*>(cache_k + rq.begin * stride_row + head_off + (long long)row * stride_row) = ku[f];
-                    *reinterpret_cast<uint4*>(cache_v + rq.begin * stride_row + head_off + (long long)row * stride_row) = vu[f];
-                }
-            }
+            asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];"
+                         : "=r"(ku[f].x), "=r"(ku[f].y), "=r"(ku[f].z), "=r"(ku[f].w)
+                         : "r"(src + (2 * f) * kDecRowBytes));
+            asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];"
+                         : "=r"(vu[f].x), "=r"(vu[f].y), "=r"(vu[f].z), "=r"(vu[f].w)
+                         : "r"(src + (2 * f + 1) * kDecRowBytes));
         }
         float s[kDecFlight][GT];
 #pragma unroll
         for (int f = 0; f < kDecFlight; ++f) {
+            const bool valid = base + f * kDecHalfWarps + hw < row1;
             float kx[8];
             unpack_bf16x8(ku[f], kx);
 #pragma unroll
@@ -141,7 +181,7 @@ decode_kernel(const __grid_constant__ DecodeBatch batch, const __nv_bfloat16* __
                 for (int i = 0; i < 8; ++i) d = fmaf(qv[g][i], kx[i], d);
 #pragma unroll
                 for (int ofs = 8; ofs > 0; ofs >>= 1) d += __shfl_xor_sync(0xffffffffu, d, ofs, 16);
-                s[f][g] = valid[f] ? d : -INFINITY;
+                s[f][g] = valid ? d : -INFINITY;
             }
         }
 #pragma unroll
@@ -169,6 +209,17 @@ decode_kernel(const __grid_constant__ DecodeBatch batch, const __nv_bfloat16* __
                 for (int i = 0; i < 8; ++i) o[g][i] = fmaf(p[f], vx[i], o[g][i]);
             }
         }
+    };
+
+    // the step count does not depend on the half-warp, so both halves of a warp reach the shuffles
+    const int n_steps = (row1 - row0 + kDecHalfWarps * kDecFlight - 1) / (kDecHalfWarps * kDecFlight);
+#pragma unroll
+    for (int st = 0; st < kDecRing - 1; ++st) issue(st);
+    for (int st = 0; st < n_steps; ++st) {
+        // the buffer refilled here was read into registers one iteration ago
+        issue(st + kDecRing - 1);
+        asm volatile("cp.async.wait_group %0;" ::"n"(kDecRing - 1) : "memory");
+        consume(st);
     }
 
     // ---- combine: the two half-warps of a warp in registers, then the warps in warp order -------
@@ -224,59 +275,120 @@ decode_kernel(const __grid_constant__ DecodeBatch batch, const __nv_bfloat16* __
             }
         }
     }
-    if (n_splits == 1) return;
+}
 
-    // ---- several splits: the CTA that arrives last adds them in split order ----------------------
-    __threadfence();
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        int* cnt = arrivals + rq.arrival_begin + h * n_pass + pass;
-        const int prev = atomicAdd(cnt, 1);
-        sh.last = (prev == n_splits - 1);
-        if (sh.last) *cnt = 0;                                   // ready for the next step
-    }
-    __syncthreads();
-    if (!sh.last) return;
-    __threadfence();
-    if (threadIdx.x < kHeadDim) {
-        const int t = threadIdx.x;
-        const float* base = parts + ((long long)rq.part_begin + (long long)(h * n_pass + pass) * n_splits * GT) * part_stride;
+// Several splits: adds the partial results of one (request, KV head, pass, query head) in split
+// order.  One CTA of 128 threads per such unit, thread t owns feature t; the records of eight
+// splits are requested together (the loop is bound by the latency of these loads).  Launched
+// behind decode_kernel with programmatic stream serialisation: no counters, no atomics, nothing in
+// the workspace has to be cleared, and the order of additions is fixed.
+__global__ void __launch_bounds__(kHeadDim)
+decode_combine_kernel(const __grid_constant__ DecodeBatch batch, int gt, int n_pass, int n_q_heads, int group,
+                      float scale_log2, const float* __restrict__ parts, float* __restrict__ out) {
+    const DecodeReq rq = batch.r[blockIdx.y];
+    const int n_splits = rq.n_splits;
+    const int g = (int)blockIdx.x % gt, unit = (int)blockIdx.x / gt;     // unit = h * n_pass + pass
+    const int pass = unit % n_pass, h = unit / n_pass;
+    const int t = threadIdx.x;
+    grid_dependency_wait();
+    if (n_splits == 1) return;                                   // decode_kernel wrote the output itself
+    const long long part_stride = kHeadDim + 2;
+    const float* base = parts + ((long long)rq.part_begin + (long long)unit * n_splits * gt + g) * part_stride;
+    const long long step = (long long)gt * part_stride;          // between the records of two splits
+    constexpr int kBatch = 8;
+    float mx = -INFINITY;
+    for (int s0 = 0; s0 < n_splits; s0 += kBatch) {
+        float mv[kBatch];
 #pragma unroll
-        for (int g = 0; g < GT; ++g) {
-            float mx = -INFINITY;
-            for (int sp = 0; sp < n_splits; ++sp) mx = fmaxf(mx, __ldcg(base + ((long long)sp * GT + g) * part_stride));
-            float lsum = 0.f, osum = 0.f;
-            for (int sp = 0; sp < n_splits; ++sp) {
-                const float* rec = base + ((long long)sp * GT + g) * part_stride;
-                const float a = dec_ex2((__ldcg(rec) - mx) * scale_log2);
-                lsum = fmaf(__ldcg(rec + 1), a, lsum);
-                osum = fmaf(__ldcg(rec + 2 + t), a, osum);
-            }
-            out[((long long)rq.index * n_q_heads + qh0 + g) * kHeadDim + t] = osum / lsum;
+        for (int j = 0; j < kBatch; ++j) mv[j] = (s0 + j < n_splits) ? __ldcg(base + (s0 + j) * step) : -INFINITY;
+#pragma unroll
+        for (int j = 0; j < kBatch; ++j) mx = fmaxf(mx, mv[j]);
+    }
+    float lsum = 0.f, osum = 0.f;
+    for (int s0 = 0; s0 < n_splits; s0 += kBatch) {
+        float mv[kBatch], lv[kBatch], ov[kBatch];
+#pragma unroll
+        for (int j = 0; j < kBatch; ++j) {
+            const bool in = s0 + j < n_splits;
+            const float* rec = base + (s0 + j) * step;
+            mv[j] = in ? __ldcg(rec) : -INFINITY;
+            lv[j] = in ? __ldcg(rec + 1) : 0.f;
+            ov[j] = in ? __ldcg(rec + 2 + t) : 0.f;
+        }
+#pragma unroll
+        for (int j = 0; j < kBatch; ++j) {
+            const float a = dec_ex2((mv[j] - mx) * scale_log2);  // 0 past the last split
+            lsum = fmaf(lv[j], a, lsum);
+            osum = fmaf(ov[j], a, osum);
         }
     }
+    out[((long long)rq.index * n_q_heads + h * group + pass * gt + g) * kHeadDim + t] = osum / lsum;
 }
 
 }  // namespace
 
+// The ring needs more dynamic shared memory than the default limit: raised once per device.
+static cudaError_t configure_decode() {
+    static unsigned long long configured = 0;
+    return once_per_device(configured, []() {
+        cudaError_t e = cudaFuncSetAttribute(decode_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kDecRingBytes);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(decode_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kDecRingBytes);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(decode_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, kDecRingBytes);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(decode_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, kDecRingBytes);
+        return e;
+    });
+}
+
+// CTAs of decode_kernel<gt> that one SM holds at a time on the current device (looked up once per
+// device); 0 if the query fails.  The planner sizes the grid to one such wave.
+int decode_ctas_per_sm(int gt) {
+    static int cache[64][4] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 0;
+    const int idx = gt == 8 ? 3 : gt == 4 ? 2 : gt == 2 ? 1 : 0;
+    int v = __atomic_load_n(&cache[dev][idx], __ATOMIC_ACQUIRE);
+    if (v > 0) return v;
+    if (configure_decode() != cudaSuccess) { cudaGetLastError(); return 0; }
+    cudaError_t err;
+    if (idx == 3) err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&v, decode_kernel<8>, kDecThreads, kDecRingBytes);
+    else if (idx == 2) err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&v, decode_kernel<4>, kDecThreads, kDecRingBytes);
+    else if (idx == 1) err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&v, decode_kernel<2>, kDecThreads, kDecRingBytes);
+    else err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&v, decode_kernel<1>, kDecThreads, kDecRingBytes);
+    if (err != cudaSuccess || v <= 0) { cudaGetLastError(); return 0; }
+    __atomic_store_n(&cache[dev][idx], v, __ATOMIC_RELEASE);
+    return v;
+}
+
 cudaError_t launch_decode(const DecodeBatch& batch, int total_ctas, int gt, const void* q,
                           const void* k_new, const void* v_new, void* cache_k, void* cache_v,
                           long long stride_row, long long stride_head, int n_q_heads, int n_kv_heads,
-                          int rows_per_split, float scale_log2, float* parts, int* arrivals,
-                          float* out, cudaStream_t stream) {
+                          int rows_per_split, float scale_log2, float* parts, float* out,
+                          cudaStream_t stream) {
     if (total_ctas <= 0) return cudaSuccess;
     const int group = n_q_heads / n_kv_heads;
+    cudaError_t err = configure_decode();
+    if (err != cudaSuccess) return err;
 #define LOOKM_LAUNCH_DECODE(GT)                                                                     \
-    return launch_chained(decode_kernel<GT>, dim3((unsigned)total_ctas), dim3(kDecThreads), 0, stream, \
-                          batch, (const __nv_bfloat16*)q, (const __nv_bfloat16*)k_new,              \
-                          (const __nv_bfloat16*)v_new, (__nv_bfloat16*)cache_k, (__nv_bfloat16*)cache_v, \
-                          stride_row, stride_head, n_q_heads, n_kv_heads, group, rows_per_split,    \
-                          scale_log2, parts, arrivals, out);
+    err = launch_chained(decode_kernel<GT>, dim3((unsigned)total_ctas), dim3(kDecThreads),          \
+                         (size_t)kDecRingBytes, stream,                                             \
+                         batch, (const __nv_bfloat16*)q, (const __nv_bfloat16*)k_new,               \
+                         (const __nv_bfloat16*)v_new, (__nv_bfloat16*)cache_k, (__nv_bfloat16*)cache_v, \
+                         stride_row, stride_head, n_q_heads, n_kv_heads, group, rows_per_split,     \
+                         scale_log2, parts, out);
     if (gt == 8) { LOOKM_LAUNCH_DECODE(8) }
-    if (gt == 4) { LOOKM_LAUNCH_DECODE(4) }
-    if (gt == 2) { LOOKM_LAUNCH_DECODE(2) }
-    LOOKM_LAUNCH_DECODE(1)
+    else if (gt == 4) { LOOKM_LAUNCH_DECODE(4) }
+    else if (gt == 2) { LOOKM_LAUNCH_DECODE(2) }
+    else { LOOKM_LAUNCH_DECODE(1) }
 #undef LOOKM_LAUNCH_DECODE
+    return err;
+}
+
+cudaError_t launch_decode_combine(const DecodeBatch& batch, int gt, int n_q_heads, int n_kv_heads,
+                                  float scale_log2, const float* parts, float* out, cudaStream_t stream) {
+    const int group = n_q_heads / n_kv_heads;
+    const int n_pass = group / gt;
+    return launch_chained(decode_combine_kernel, dim3((unsigned)(n_kv_heads * n_pass * gt), (unsigned)batch.n_req),
+                          dim3(kHeadDim), 0, stream, batch, gt, n_pass, n_q_heads, group, scale_log2, parts, out);
 }
 
 }  // namespace lookm

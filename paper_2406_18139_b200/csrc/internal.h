@@ -85,6 +85,10 @@ cudaError_t launch_tile_kernel(int kind, const CUtensorMap& map_a, const CUtenso
 cudaError_t launch_lse_split(const float* lse, int n_q_heads, long long T, float scale_log2,
                              unsigned short* lse_split, cudaStream_t stream);
 
+// One CTA that waits, with the tile kernels' own bounded wait and the given limit, on an mbarrier
+// nobody arrives at; on expiry it writes LOOKM_ERR_DEVICE_TIMEOUT to *status like they do.
+cudaError_t launch_wait_probe(unsigned long long limit_ns, int* status, cudaStream_t stream);
+
 cudaError_t launch_select(const float* scores, const uint8_t* mask, const Req* reqs, int n_req,
                           int n_kv_heads, long long T, int* kept_idx, int* evict_idx, int* rank,
                           const void* k_for_norms, long long stride_tok, long long stride_head,
@@ -146,17 +150,44 @@ struct DecodeReq {
     int n_splits;         // CTAs per (KV head, pass)
     int cta_begin;        // first CTA of the request in this launch
     int part_begin;       // first partial-result record of the request in the workspace
-    int arrival_begin;    // first arrival counter of the request
+    int pad;
 };
 constexpr int kDecodeChunk = 96;
 struct DecodeBatch { int n_req; int pad; DecodeReq r[kDecodeChunk]; };
+
+#ifndef LOOKM_DEC_THREADS
+#define LOOKM_DEC_THREADS 256
+#endif
+constexpr int kDecodeThreads = LOOKM_DEC_THREADS;             // threads per CTA of the decode kernel
+constexpr int kDecodeMaxCtasPerSm = 2048 / kDecodeThreads;    // what an SM's thread limit allows
+int decode_ctas_per_sm(int gt);          // resident CTAs per SM of the kernel for this gt (0: unknown)
 
 // gt: query heads handled per pass over the rows (1, 2, 4 or 8; divides the group size)
 cudaError_t launch_decode(const DecodeBatch& batch, int total_ctas, int gt, const void* q,
                           const void* k_new, const void* v_new, void* cache_k, void* cache_v,
                           long long stride_row, long long stride_head, int n_q_heads, int n_kv_heads,
-                          int rows_per_split, float scale_log2, float* parts, int* arrivals,
-                          float* out, cudaStream_t stream);
+                          int rows_per_split, float scale_log2, float* parts, float* out,
+                          cudaStream_t stream);
+// adds the splits of every request of the batch that has more than one (chained behind launch_decode)
+cudaError_t launch_decode_combine(const DecodeBatch& batch, int gt, int n_q_heads, int n_kv_heads,
+                                  float scale_log2, const float* parts, float* out, cudaStream_t stream);
+
+// Function attributes (the dynamic shared-memory limit) are set once per device, not per launch:
+// `mask` holds one bit per device ordinal on which `configure` has succeeded.  Two threads may both
+// run `configure` the first time, which is harmless.
+#ifdef __CUDACC__
+template <class F>
+inline cudaError_t once_per_device(unsigned long long& mask, F configure) {
+    int dev = 0;
+    cudaError_t err = cudaGetDevice(&dev);
+    if (err != cudaSuccess) return err;
+    const unsigned long long bit = 1ull << (dev & 63);
+    if (__atomic_load_n(&mask, __ATOMIC_ACQUIRE) & bit) return cudaSuccess;
+    err = configure();
+    if (err == cudaSuccess) __atomic_fetch_or(&mask, bit, __ATOMIC_RELEASE);
+    return err;
+}
+#endif
 
 // Launch with programmatic stream serialisation: the grid may be set up while the kernel before it
 // in the stream drains.  Every kernel launched this way starts with grid_dependency_wait(), which

@@ -757,18 +757,27 @@ cudaError_t launch_invert_assignment(const int* assign, const int* kept_idx, con
     const size_t smem = ((size_t)32 * (wide_counts ? sizeof(unsigned) : sizeof(unsigned short)) + sizeof(int))
                         << digit_bits;
     dim3 grid(n_kv_heads, n_req);
-    cudaError_t err;
-#define LOOKM_LAUNCH_INVERT(CT, BITS)                                                               \
-    err = cudaFuncSetAttribute(invert_assignment_kernel<CT, BITS>,                                  \
-                               cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);             \
-    if (err != cudaSuccess) return err;                                                             \
-    err = launch_chained(invert_assignment_kernel<CT, BITS>, grid, dim3(kInvThreads), smem, stream, \
-                         assign, kept_idx, evict_idx, sim, reqs, n_kv_heads, T, row_ptr, ent_pos,   \
-                         ent_w, unit_first, slot_cnt, sort_a, sort_b, status);
-    if (wide_counts) { LOOKM_LAUNCH_INVERT(unsigned, kInvDigitBits32) }
-    else { LOOKM_LAUNCH_INVERT(unsigned short, kInvDigitBits16) }
-#undef LOOKM_LAUNCH_INVERT
-    return err;
+    // the shared-memory limit is raised once per device to the most either instantiation can ask
+    // for (32 warps x 2^bits counters and 2^bits totals)
+    static unsigned long long configured = 0;
+    cudaError_t err = once_per_device(configured, [&]() {
+        const int max16 = (int)(((size_t)32 * sizeof(unsigned short) + sizeof(int)) << kInvDigitBits16);
+        const int max32 = (int)(((size_t)32 * sizeof(unsigned) + sizeof(int)) << kInvDigitBits32);
+        cudaError_t e = cudaFuncSetAttribute(invert_assignment_kernel<unsigned short, kInvDigitBits16>,
+                                             cudaFuncAttributeMaxDynamicSharedMemorySize, max16);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(invert_assignment_kernel<unsigned, kInvDigitBits32>,
+                                     cudaFuncAttributeMaxDynamicSharedMemorySize, max32);
+        return e;
+    });
+    if (err != cudaSuccess) return err;
+    if (wide_counts)
+        return launch_chained(invert_assignment_kernel<unsigned, kInvDigitBits32>, grid, dim3(kInvThreads), smem,
+                              stream, assign, kept_idx, evict_idx, sim, reqs, n_kv_heads, T, row_ptr, ent_pos,
+                              ent_w, unit_first, slot_cnt, sort_a, sort_b, status);
+    return launch_chained(invert_assignment_kernel<unsigned short, kInvDigitBits16>, grid, dim3(kInvThreads), smem,
+                          stream, assign, kept_idx, evict_idx, sim, reqs, n_kv_heads, T, row_ptr, ent_pos,
+                          ent_w, unit_first, slot_cnt, sort_a, sort_b, status);
 }
 
 int merge_warps_per_sm() { return kMergeWarps; }
@@ -782,7 +791,10 @@ cudaError_t launch_merge(const void* k, const void* v, long long stride_tok, lon
     if (total_units <= 0) return cudaSuccess;
     if (stride_tok <= 0 || stride_tok >= (1ll << 31)) return cudaErrorInvalidValue;   // byte stride kept in 32 bits
     const int smem = (int)sizeof(MergeShared) + 128;
-    cudaError_t err = cudaFuncSetAttribute(merge_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    static unsigned long long configured = 0;
+    cudaError_t err = once_per_device(configured, [&]() {
+        return cudaFuncSetAttribute(merge_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    });
     if (err != cudaSuccess) return err;
     long long blocks = (total_units + kMergeWarps - 1) / kMergeWarps;
     if (blocks > num_sms) blocks = num_sms;              // persistent: one CTA per SM

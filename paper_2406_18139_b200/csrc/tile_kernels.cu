@@ -214,14 +214,15 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
             ptx::prefetch_tensormap(&map_a);
             ptx::prefetch_tensormap(&map_b);
             if (KIND == kSweep2) ptx::prefetch_tensormap(&map_x);
-            uint32_t gb = 0;                         // running streamed-tile index
-            int n = 0;                               // items done by this CTA
-            for (int round = 0;; ++round, ++n) {
+            uint32_t gb = 0;                         // streamed tiles armed so far
+            int n = 0;                               // stationary tiles armed so far
+            bool stop = false;                       // a wait gave up: arm nothing more
+            for (int round = 0; !stop; ++round, ++n) {
                 const int item = item_of_round(round, blockIdx.x, n_cta);
                 if (item >= p.n_items) { if (round * n_cta >= p.n_items) break; --n; continue; }
                 const Item it = decode_item<KIND>(p, tbl, item);
                 const int ab = n & 1;
-                ptx::mbar_wait(ptx::smem_u32(&sh.a_empty[ab]), ((n >> 1) & 1) ^ 1, abort_flag);
+                if (!ptx::mbar_wait(ptx::smem_u32(&sh.a_empty[ab]), ((n >> 1) & 1) ^ 1, abort_flag)) break;
                 const uint32_t abar = ptx::smem_u32(&sh.a_full[ab]);
                 ptx::mbar_arrive_expect_tx(abar, kTileBytes);
                 const uint32_t adst = ptx::smem_u32(&sh.a[ab][0]);
@@ -231,7 +232,10 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                 ptx::tma_load_3d(adst + kHalfBytes, &map_a, 64, a_head, a_row, abar);
                 for (int t = 0; t < it.nt; ++t, ++gb) {
                     const int s = gb % kStages;
-                    ptx::mbar_wait(ptx::smem_u32(&sh.b_empty[s]), ((gb / kStages) & 1) ^ 1, abort_flag);
+                    if (!ptx::mbar_wait(ptx::smem_u32(&sh.b_empty[s]), ((gb / kStages) & 1) ^ 1, abort_flag)) {
+                        stop = true;
+                        break;
+                    }
                     const uint32_t bbar = ptx::smem_u32(&sh.b_full[s]);
                     ptx::mbar_arrive_expect_tx(bbar, KIND == kSweep2 ? kTileBytes + kSplitBytes : kTileBytes);
                     const uint32_t bdst = ptx::smem_u32(&sh.b[s][0]);
@@ -253,15 +257,19 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                     }
                 }
             }
-            // Every load issued above is consumed by the MMA warp before it finishes, except
-            // after an abort: then wait (bounded, ignoring the flag) until the last ring of
-            // loads has landed so that no copy is in flight when the CTA exits.
+            // Every load issued above is consumed by an MMA before the kernel ends, except after an
+            // abort.  Then nothing more was armed once a wait had given up (n and gb count exactly
+            // the tiles armed), and the copies of the last ring of streamed tiles and of the last two
+            // stationary tiles may still be on their way: wait for them (bounded, the flag is
+            // ignored; a TMA load completes whether or not anybody consumes it), so that no copy
+            // writes shared memory after the CTA has left.
             if (*abort_flag) {
-                int dummy = 0;
-                const uint32_t last = gb;
-                for (uint32_t g = (last > (uint32_t)kStages ? last - kStages : 0); g < last; ++g)
-                    ptx::mbar_wait(ptx::smem_u32(&sh.b_full[g % kStages]), (g / kStages) & 1, &dummy,
+                int ignore = 0;
+                for (uint32_t g = (gb > (uint32_t)kStages ? gb - kStages : 0); g < gb; ++g)
+                    ptx::mbar_wait(ptx::smem_u32(&sh.b_full[g % kStages]), (g / kStages) & 1, &ignore,
                                    200000000ull);
+                for (int m = (n > 2 ? n - 2 : 0); m < n; ++m)
+                    ptx::mbar_wait(ptx::smem_u32(&sh.a_full[m & 1]), (m >> 1) & 1, &ignore, 200000000ull);
             }
         }
     } else if (warp == 1 || warp == kEpiWarp0 + kGroups * 4) {
@@ -275,20 +283,26 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
             constexpr uint32_t idesc = ptx::umma_idesc_bf16(kTile, kTile);
             uint32_t gb = 0;
             int n = 0;
-            for (int round = 0;; ++round, ++n) {
+            bool stop = false;                       // a wait gave up: issue nothing more
+            for (int round = 0; !stop; ++round, ++n) {
                 const int item = item_of_round(round, blockIdx.x, n_cta);
                 if (item >= p.n_items) { if (round * n_cta >= p.n_items) break; --n; continue; }
                 const Item it = decode_item<KIND>(p, tbl, item);
                 const int ab = n & 1;
-                ptx::mbar_wait(ptx::smem_u32(&sh.a_full[ab]), (n >> 1) & 1, abort_flag);
+                if (!ptx::mbar_wait(ptx::smem_u32(&sh.a_full[ab]), (n >> 1) & 1, abort_flag)) break;
                 const uint32_t a_addr = ptx::smem_u32(&sh.a[ab][0]);
                 bool issued = false;
                 for (int t = 0; t < it.nt; ++t, ++gb) {
                     if ((gb & (kIssuers - 1)) != me) continue;
                     const int s = gb % kStages;
                     const int buf = gb % kAccum;
-                    ptx::mbar_wait(ptx::smem_u32(&sh.b_full[s]), (gb / kStages) & 1, abort_flag);
-                    ptx::mbar_wait(ptx::smem_u32(&sh.t_empty[buf]), ((gb / kAccum) & 1) ^ 1, abort_flag);
+                    // no MMA is issued on operands that have not landed or into an accumulator that
+                    // is still being read
+                    if (!ptx::mbar_wait(ptx::smem_u32(&sh.b_full[s]), (gb / kStages) & 1, abort_flag) ||
+                        !ptx::mbar_wait(ptx::smem_u32(&sh.t_empty[buf]), ((gb / kAccum) & 1) ^ 1, abort_flag)) {
+                        stop = true;
+                        break;
+                    }
                     ptx::tc_fence_after_sync();
                     const uint32_t b_addr = ptx::smem_u32(&sh.b[s][0]);
                     const uint32_t d_tmem = tmem_base + buf * kTile;
@@ -307,6 +321,7 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                     ptx::umma_commit(ptx::smem_u32(&sh.t_full[buf]));
                     issued = true;
                 }
+                if (stop) break;
                 // the stationary tile is free when both issuers are through with the item: an
                 // issuer that used it arrives when its MMAs have completed, the other one at once
                 if (issued) ptx::umma_commit(ptx::smem_u32(&sh.a_empty[ab]));
@@ -589,7 +604,32 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     if (threadIdx.x == 0 && sh.abort_flag) atomicExch(p.status, (int)LOOKM_ERR_DEVICE_TIMEOUT);
 }
 
+// The failure path of the bounded waits, exercised without starving a production kernel: thread 0
+// waits with ptx::mbar_wait on an mbarrier that nobody arrives at, the other threads on the same
+// barrier see either the limit or the abort flag, and the CTA reports the expiry exactly as
+// tile_kernel does (shared abort flag -> status word).
+__global__ void __launch_bounds__(128)
+wait_probe_kernel(unsigned long long limit_ns, int* status) {
+    __shared__ unsigned long long bar;
+    __shared__ int abort_flag;
+    if (threadIdx.x == 0) {
+        ptx::mbar_init(ptx::smem_u32(&bar), 1);
+        abort_flag = 0;
+        ptx::fence_mbar_init();
+    }
+    __syncthreads();
+    volatile int* flag = &abort_flag;
+    const bool arrived = ptx::mbar_wait(ptx::smem_u32(&bar), 0, flag, limit_ns);
+    __syncthreads();
+    if (threadIdx.x == 0 && (abort_flag || !arrived)) atomicExch(status, (int)LOOKM_ERR_DEVICE_TIMEOUT);
+}
+
 }  // namespace
+
+cudaError_t launch_wait_probe(unsigned long long limit_ns, int* status, cudaStream_t stream) {
+    wait_probe_kernel<<<1, 128, 0, stream>>>(limit_ns, status);
+    return cudaGetLastError();
+}
 
 cudaError_t launch_tile_kernel(int kind, const CUtensorMap& map_a, const CUtensorMap& map_b,
                                const CUtensorMap* map_x, const TileParams& p, int num_sms,
@@ -598,16 +638,21 @@ cudaError_t launch_tile_kernel(int kind, const CUtensorMap& map_a, const CUtenso
     const int smem = (int)sizeof(Shared) + 1024;
     const int grid = p.n_items < num_sms ? p.n_items : num_sms;
     const CUtensorMap& mx = map_x ? *map_x : map_b;      // only sweep 2 uses it
-    cudaError_t err;
-#define LOOKM_LAUNCH(K)                                                                          \
-    err = cudaFuncSetAttribute(tile_kernel<K>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem); \
-    if (err != cudaSuccess) return err;                                                          \
-    err = launch_chained(tile_kernel<K>, dim3(grid), dim3(kThreads), (size_t)smem, stream, map_a, map_b, mx, p);
-    if (kind == kSweep1) { LOOKM_LAUNCH(kSweep1) }
-    else if (kind == kSweep2) { LOOKM_LAUNCH(kSweep2) }
-    else { LOOKM_LAUNCH(kMatch) }
-#undef LOOKM_LAUNCH
-    return err;
+    static unsigned long long configured = 0;
+    cudaError_t err = once_per_device(configured, [&]() {
+        cudaError_t e = cudaFuncSetAttribute(tile_kernel<kSweep1>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(tile_kernel<kSweep2>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(tile_kernel<kMatch>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        return e;
+    });
+    if (err != cudaSuccess) return err;
+    if (kind == kSweep1)
+        return launch_chained(tile_kernel<kSweep1>, dim3(grid), dim3(kThreads), (size_t)smem, stream, map_a, map_b, mx, p);
+    if (kind == kSweep2)
+        return launch_chained(tile_kernel<kSweep2>, dim3(grid), dim3(kThreads), (size_t)smem, stream, map_a, map_b, mx, p);
+    return launch_chained(tile_kernel<kMatch>, dim3(grid), dim3(kThreads), (size_t)smem, stream, map_a, map_b, mx, p);
 }
 
 cudaError_t launch_lse_split(const float* lse, int n_q_heads, long long T, float scale_log2,

@@ -125,3 +125,21 @@ def test_decode_step_host_side_argument_errors():
     assert B.lookm_decode_workspace_size(B.CacheLayout(32, 8, 64, 64, 4096, 0.0), [10]) == 0
     n1 = B.lookm_decode_workspace_size(lay, [10])
     assert n1 > 0 and n1 % 256 == 0 and B.lookm_decode_workspace_size(lay, [1 << 20]) == n1
+
+
+def test_wait_expiry_selftest_argument_errors():
+    lib = B.lib()
+    fake = C.c_void_p(0x1000)
+    assert lib.lookm_selftest_wait_expiry(0, fake, 256, None) == B.ERR_INVALID_ARG
+    assert lib.lookm_selftest_wait_expiry(100001, fake, 256, None) == B.ERR_INVALID_ARG
+    assert lib.lookm_selftest_wait_expiry(1000, None, 256, None) == B.ERR_INVALID_ARG
+    assert lib.lookm_selftest_wait_expiry(1000, C.c_void_p(0x1010), 256, None) == B.ERR_INVALID_ARG
+    assert lib.lookm_selftest_wait_expiry(1000, fake, 128, None) == B.ERR_WORKSPACE_TOO_SMALL
+
+
+def test_the_binding_loads_the_in_tree_library_only():
+    here = os.path.join(ROOT, "paper_2406_18139_b200", "liblookm.so")
+    assert os.path.samefile(B.LIB_PATH, here)
+    B.lib()
+    mapped = [l.split()[-1] for l in open("/proc/self/maps") if "liblookm" in l]
+    assert mapped and all(os.path.samefile(m, here) for m in mapped)

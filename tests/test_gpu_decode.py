@@ -102,7 +102,9 @@ def test_batch_of_requests_with_their_own_lengths(B):
     out = torch.full((n_req, Hq, 128), np.nan, dtype=torch.float32, device="cuda")
     B.check(B.lookm_decode_step_varlen(q, kn, vn, dk, dv, begins, lens, lay, out, ws))
     torch.cuda.synchronize()
-    assert B.lookm_last_launch_count() == 2
+    # two launches of at most 96 requests, each followed by one combine launch if any of its
+    # requests was cut into several splits
+    assert 2 <= B.lookm_last_launch_count() <= 4
     got = out.cpu().numpy().astype(np.float64)
     f = synth.bf16_to_f32
     K, V = f(ck_b), f(cv_b)

@@ -394,3 +394,29 @@ def test_merge_single_kept_token_and_bad_index_status(B):
     B.check(B.lookm_merge(k, v, kept, ev, assign, sim, [0, L], [1], [0], lay, 0, out_k, out_v, ws))
     assert B.lookm_device_status(ws) == B.ERR_DEVICE_BAD_INDEX
     assert B.lookm_device_status(ws) == B.OK          # reading clears it
+
+
+def test_an_expired_device_wait_is_reported_and_the_context_stays_usable(B):
+    """The tile kernels bound every mbarrier wait; when one runs out the CTA raises its abort flag,
+    leaves, and the status word says so.  Here a one-CTA kernel waits 1 ms, through the same wait
+    routine, on a barrier nobody arrives at."""
+    import torch
+    ws = torch.empty(4096, dtype=torch.uint8, device="cuda")
+    t0 = torch.cuda.Event(enable_timing=True)
+    t1 = torch.cuda.Event(enable_timing=True)
+    t0.record()
+    B.check(B.lookm_selftest_wait_expiry(1000, ws))
+    t1.record()
+    assert B.lookm_device_status(ws) == B.ERR_DEVICE_TIMEOUT
+    assert B.lookm_device_status(ws) == B.OK              # reading clears it
+    assert 0.9 <= t0.elapsed_time(t1) <= 50.0             # the limit was 1 ms; it neither returned early nor hung
+    # the context still works: a real kernel of the library runs and reports no error
+    L = 300
+    w = synth.tiny(L, 2, 2, 60, 8, 0, seed=3)
+    (q, k, v), _, mask, _ = _tensors(w)
+    lay = B.make_layout(q, k)
+    ws2 = B.alloc_workspace(lay, [L])
+    scores = torch.zeros(2, L, dtype=torch.float32, device="cuda")
+    B.check(B.lookm_score(q, k, [0, L], lay, scores, None, 0, ws2))
+    assert B.lookm_device_status(ws2) == B.OK
+    assert abs(float(scores.sum()) - 2 * L) <= 1e-2
