@@ -36,38 +36,73 @@
 namespace lookm {
 namespace {
 
-constexpr int kStages = 4;                       // ring of streamed tiles
+#ifndef LOOKM_TILE_STAGES
+#define LOOKM_TILE_STAGES 4
+#endif
+#ifndef LOOKM_TILE_ABUF
+#define LOOKM_TILE_ABUF 2
+#endif
+constexpr int kStages = LOOKM_TILE_STAGES;       // ring of streamed tiles
+constexpr int kABuf = LOOKM_TILE_ABUF;           // buffers of the stationary tile (2: the next item's is
+                                                 // loaded while this item's is in use)
+#ifndef LOOKM_TILE_GROUPS
+#define LOOKM_TILE_GROUPS 4
+#endif
+#ifndef LOOKM_TILE_PIPE
+#define LOOKM_TILE_PIPE 0
+#endif
 constexpr int kAccum = 4;                        // TMEM accumulators (128 fp32 columns each)
-constexpr int kGroups = 4;                       // epilogue groups (one per TMEM accumulator)
+#ifndef LOOKM_TILE_HALVES
+#define LOOKM_TILE_HALVES 1
+#endif
+constexpr int kGroups = LOOKM_TILE_GROUPS;       // epilogue groups; tile g goes to group g mod kGroups
+constexpr int kHalves = LOOKM_TILE_HALVES;       // a group is kHalves PARTS of four warps; part p of a group
+                                                 // reads columns [p, p + 1) * kCols of the group's accumulators
+constexpr int kParts = kGroups * kHalves;        // four-warp units of the epilogue (each keeps partial results)
+constexpr int kCols = kTile / kHalves;           // accumulator columns per part
+// "Accumulator filled" barriers form a ring twice as long as the accumulators: tile g uses barrier
+// g mod kFullRing in phase g / kFullRing.  A group may reach tile g while tile g - kAccum (same
+// accumulator, other group, other issuing thread) is still being multiplied; with one barrier per
+// accumulator its parity wait would then pass at once.  With the longer ring the tile one phase
+// back is g - 2 kAccum, whose MMAs had to complete before the producer could load tile g - kAccum,
+// which it did before it loaded any tile this group has already finished.
+constexpr int kFullRing = 2 * kAccum;
+constexpr bool kPipeLoads = LOOKM_TILE_PIPE;     // sweeps: the next 32 columns are on their way from TMEM
+                                                 // while the current ones are worked on
 constexpr int kIssuers = 2;                      // MMA-issuing threads (tiles alternate between them)
 constexpr int kEpiWarp0 = 2;                     // first epilogue warp
-constexpr int kThreads = 64 + kGroups * 128 + 32;   // producer warp, MMA warp, 4 x 4 epilogue warps, second MMA warp
+constexpr int kThreads = 64 + kParts * 128 + 32; // producer warp, MMA warp, kParts x 4 epilogue warps, second MMA warp
 constexpr int kHalfBytes = kTile * 64 * 2;       // one TMA box: 128 rows x 64 bf16 (128 B rows)
 constexpr int kTileBytes = 2 * kHalfBytes;       // 128 x 128 bf16
 constexpr int kSplitBytes = kTile * 16 * 2;      // 128 rows x 16 bf16 (32-byte rows, 32-byte swizzle)
-constexpr int kReqCache = 32;                    // request-table entries cached in shared memory
+constexpr int kReqCache = 16;                    // request-table entries cached in shared memory
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kReferenceSlack = 1.152921504606847e18f;   // 2^60: largest chunk sum kept against a stale reference
 constexpr float kLn2 = 0.6931471805599453f;
 
+template <int KIND>
 struct __align__(1024) Shared {
-    uint8_t a[2][kTileBytes];                    // stationary tiles (double-buffered across items)
+    static constexpr int kXStages = (KIND == kSweep2) ? kStages : 1;   // only sweep 2 streams companions
+    static constexpr int kPlanes = (KIND == kSweep2) ? 1 : 2;          // values per row and part to combine
+    uint8_t a[kABuf][kTileBytes];                // stationary tiles
     uint8_t b[kStages][kTileBytes];              // streamed tiles
-    uint8_t bx[kStages][kSplitBytes];            // sweep 2: the streamed tiles' 16-column companions
+    uint8_t bx[kXStages][kSplitBytes];           // sweep 2: the streamed tiles' 16-column companions
     union {
-        float side[kGroups][2][kTile];           // match: per epilogue group, double-buffered column data
+        float side[kParts][2][kCols];            // match: per epilogue part, double-buffered column data
         uint8_t ax[kSplitBytes];                 // sweep 2: constant ones tile that multiplies bx
     };
-    float comb[2][kGroups][2][kTile];            // partial results of the groups, double-buffered
+    float comb[2][kParts][kPlanes][kTile];       // partial results of the parts, double-buffered
     Req reqs[kReqCache];                         // copy of the request table (when it fits)
-    unsigned long long a_full[2], a_empty[2];
+    unsigned long long a_full[kABuf], a_empty[kABuf];
     unsigned long long b_full[kStages], b_empty[kStages];
-    unsigned long long t_full[kAccum], t_empty[kAccum];
+    unsigned long long t_full[2 * kAccum], t_empty[kAccum];   // t_full: see kFullRing
     unsigned long long comb_full[2], comb_free[2];   // partial results of an item written / read
     unsigned long long mma_done;                 // every MMA of this CTA has completed
     uint32_t tmem_base;
     int abort_flag;
 };
+static_assert(sizeof(Shared<kSweep1>) + 1024 <= 232448 && sizeof(Shared<kSweep2>) + 1024 <= 232448 &&
+              sizeof(Shared<kMatch>) + 1024 <= 232448, "shared memory of the tile kernels exceeds 227 KB");
 
 // The softmax epilogues are bound by the special-function unit (16 ex2 per clock and SM), so one
 // column in kPolyEvery is exponentiated on the FMA pipe instead.
@@ -152,14 +187,14 @@ __global__ void __launch_bounds__(kThreads, 1)
 tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
             const __grid_constant__ CUtensorMap map_x, const TileParams p) {
     extern __shared__ uint8_t smem_raw[];
-    Shared& sh = *reinterpret_cast<Shared*>(
+    Shared<KIND>& sh = *reinterpret_cast<Shared<KIND>*>(
         (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
     volatile int* abort_flag = &sh.abort_flag;
 
     if (threadIdx.x == 0) {
-        for (int i = 0; i < 2; ++i) {
+        for (int i = 0; i < kABuf; ++i) {
             ptx::mbar_init(ptx::smem_u32(&sh.a_full[i]), 1);
             ptx::mbar_init(ptx::smem_u32(&sh.a_empty[i]), kIssuers);
         }
@@ -167,13 +202,12 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
             ptx::mbar_init(ptx::smem_u32(&sh.b_full[i]), 1);
             ptx::mbar_init(ptx::smem_u32(&sh.b_empty[i]), 1);
         }
-        for (int i = 0; i < kAccum; ++i) {
-            ptx::mbar_init(ptx::smem_u32(&sh.t_full[i]), 1);
-            ptx::mbar_init(ptx::smem_u32(&sh.t_empty[i]), 4);   // one arrival per epilogue warp
-        }
+        for (int i = 0; i < kFullRing; ++i) ptx::mbar_init(ptx::smem_u32(&sh.t_full[i]), 1);
+        for (int i = 0; i < kAccum; ++i)
+            ptx::mbar_init(ptx::smem_u32(&sh.t_empty[i]), 4 * kHalves);   // one arrival per epilogue warp of a group
         for (int i = 0; i < 2; ++i) {
-            ptx::mbar_init(ptx::smem_u32(&sh.comb_full[i]), (kGroups - 1) * 4);   // warps of the other groups
-            ptx::mbar_init(ptx::smem_u32(&sh.comb_free[i]), 4);                   // warps of the combining group
+            ptx::mbar_init(ptx::smem_u32(&sh.comb_full[i]), (kParts - 1) * 4);    // warps of the other parts
+            ptx::mbar_init(ptx::smem_u32(&sh.comb_free[i]), 4);                   // warps of the combining part
         }
         ptx::mbar_init(ptx::smem_u32(&sh.mma_done), kIssuers);
         sh.abort_flag = 0;
@@ -221,8 +255,8 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                 const int item = item_of_round(round, blockIdx.x, n_cta);
                 if (item >= p.n_items) { if (round * n_cta >= p.n_items) break; --n; continue; }
                 const Item it = decode_item<KIND>(p, tbl, item);
-                const int ab = n & 1;
-                if (!ptx::mbar_wait(ptx::smem_u32(&sh.a_empty[ab]), ((n >> 1) & 1) ^ 1, abort_flag)) break;
+                const int ab = n % kABuf;
+                if (!ptx::mbar_wait(ptx::smem_u32(&sh.a_empty[ab]), ((n / kABuf) & 1) ^ 1, abort_flag)) break;
                 const uint32_t abar = ptx::smem_u32(&sh.a_full[ab]);
                 ptx::mbar_arrive_expect_tx(abar, kTileBytes);
                 const uint32_t adst = ptx::smem_u32(&sh.a[ab][0]);
@@ -249,7 +283,7 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                         const int h = it.head * p.group + t % p.group;
                         ptx::tma_load_3d(bdst, &map_b, 0, h, row, bbar);
                         ptx::tma_load_3d(bdst + kHalfBytes, &map_b, 64, h, row, bbar);
-                        ptx::tma_load_3d(ptx::smem_u32(&sh.bx[s][0]), &map_x, 0, h, row, bbar);
+                        ptx::tma_load_3d(ptx::smem_u32(&sh.bx[s % Shared<KIND>::kXStages][0]), &map_x, 0, h, row, bbar);
                     } else {
                         const int row = (int)(it.kept_row0 + (long long)t * kTile);
                         ptx::tma_load_2d(bdst, &map_b, 0, row, bbar);
@@ -268,11 +302,11 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                 for (uint32_t g = (gb > (uint32_t)kStages ? gb - kStages : 0); g < gb; ++g)
                     ptx::mbar_wait(ptx::smem_u32(&sh.b_full[g % kStages]), (g / kStages) & 1, &ignore,
                                    200000000ull);
-                for (int m = (n > 2 ? n - 2 : 0); m < n; ++m)
-                    ptx::mbar_wait(ptx::smem_u32(&sh.a_full[m & 1]), (m >> 1) & 1, &ignore, 200000000ull);
+                for (int m = (n > kABuf ? n - kABuf : 0); m < n; ++m)
+                    ptx::mbar_wait(ptx::smem_u32(&sh.a_full[m % kABuf]), (m / kABuf) & 1, &ignore, 200000000ull);
             }
         }
-    } else if (warp == 1 || warp == kEpiWarp0 + kGroups * 4) {
+    } else if (warp == 1 || warp == kEpiWarp0 + kParts * 4) {
         // ------------------------------------------------------------ MMA issuers -----------
         // One thread spends about as long on the waits, fences, commits and loop bookkeeping of a
         // tile as the tensor core needs for its eight MMAs, and it is blocked while they are
@@ -288,8 +322,8 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                 const int item = item_of_round(round, blockIdx.x, n_cta);
                 if (item >= p.n_items) { if (round * n_cta >= p.n_items) break; --n; continue; }
                 const Item it = decode_item<KIND>(p, tbl, item);
-                const int ab = n & 1;
-                if (!ptx::mbar_wait(ptx::smem_u32(&sh.a_full[ab]), (n >> 1) & 1, abort_flag)) break;
+                const int ab = n % kABuf;
+                if (!ptx::mbar_wait(ptx::smem_u32(&sh.a_full[ab]), (n / kABuf) & 1, abort_flag)) break;
                 const uint32_t a_addr = ptx::smem_u32(&sh.a[ab][0]);
                 bool issued = false;
                 for (int t = 0; t < it.nt; ++t, ++gb) {
@@ -316,9 +350,9 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                     }
                     if (KIND == kSweep2)                 // accumulator += ones x (-lse / scale)^T
                         ptx::umma_bf16(d_tmem, ptx::umma_desc_sw32(ptx::smem_u32(&sh.ax[0])),
-                                       ptx::umma_desc_sw32(ptx::smem_u32(&sh.bx[s][0])), idesc, 1u);
+                                       ptx::umma_desc_sw32(ptx::smem_u32(&sh.bx[s % Shared<KIND>::kXStages][0])), idesc, 1u);
                     ptx::umma_commit(ptx::smem_u32(&sh.b_empty[s]));
-                    ptx::umma_commit(ptx::smem_u32(&sh.t_full[buf]));
+                    ptx::umma_commit(ptx::smem_u32(&sh.t_full[gb % kFullRing]));
                     issued = true;
                 }
                 if (stop) break;
@@ -335,7 +369,9 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         }
     } else {
         // ------------------------------------------------------------ epilogue --------------
-        const int wg = (warp - kEpiWarp0) >> 2;              // epilogue group 0..3
+        const int part = (warp - kEpiWarp0) >> 2;            // four-warp unit of the epilogue
+        const int wg = part / kHalves;                       // its group
+        const int col0 = (part % kHalves) * kCols;           // first accumulator column it reads
         const int quarter = warp & 3;                        // TMEM lane quarter this warp may read
         const int row = quarter * 32 + lane;                 // row of the stationary tile
         const uint32_t lane_addr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
@@ -355,8 +391,8 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
 
             for (int t = 0; t < it.nt; ++t, ++gb) {
                 if ((int)(gb % kGroups) != wg) continue;
-                const int buf = wg;
-                float* side = sh.side[wg][lt & 1];
+                const int buf = (int)(gb % kAccum);
+                float* side = sh.side[part][lt & 1];
                 bool diag = false;                           // tile crosses the causal diagonal
                 int col_limit = kTile;                       // valid columns of the tile (match, sweep 2)
                 int diag_from = 0;                           // sweep 2: first column this row may use
@@ -370,13 +406,15 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                     diag = (ib == it.blk) || (col_limit < kTile);
                     diag_from = (ib == it.blk) ? row : 0;
                 } else {
-                    const int slot = t * kTile + row;
-                    side[row] = (slot < it.B) ? p.rnorm_kept[it.kept_row0 + slot] : 0.f;
+                    if (row < kCols) {
+                        const int slot = t * kTile + col0 + row;
+                        side[row] = (slot < it.B) ? p.rnorm_kept[it.kept_row0 + slot] : 0.f;
+                    }
                     col_limit = min(kTile, it.B - t * kTile);
-                    ptx::named_barrier_sync(1 + wg, 128);
+                    ptx::named_barrier_sync(1 + part, 128);
                 }
                 ++lt;
-                ptx::mbar_wait(ptx::smem_u32(&sh.t_full[buf]), (gb / kAccum) & 1, abort_flag);
+                ptx::mbar_wait(ptx::smem_u32(&sh.t_full[gb % kFullRing]), (gb / kFullRing) & 1, abort_flag);
                 ptx::tc_fence_after_sync();
                 if (KIND == kMatch) {
                     // running arg-max of dot / |kept key| over kept slots, 16 columns at a time with
@@ -384,8 +422,8 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                     // the work on 32 columns).  The maximum of the 16 is taken first; only when it
                     // beats the running best is its first column looked up, so a strict comparison
                     // in ascending slot order keeps the lowest slot.
-                    auto columns16 = [&](const uint32_t (&r)[16], int c0) {
-                        const float4* sd = reinterpret_cast<const float4*>(side + c0);
+                    auto columns16 = [&](const uint32_t (&r)[16], int c0) {      // c0: column of the tile
+                        const float4* sd = reinterpret_cast<const float4*>(side + (c0 - col0));
                         float v[16];
 #pragma unroll
                         for (int c4 = 0; c4 < 4; ++c4) {
@@ -415,15 +453,15 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                         }
                     };
                     uint32_t ra[16], rb[16];
-                    const uint32_t tbase = lane_addr + buf * kTile;
+                    const uint32_t tbase = lane_addr + buf * kTile + col0;
                     ptx::tmem_ld_32x16(tbase, ra);
 #pragma unroll
-                    for (int k = 0; k < 4; ++k) {
+                    for (int k = 0; k < kCols / 32; ++k) {
                         ptx::tmem_ld_wait16(ra);
                         ptx::tmem_ld_32x16(tbase + (2 * k + 1) * 16, rb, ra);
-                        columns16(ra, 2 * k * 16);
+                        columns16(ra, col0 + 2 * k * 16);
                         ptx::tmem_ld_wait16(rb);
-                        if (k < 3) {
+                        if (k < kCols / 32 - 1) {
                             ptx::tmem_ld_32x16(tbase + (2 * k + 2) * 16, ra, rb);
                         } else {
                             // everything is in registers: hand the accumulator back
@@ -431,23 +469,12 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                             __syncwarp();
                             if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&sh.t_empty[buf]));
                         }
-                        columns16(rb, (2 * k + 1) * 16);
+                        columns16(rb, col0 + (2 * k + 1) * 16);
                     }
                     continue;
                 }
-#pragma unroll 1
-                for (int ch = 0; ch < 4; ++ch) {
-                    uint32_t raw[32];
-                    ptx::tmem_ld_32x32(lane_addr + buf * kTile + ch * 32, raw);
-                    ptx::tmem_ld_wait();
-                    if (ch == 3) {
-                        // the last columns are in registers: hand the accumulator back now, so
-                        // that the next tile's MMAs run while this chunk is still being worked on
-                        ptx::tc_fence_before_sync();
-                        __syncwarp();
-                        if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&sh.t_empty[buf]));
-                    }
-                    const int c0 = ch * 32;
+                // work on 32 columns of the accumulator, c0 = first column of the chunk
+                auto process = [&](const uint32_t (&raw)[32], int c0) {
                     if (KIND == kSweep1) {
                         // softmax statistics of row `pos` over key columns c0..c0+31: l_run is the
                         // sum of exp2(x - m_run), where m_run is a REFERENCE, not necessarily the
@@ -526,6 +553,37 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                             }
                         }
                     }
+                };
+                // the last columns are in registers: hand the accumulator back, so that the next
+                // tile's MMAs run while this chunk is still being worked on
+                auto release = [&]() {
+                    ptx::tc_fence_before_sync();
+                    __syncwarp();
+                    if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&sh.t_empty[buf]));
+                };
+                const uint32_t tbase = lane_addr + buf * kTile + col0;
+                if (kPipeLoads) {
+                    uint32_t ra[32], rb[32];
+                    ptx::tmem_ld_32x32(tbase, ra);
+#pragma unroll 1
+                    for (int hf = 0; hf < kCols / 64; ++hf) {
+                        ptx::tmem_ld_wait32(ra);
+                        ptx::tmem_ld_32x32(tbase + (2 * hf + 1) * 32, rb, ra);
+                        process(ra, col0 + 2 * hf * 32);
+                        ptx::tmem_ld_wait32(rb);
+                        if (hf < kCols / 64 - 1) ptx::tmem_ld_32x32(tbase + (2 * hf + 2) * 32, ra, rb);
+                        else release();
+                        process(rb, col0 + (2 * hf + 1) * 32);
+                    }
+                } else {
+#pragma unroll 1
+                    for (int ch = 0; ch < kCols / 32; ++ch) {
+                        uint32_t raw[32];
+                        ptx::tmem_ld_32x32(tbase + ch * 32, raw);
+                        ptx::tmem_ld_wait();
+                        if (ch == kCols / 32 - 1) release();
+                        process(raw, col0 + ch * 32);
+                    }
                 }
             }
 
@@ -535,32 +593,33 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
             // item without waiting for anybody.  Values are always combined in group order.
             const int cslot = n & 1;
             const uint32_t cuse = static_cast<uint32_t>(n) >> 1;         // earlier uses of this buffer
-            const int combiner = static_cast<int>((gb - 1u) % kGroups);
-            float (*cb)[2][kTile] = sh.comb[cslot];
-            if (wg != combiner) {
+            const int combiner = static_cast<int>((gb - 1u) % kGroups) * kHalves + (kHalves - 1);
+            float (*cb)[Shared<KIND>::kPlanes][kTile] = sh.comb[cslot];
+            constexpr int kP1 = Shared<KIND>::kPlanes - 1;       // second value of a row (not in sweep 2)
+            if (part != combiner) {
                 // the buffer's previous contents (two items ago) have been read
                 ptx::mbar_wait(ptx::smem_u32(&sh.comb_free[cslot]), (cuse & 1u) ^ 1u, abort_flag);
-                if (KIND == kSweep1) { cb[wg][0][row] = m_run; cb[wg][1][row] = l_run; }
-                else if (KIND == kSweep2) { cb[wg][0][row] = (acc0 + acc1) + (acc2 + acc3); }
-                else { cb[wg][0][row] = best; cb[wg][1][row] = __int_as_float(best_slot); }
+                if (KIND == kSweep1) { cb[part][0][row] = m_run; cb[part][kP1][row] = l_run; }
+                else if (KIND == kSweep2) { cb[part][0][row] = (acc0 + acc1) + (acc2 + acc3); }
+                else { cb[part][0][row] = best; cb[part][kP1][row] = __int_as_float(best_slot); }
                 __syncwarp();
                 if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&sh.comb_full[cslot]));
             } else {
                 ptx::mbar_wait(ptx::smem_u32(&sh.comb_full[cslot]), cuse & 1u, abort_flag);
                 if (pos < it.L && !*abort_flag) {
                     if (KIND == kSweep1) {
-                        float mg[kGroups], lg[kGroups];
+                        float mg[kParts], lg[kParts];
 #pragma unroll
-                        for (int g = 0; g < kGroups; ++g) {
-                            mg[g] = (g == wg) ? m_run : cb[g][0][row];
-                            lg[g] = (g == wg) ? l_run : cb[g][1][row];
+                        for (int g = 0; g < kParts; ++g) {
+                            mg[g] = (g == part) ? m_run : cb[g][0][row];
+                            lg[g] = (g == part) ? l_run : cb[g][kP1][row];
                         }
                         float m = mg[0];
 #pragma unroll
-                        for (int g = 1; g < kGroups; ++g) m = fmaxf(m, mg[g]);
+                        for (int g = 1; g < kParts; ++g) m = fmaxf(m, mg[g]);
                         float l = lg[0] * ptx::ex2((mg[0] - m) * c2);
 #pragma unroll
-                        for (int g = 1; g < kGroups; ++g) l += lg[g] * ptx::ex2((mg[g] - m) * c2);
+                        for (int g = 1; g < kParts; ++g) l += lg[g] * ptx::ex2((mg[g] - m) * c2);
                         // natural-log log-sum-exp of the scaled logits
                         const float lse = (m * c2 + ptx::lg2(l)) * kLn2;
                         p.lse[(long long)it.head * p.T + it.tok_begin + pos] = lse;
@@ -568,20 +627,20 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                                         lse, c2);
                     } else if (KIND == kSweep2) {
                         const float own = (acc0 + acc1) + (acc2 + acc3);
-                        float a = (wg == 0) ? own : cb[0][0][row];
+                        float a = (part == 0) ? own : cb[0][0][row];
 #pragma unroll
-                        for (int g = 1; g < kGroups; ++g) a += (g == wg) ? own : cb[g][0][row];
+                        for (int g = 1; g < kParts; ++g) a += (g == part) ? own : cb[g][0][row];
                         p.scores[(long long)it.head * p.T + it.tok_begin + pos] = a;
                     } else {
                         const long long gi = (long long)it.head * p.T + it.tok_begin + pos;
                         const int e = p.rank[gi];
                         if (e >= 0) {
-                            float bb = (wg == 0) ? best : cb[0][0][row];
-                            int bs = (wg == 0) ? best_slot : __float_as_int(cb[0][1][row]);
+                            float bb = (part == 0) ? best : cb[0][0][row];
+                            int bs = (part == 0) ? best_slot : __float_as_int(cb[0][kP1][row]);
 #pragma unroll
-                            for (int g = 1; g < kGroups; ++g) {
-                                const float b1 = (g == wg) ? best : cb[g][0][row];
-                                const int s1 = (g == wg) ? best_slot : __float_as_int(cb[g][1][row]);
+                            for (int g = 1; g < kParts; ++g) {
+                                const float b1 = (g == part) ? best : cb[g][0][row];
+                                const int s1 = (g == part) ? best_slot : __float_as_int(cb[g][kP1][row]);
                                 if (b1 > bb || (b1 == bb && s1 < bs)) { bb = b1; bs = s1; }
                             }
                             p.assign[it.ev0 + e] = bs;
@@ -635,24 +694,25 @@ cudaError_t launch_tile_kernel(int kind, const CUtensorMap& map_a, const CUtenso
                                const CUtensorMap* map_x, const TileParams& p, int num_sms,
                                cudaStream_t stream) {
     if (p.n_items <= 0) return cudaSuccess;
-    const int smem = (int)sizeof(Shared) + 1024;
+    const int smem_of[3] = {(int)sizeof(Shared<kSweep1>) + 1024, (int)sizeof(Shared<kSweep2>) + 1024,
+                            (int)sizeof(Shared<kMatch>) + 1024};
     const int grid = p.n_items < num_sms ? p.n_items : num_sms;
     const CUtensorMap& mx = map_x ? *map_x : map_b;      // only sweep 2 uses it
     static unsigned long long configured = 0;
     cudaError_t err = once_per_device(configured, [&]() {
-        cudaError_t e = cudaFuncSetAttribute(tile_kernel<kSweep1>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        cudaError_t e = cudaFuncSetAttribute(tile_kernel<kSweep1>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_of[kSweep1]);
         if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(tile_kernel<kSweep2>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+            e = cudaFuncSetAttribute(tile_kernel<kSweep2>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_of[kSweep2]);
         if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(tile_kernel<kMatch>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+            e = cudaFuncSetAttribute(tile_kernel<kMatch>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_of[kMatch]);
         return e;
     });
     if (err != cudaSuccess) return err;
     if (kind == kSweep1)
-        return launch_chained(tile_kernel<kSweep1>, dim3(grid), dim3(kThreads), (size_t)smem, stream, map_a, map_b, mx, p);
+        return launch_chained(tile_kernel<kSweep1>, dim3(grid), dim3(kThreads), (size_t)smem_of[kSweep1], stream, map_a, map_b, mx, p);
     if (kind == kSweep2)
-        return launch_chained(tile_kernel<kSweep2>, dim3(grid), dim3(kThreads), (size_t)smem, stream, map_a, map_b, mx, p);
-    return launch_chained(tile_kernel<kMatch>, dim3(grid), dim3(kThreads), (size_t)smem, stream, map_a, map_b, mx, p);
+        return launch_chained(tile_kernel<kSweep2>, dim3(grid), dim3(kThreads), (size_t)smem_of[kSweep2], stream, map_a, map_b, mx, p);
+    return launch_chained(tile_kernel<kMatch>, dim3(grid), dim3(kThreads), (size_t)smem_of[kMatch], stream, map_a, map_b, mx, p);
 }
 
 cudaError_t launch_lse_split(const float* lse, int n_q_heads, long long T, float scale_log2,
