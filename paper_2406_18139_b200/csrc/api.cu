@@ -122,7 +122,8 @@ int build_plan(Plan& pl, const lookm_layout* lay, int n_req, const int* cu_seqle
         units += (long long)pl.n_kv_heads * n_units;
         it0 += (long long)q.nblk * pl.n_q_heads;
         it1 += (long long)q.nblk * pl.n_kv_heads;
-        it2 += (q.E > 0 && merges) ? (long long)q.nblk * pl.n_kv_heads : 0;
+        // match items: blocks of 128 entries of every head's evicted list
+        it2 += (q.E > 0 && merges) ? (long long)((q.E + kTile - 1) / kTile) * pl.n_kv_heads : 0;
         slots += (long long)q.B * pl.n_kv_heads;
     }
     pl.total_units = units;
@@ -331,7 +332,7 @@ int run_score(const Plan& pl, const DeviceInfo& di, const lookm_layout* lay, con
 
 // norms_done: 1 / |k| of every key row is already in the workspace (written by the selection launch)
 int run_match(const Plan& pl, const DeviceInfo& di, const lookm_layout* lay, const void* k,
-              const int* kept_idx, const int* rank, int* assign, float* sim, void* ws,
+              const int* kept_idx, const int* evict_idx, int* assign, float* sim, void* ws,
               bool norms_done, cudaStream_t st) {
     if (pl.n_items[kMatch] == 0) { mark_stage(4, st); mark_stage(5, st); return LOOKM_OK; }
     float* rnorm_all = at<float>(ws, pl.o_rnorm_all);
@@ -348,17 +349,19 @@ int run_match(const Plan& pl, const DeviceInfo& di, const lookm_layout* lay, con
                                   kept_keys, rnorm_kept, at<int>(ws, pl.o_status), st));
     ++g_launches;
     mark_stage(4, st);
-    CUtensorMap map_k, map_c;
-    LOOKM_TRY(make_map_3d(&map_k, k, pl.T, pl.n_kv_heads, lay->kv_stride_tok, lay->kv_stride_head));
+    CUtensorMap map_c;                           // the evicted rows are gathered, not tiled
     LOOKM_TRY(make_map_2d(&map_c, kept_keys, pl.total_slots));
     TileParams p = tile_params(pl, ws, lay);
     p.n_items = pl.n_items[kMatch];
-    p.rank = rank;
+    p.evict_idx = evict_idx;
+    p.k_rows = k;
+    p.k_stride_tok = lay->kv_stride_tok;
+    p.k_stride_head = lay->kv_stride_head;
     p.rnorm_all = rnorm_all;
     p.rnorm_kept = rnorm_kept;
     p.assign = assign;
     p.sim = sim;
-    LOOKM_CUDA(launch_tile_kernel(kMatch, map_k, map_c, nullptr, p, di.sms, st));
+    LOOKM_CUDA(launch_tile_kernel(kMatch, map_c, map_c, nullptr, p, di.sms, st));
     ++g_launches;
     mark_stage(5, st);
     return LOOKM_OK;
@@ -475,7 +478,7 @@ int compress_common(const void* q, const void* k, const void* v, const uint8_t* 
                              di.sms, st));
     ++g_launches;
     mark_stage(3, st);
-    LOOKM_TRY(run_match(pl, di, lay, k, kept, rank, assign, sim, ws, true, st));
+    LOOKM_TRY(run_match(pl, di, lay, k, kept, evict, assign, sim, ws, true, st));
     LOOKM_TRY(run_merge(pl, lay, k, v, kept, evict, assign, sim, varlen_output, out_k, out_v, ws, st));
     return LOOKM_OK;
 }
@@ -612,13 +615,7 @@ int lookm_match(const void* k, const int* kept_idx, const int* evict_idx, const 
     LOOKM_TRY(device_info(di));
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     LOOKM_TRY(begin_call(pl, workspace, st));
-    int* rank = at<int>(workspace, pl.o_rank);
-    LOOKM_CUDA(cudaMemsetAsync(rank, 0xFF, sizeof(int) * (size_t)pl.n_kv_heads * (size_t)pl.T, st));
-    LOOKM_CUDA(launch_rank_from_lists(at<Req>(workspace, pl.o_reqs), pl.n_req, pl.n_kv_heads, pl.T,
-                                      pl.max_L, kept_idx, evict_idx, rank,
-                                      at<int>(workspace, pl.o_status), st));
-    ++g_launches;
-    return run_match(pl, di, layout, k, kept_idx, rank, assign, sim, workspace, false, st);
+    return run_match(pl, di, layout, k, kept_idx, evict_idx, assign, sim, workspace, false, st);
 }
 
 int lookm_match_from_sim(const float* sim_matrix, const int* cu_seqlens_host, int n_requests,

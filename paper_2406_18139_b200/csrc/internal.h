@@ -67,7 +67,9 @@ struct TileParams {
     unsigned short* lse_split;   // [T, n_q_heads, 16] bf16: -lse / scale as three bf16 terms and 13
                                  // zeros per query row (sweep 1 writes, sweep 2 loads it by TMA)
     float* scores;               // [n_kv_heads, T]
-    const int* rank;             // [n_kv_heads, T]      (match)
+    const int* evict_idx;        // evicted-list layout  (match: rows of the stationary tiles)
+    const void* k_rows;          // K [tokens, heads, 128] bf16 with the strides below (match)
+    long long k_stride_tok, k_stride_head;
     const float* rnorm_all;      // [n_kv_heads, T]      (match)
     const float* rnorm_kept;     // kept-list layout     (match)
     int* assign;                 // evicted-list layout  (match)
@@ -105,10 +107,6 @@ cudaError_t launch_gather_kept(const void* k, long long stride_tok, long long st
 
 cudaError_t launch_argmax_rows(const float* sim_matrix, const Req* reqs, int n_req, int n_kv_heads,
                                int max_evicted, int* assign, float* sim, cudaStream_t stream);
-
-cudaError_t launch_rank_from_lists(const Req* reqs, int n_req, int n_kv_heads, long long T,
-                                   int max_len, const int* kept_idx, const int* evict_idx,
-                                   int* rank, int* status, cudaStream_t stream);
 
 // Copies up to kReqChunk table entries, passed by value as a kernel argument, into the workspace;
 // this keeps the host free of any synchronising copy.

@@ -684,38 +684,12 @@ merge_kernel(const __nv_bfloat16* __restrict__ k, const __nv_bfloat16* __restric
     (void)status;
 }
 
-// Inverse map of given kept / evicted lists (used when the lists come from the caller).
-__global__ void __launch_bounds__(256)
-rank_from_lists_kernel(const Req* __restrict__ reqs, int n_kv_heads, long long T,
-                       const int* __restrict__ kept_idx, const int* __restrict__ evict_idx,
-                       int* __restrict__ rank, int* status) {
-    const Req rq = reqs[blockIdx.z];
-    const int h = blockIdx.y;
-    const int i = blockIdx.x * 256 + threadIdx.x;
-    if (i >= rq.L) return;
-    int pos, val;
-    if (i < rq.B) { pos = kept_idx[rq.kept_off + (long long)h * rq.B + i]; val = -1 - i; }
-    else { pos = evict_idx[rq.ev_off + (long long)h * rq.E + (i - rq.B)]; val = i - rq.B; }
-    if (pos < 0 || pos >= rq.L) { atomicExch(status, (int)LOOKM_ERR_DEVICE_BAD_INDEX); return; }
-    rank[(long long)h * T + rq.tok_begin + pos] = val;
-}
-
 __global__ void write_table_kernel(const __grid_constant__ ReqChunk chunk, int count, Req* dst) {
     const int i = threadIdx.x;
     if (i < count) dst[i] = chunk.r[i];
 }
 
 }  // namespace
-
-cudaError_t launch_rank_from_lists(const Req* reqs, int n_req, int n_kv_heads, long long T,
-                                   int max_len, const int* kept_idx, const int* evict_idx,
-                                   int* rank, int* status, cudaStream_t stream) {
-    if (max_len <= 0) return cudaSuccess;
-    dim3 grid((max_len + 255) / 256, n_kv_heads, n_req);
-    rank_from_lists_kernel<<<grid, 256, 0, stream>>>(reqs, n_kv_heads, T, kept_idx, evict_idx, rank,
-                                                     status);
-    return cudaGetLastError();
-}
 
 cudaError_t launch_write_table(const ReqChunk& chunk, int count, Req* dst, cudaStream_t stream) {
     write_table_kernel<<<1, 64, 0, stream>>>(chunk, count, dst);

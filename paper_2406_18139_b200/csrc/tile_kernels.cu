@@ -22,8 +22,10 @@
 //            three bf16 terms in a 16-column companion of the query tensor, and a ninth MMA per
 //            tile multiplies it with a constant tile of ones, so the accumulator already holds
 //            s_ij - lse_i / scale and the epilogue needs no per-column data at all.
-//   match  : A = 128 key rows (all positions; kept rows are ignored at the end), B = tiles of the
-//            compacted kept keys.  Thread keeps the largest s_ij / |k_j| and its slot.
+//   match  : A = 128 EVICTED key rows in the order of the evicted list, gathered by a warp of its
+//            own with 16-byte cp.async copies into the 128-byte-swizzled layout the tensor core
+//            expects; B = tiles of the compacted kept keys.  Thread keeps the largest
+//            s_ij / |k_j| and its slot.
 //
 // Work items are laid out heaviest first and dealt to the CTAs in serpentine order; every role
 // walks the same item sequence on its own, so no scheduling state is shared.
@@ -71,7 +73,9 @@ constexpr bool kPipeLoads = LOOKM_TILE_PIPE;     // sweeps: the next 32 columns 
                                                  // while the current ones are worked on
 constexpr int kIssuers = 2;                      // MMA-issuing threads (tiles alternate between them)
 constexpr int kEpiWarp0 = 2;                     // first epilogue warp
-constexpr int kThreads = 64 + kParts * 128 + 32; // producer warp, MMA warp, kParts x 4 epilogue warps, second MMA warp
+constexpr int kGatherWarp = kEpiWarp0 + kParts * 4 + 1;    // match: gathers the evicted rows of the A tiles
+// producer warp, MMA warp, kParts x 4 epilogue warps, second MMA warp (+ the gather warp of the match)
+__host__ __device__ constexpr int threads_of(int kind) { return 64 + kParts * 128 + 32 + (kind == kMatch ? 32 : 0); }
 constexpr int kHalfBytes = kTile * 64 * 2;       // one TMA box: 128 rows x 64 bf16 (128 B rows)
 constexpr int kTileBytes = 2 * kHalfBytes;       // 128 x 128 bf16
 constexpr int kSplitBytes = kTile * 16 * 2;      // 128 rows x 16 bf16 (32-byte rows, 32-byte swizzle)
@@ -138,7 +142,7 @@ __global__ void lse_split_kernel(const float* __restrict__ lse, int n_q_heads, l
 }
 
 struct Item {
-    int tok_begin, L, B, blk, head, nt;
+    int tok_begin, L, B, E, blk, head, nt;
     long long kept_row0;      // match: first row of this (request, head) in the kept-key matrix
     long long ev0;            // match: start of its evicted list
 };
@@ -156,6 +160,7 @@ __device__ __forceinline__ Item decode_item(const TileParams& p, const Req* tbl,
     it.tok_begin = rq.tok_begin;
     it.L = rq.L;
     it.B = rq.B;
+    it.E = rq.E;
     it.kept_row0 = 0;
     it.ev0 = 0;
     if (KIND == kSweep1) {                       // heaviest first: last query block first
@@ -166,7 +171,7 @@ __device__ __forceinline__ Item decode_item(const TileParams& p, const Req* tbl,
         it.blk = u / p.n_kv_heads;
         it.head = u % p.n_kv_heads;
         it.nt = (rq.nblk - it.blk) * p.group;
-    } else {
+    } else {                                     // blk: block of 128 entries of the evicted list
         it.blk = u / p.n_kv_heads;
         it.head = u % p.n_kv_heads;
         it.nt = (rq.B + kTile - 1) / kTile;
@@ -183,7 +188,7 @@ __device__ __forceinline__ int item_of_round(int round, int cta, int n_cta) {
 }
 
 template <int KIND>
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(threads_of(KIND), 1)
 tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
             const __grid_constant__ CUtensorMap map_x, const TileParams p) {
     extern __shared__ uint8_t smem_raw[];
@@ -228,7 +233,7 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     grid_dependency_wait();
     const Req* tbl = p.reqs;
     if (p.n_req <= kReqCache) {                  // the table is read once per item by every role
-        for (int i = threadIdx.x; i < p.n_req * (int)(sizeof(Req) / 4); i += kThreads)
+        for (int i = threadIdx.x; i < p.n_req * (int)(sizeof(Req) / 4); i += threads_of(KIND))
             reinterpret_cast<int*>(sh.reqs)[i] = reinterpret_cast<const int*>(p.reqs)[i];
         tbl = sh.reqs;
     }
@@ -256,14 +261,16 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                 if (item >= p.n_items) { if (round * n_cta >= p.n_items) break; --n; continue; }
                 const Item it = decode_item<KIND>(p, tbl, item);
                 const int ab = n % kABuf;
-                if (!ptx::mbar_wait(ptx::smem_u32(&sh.a_empty[ab]), ((n / kABuf) & 1) ^ 1, abort_flag)) break;
-                const uint32_t abar = ptx::smem_u32(&sh.a_full[ab]);
-                ptx::mbar_arrive_expect_tx(abar, kTileBytes);
-                const uint32_t adst = ptx::smem_u32(&sh.a[ab][0]);
-                const int a_head = it.head;
-                const int a_row = it.tok_begin + it.blk * kTile;
-                ptx::tma_load_3d(adst, &map_a, 0, a_head, a_row, abar);
-                ptx::tma_load_3d(adst + kHalfBytes, &map_a, 64, a_head, a_row, abar);
+                if (KIND != kMatch) {                    // the match's stationary tiles come from the gather warp
+                    if (!ptx::mbar_wait(ptx::smem_u32(&sh.a_empty[ab]), ((n / kABuf) & 1) ^ 1, abort_flag)) break;
+                    const uint32_t abar = ptx::smem_u32(&sh.a_full[ab]);
+                    ptx::mbar_arrive_expect_tx(abar, kTileBytes);
+                    const uint32_t adst = ptx::smem_u32(&sh.a[ab][0]);
+                    const int a_head = it.head;
+                    const int a_row = it.tok_begin + it.blk * kTile;
+                    ptx::tma_load_3d(adst, &map_a, 0, a_head, a_row, abar);
+                    ptx::tma_load_3d(adst + kHalfBytes, &map_a, 64, a_head, a_row, abar);
+                }
                 for (int t = 0; t < it.nt; ++t, ++gb) {
                     const int s = gb % kStages;
                     if (!ptx::mbar_wait(ptx::smem_u32(&sh.b_empty[s]), ((gb / kStages) & 1) ^ 1, abort_flag)) {
@@ -302,9 +309,53 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                 for (uint32_t g = (gb > (uint32_t)kStages ? gb - kStages : 0); g < gb; ++g)
                     ptx::mbar_wait(ptx::smem_u32(&sh.b_full[g % kStages]), (g / kStages) & 1, &ignore,
                                    200000000ull);
-                for (int m = (n > kABuf ? n - kABuf : 0); m < n; ++m)
-                    ptx::mbar_wait(ptx::smem_u32(&sh.a_full[m % kABuf]), (m / kABuf) & 1, &ignore, 200000000ull);
+                if (KIND != kMatch)
+                    for (int m = (n > kABuf ? n - kABuf : 0); m < n; ++m)
+                        ptx::mbar_wait(ptx::smem_u32(&sh.a_full[m % kABuf]), (m / kABuf) & 1, &ignore, 200000000ull);
             }
+        }
+    } else if (KIND == kMatch && warp == kGatherWarp) {
+        // ------------------------------------------------------------ gather warp (match) ---
+        // Stationary tile of an item: rows e0 .. e0 + 127 of the head's evicted list, i.e. the key
+        // rows at positions evict_idx[e].  Lane l copies 16-byte chunk (l mod 16) of two rows per
+        // step (half a warp per 256-byte row), 64 steps per tile, into the layout a TMA box pair
+        // with the 128-byte swizzle would have produced: 64 features (128 bytes) per row and box,
+        // chunk c of row r at r * 128 + ((c xor (r mod 8)) * 16).  Rows past the end of the list are
+        // zero-filled.  The copies are waited for and published to the tensor core's proxy before
+        // the tile is announced, one item ahead of the MMAs.
+        const int l16 = lane & 15;
+        const int box = l16 >> 3, c8 = l16 & 7;
+        int n = 0;
+        for (int round = 0;; ++round, ++n) {
+            const int item = item_of_round(round, blockIdx.x, n_cta);
+            if (item >= p.n_items) { if (round * n_cta >= p.n_items) break; --n; continue; }
+            const Item it = decode_item<KIND>(p, tbl, item);
+            const int ab = n % kABuf;
+            int free_now = 1;                            // one lane waits, the warp follows its verdict
+            if (lane == 0)
+                free_now = ptx::mbar_wait(ptx::smem_u32(&sh.a_empty[ab]), ((n / kABuf) & 1) ^ 1, abort_flag) ? 1 : 0;
+            if (!__shfl_sync(0xffffffffu, free_now, 0)) break;
+            const uint32_t adst = ptx::smem_u32(&sh.a[ab][0]) + box * kHalfBytes;
+            const int* ev = p.evict_idx + it.ev0 + it.blk * kTile;
+            const int n_rows = min(kTile, it.E - it.blk * kTile);
+            const char* src0 = reinterpret_cast<const char*>(p.k_rows) +
+                               2 * ((long long)it.tok_begin * p.k_stride_tok + (long long)it.head * p.k_stride_head) + l16 * 16;
+#pragma unroll 8
+            for (int st = 0; st < kTile / 2; ++st) {
+                const int r = 2 * st + (lane >> 4);
+                const bool valid = r < n_rows;
+                int pos = valid ? __ldg(ev + r) : 0;
+                if (pos < 0 || pos >= it.L) { atomicExch(p.status, (int)LOOKM_ERR_DEVICE_BAD_INDEX); pos = 0; }
+                const char* src = src0 + 2 * (long long)pos * p.k_stride_tok;
+                const uint32_t dst = adst + r * 128 + ((c8 ^ (r & 7)) << 4);
+                const int nbytes = valid ? 16 : 0;
+                asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(nbytes) : "memory");
+            }
+            asm volatile("cp.async.commit_group;" ::: "memory");
+            asm volatile("cp.async.wait_group 0;" ::: "memory");
+            ptx::fence_proxy_async_shared();
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&sh.a_full[ab]));
         }
     } else if (warp == 1 || warp == kEpiWarp0 + kParts * 4) {
         // ------------------------------------------------------------ MMA issuers -----------
@@ -383,7 +434,8 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
             const int item = item_of_round(round, blockIdx.x, n_cta);
             if (item >= p.n_items) { if (round * n_cta >= p.n_items) break; --n; continue; }
             const Item it = decode_item<KIND>(p, tbl, item);
-            const int pos = it.blk * kTile + row;            // position of this thread's row
+            const int pos = it.blk * kTile + row;            // position of this thread's row (match: its
+                                                             // index in the evicted list)
             float m_run = -INFINITY, l_run = 0.f;            // sweep 1
             float acc0 = 0.f, acc1 = 0.f, acc2 = 0.f, acc3 = 0.f;   // sweep 2
             float best = -INFINITY;                          // match
@@ -606,7 +658,7 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                 if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&sh.comb_full[cslot]));
             } else {
                 ptx::mbar_wait(ptx::smem_u32(&sh.comb_full[cslot]), cuse & 1u, abort_flag);
-                if (pos < it.L && !*abort_flag) {
+                if (pos < (KIND == kMatch ? it.E : it.L) && !*abort_flag) {
                     if (KIND == kSweep1) {
                         float mg[kParts], lg[kParts];
 #pragma unroll
@@ -632,9 +684,11 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                         for (int g = 1; g < kParts; ++g) a += (g == part) ? own : cb[g][0][row];
                         p.scores[(long long)it.head * p.T + it.tok_begin + pos] = a;
                     } else {
-                        const long long gi = (long long)it.head * p.T + it.tok_begin + pos;
-                        const int e = p.rank[gi];
-                        if (e >= 0) {
+                        int at = p.evict_idx[it.ev0 + pos];      // position of this evicted row
+                        if (at < 0 || at >= it.L) at = 0;       // reported by the gather warp
+                        const long long gi = (long long)it.head * p.T + it.tok_begin + at;
+                        const int e = pos;
+                        {
                             float bb = (part == 0) ? best : cb[0][0][row];
                             int bs = (part == 0) ? best_slot : __float_as_int(cb[0][kP1][row]);
 #pragma unroll
@@ -709,10 +763,10 @@ cudaError_t launch_tile_kernel(int kind, const CUtensorMap& map_a, const CUtenso
     });
     if (err != cudaSuccess) return err;
     if (kind == kSweep1)
-        return launch_chained(tile_kernel<kSweep1>, dim3(grid), dim3(kThreads), (size_t)smem_of[kSweep1], stream, map_a, map_b, mx, p);
+        return launch_chained(tile_kernel<kSweep1>, dim3(grid), dim3(threads_of(kSweep1)), (size_t)smem_of[kSweep1], stream, map_a, map_b, mx, p);
     if (kind == kSweep2)
-        return launch_chained(tile_kernel<kSweep2>, dim3(grid), dim3(kThreads), (size_t)smem_of[kSweep2], stream, map_a, map_b, mx, p);
-    return launch_chained(tile_kernel<kMatch>, dim3(grid), dim3(kThreads), (size_t)smem_of[kMatch], stream, map_a, map_b, mx, p);
+        return launch_chained(tile_kernel<kSweep2>, dim3(grid), dim3(threads_of(kSweep2)), (size_t)smem_of[kSweep2], stream, map_a, map_b, mx, p);
+    return launch_chained(tile_kernel<kMatch>, dim3(grid), dim3(threads_of(kMatch)), (size_t)smem_of[kMatch], stream, map_a, map_b, mx, p);
 }
 
 cudaError_t launch_lse_split(const float* lse, int n_q_heads, long long T, float scale_log2,
