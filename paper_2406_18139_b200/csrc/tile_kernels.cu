@@ -50,9 +50,6 @@ constexpr int kABuf = LOOKM_TILE_ABUF;           // buffers of the stationary ti
 #ifndef LOOKM_TILE_GROUPS
 #define LOOKM_TILE_GROUPS 4
 #endif
-#ifndef LOOKM_TILE_PIPE
-#define LOOKM_TILE_PIPE 0
-#endif
 constexpr int kAccum = 4;                        // TMEM accumulators (128 fp32 columns each)
 #ifndef LOOKM_TILE_HALVES
 #define LOOKM_TILE_HALVES 1
@@ -69,8 +66,6 @@ constexpr int kCols = kTile / kHalves;           // accumulator columns per part
 // back is g - 2 kAccum, whose MMAs had to complete before the producer could load tile g - kAccum,
 // which it did before it loaded any tile this group has already finished.
 constexpr int kFullRing = 2 * kAccum;
-constexpr bool kPipeLoads = LOOKM_TILE_PIPE;     // sweeps: the next 32 columns are on their way from TMEM
-                                                 // while the current ones are worked on
 constexpr int kIssuers = 2;                      // MMA-issuing threads (tiles alternate between them)
 constexpr int kEpiWarp0 = 2;                     // first epilogue warp
 constexpr int kGatherWarp = kEpiWarp0 + kParts * 4 + 1;    // match: gathers the evicted rows of the A tiles
@@ -614,28 +609,13 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                     if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&sh.t_empty[buf]));
                 };
                 const uint32_t tbase = lane_addr + buf * kTile + col0;
-                if (kPipeLoads) {
-                    uint32_t ra[32], rb[32];
-                    ptx::tmem_ld_32x32(tbase, ra);
 #pragma unroll 1
-                    for (int hf = 0; hf < kCols / 64; ++hf) {
-                        ptx::tmem_ld_wait32(ra);
-                        ptx::tmem_ld_32x32(tbase + (2 * hf + 1) * 32, rb, ra);
-                        process(ra, col0 + 2 * hf * 32);
-                        ptx::tmem_ld_wait32(rb);
-                        if (hf < kCols / 64 - 1) ptx::tmem_ld_32x32(tbase + (2 * hf + 2) * 32, ra, rb);
-                        else release();
-                        process(rb, col0 + (2 * hf + 1) * 32);
-                    }
-                } else {
-#pragma unroll 1
-                    for (int ch = 0; ch < kCols / 32; ++ch) {
-                        uint32_t raw[32];
-                        ptx::tmem_ld_32x32(tbase + ch * 32, raw);
-                        ptx::tmem_ld_wait();
-                        if (ch == kCols / 32 - 1) release();
-                        process(raw, col0 + ch * 32);
-                    }
+                for (int ch = 0; ch < kCols / 32; ++ch) {
+                    uint32_t raw[32];
+                    ptx::tmem_ld_32x32(tbase + ch * 32, raw);
+                    ptx::tmem_ld_wait();
+                    if (ch == kCols / 32 - 1) release();
+                    process(raw, col0 + ch * 32);
                 }
             }
 
