@@ -264,7 +264,11 @@ int lookm_workspace_layout(const lookm_layout* layout, int n_requests, const int
  * The call performs no cudaMalloc/cudaFree and calls no allocating routine.
  *
  * The first call on each device looks up the array's device address (cudaGetSymbolAddress, with
- * that device current) and caches it; make that first call outside any stream capture.
+ * that device current) and caches it.  With lazy module loading that look-up can make the driver
+ * load this library's device image, the 16 MiB array included, at that moment: make the first
+ * call (a tiny warm-up batch will do) at start-up, outside any stream capture and off the serving
+ * path.  The cached address belongs to the device's primary context and is stale once that context
+ * has been reset.
  *
  * All calls on a device share the one array, and it keeps what the previous call left in it.
  * Each call clears the status word and rewrites everything it later reads, so back-to-back calls
