@@ -265,6 +265,78 @@ def test_match_duplicate_kept_keys_take_the_lower_slot(B):
     assert np.allclose(sim.cpu().numpy()[150:180], 1.0, atol=1e-6)
 
 
+@pytest.mark.parametrize("L,budget", [(384, 128), (300, 44), (200, 199), (131, 3)])
+def test_match_whole_blocks_single_rows_and_strided_keys(B, L, budget):
+    """The evicted rows are gathered 128 at a time: lists of exactly 128 and 256 rows, of one row, and
+    of 128 rows against 3 kept keys; the keys sit in a fused [L, 3 * H, 128] buffer (strided heads)."""
+    import torch
+    Hkv = 2
+    w = synth.tiny(L, Hkv, Hkv, budget, 0, 0, image_spans=[(5, L // 2)], seed=L + budget)
+    (q, k, v), (qf, kf, vf), mask, _ = _tensors(w)
+    fused = torch.stack([q, k, v], dim=1).reshape(L, 3 * Hkv, 128).contiguous()
+    fk = fused[:, Hkv:2 * Hkv]
+    s = np.abs(synth.normal(synth.stream_key(92, L), Hkv * L)).reshape(Hkv, L) + 1e-3
+    lists = [orc.select(s[h], mask, budget, 0) for h in range(Hkv)]
+    kept = torch.from_numpy(np.concatenate([a for a, _ in lists])).cuda()
+    ev = torch.from_numpy(np.concatenate([b for _, b in lists])).cuda()
+    E = L - budget
+    assign = torch.full((Hkv * E,), -7, dtype=torch.int32, device="cuda")
+    sim = torch.full((Hkv * E,), -7.0, dtype=torch.float32, device="cuda")
+    lay = B.make_layout(None, fk)
+    ws = B.alloc_workspace(lay, [L])
+    B.check(B.lookm_match(fk, kept, ev, [0, L], [budget], lay, assign, sim, ws))
+    assert B.lookm_device_status(ws) == B.OK
+    a_got = assign.cpu().numpy().reshape(Hkv, E)
+    s_got = sim.cpu().numpy().reshape(Hkv, E).astype(np.float64)
+    for h in range(Hkv):
+        a_ref, s_ref, S = orc.match(kf, h, lists[h][0], lists[h][1], want_matrix=True)
+        assert np.allclose(s_got[h], s_ref, atol=2e-6, rtol=0)
+        for e in np.where(a_got[h] != a_ref)[0]:
+            assert S[e, a_ref[e]] - S[e, a_got[h, e]] <= 1e-4
+
+
+def test_match_packed_batch_and_out_of_range_evicted_position(B):
+    import torch
+    Hkv = 2
+    lens, budgets = [150, 400, 129], [30, 100, 1]
+    w = synth.Workload("batch", 0, 77, 1, Hkv, Hkv, 128, False,
+                       [synth.tiny(n, Hkv, Hkv, b, 0, 0, seed=300 + n).requests[0] for n, b in zip(lens, budgets)])
+    qb, kb, vb, mask = synth.packed_layer_tensors(w, 0)
+    k, kf = to_dev(kb), synth.bf16_to_f32(kb)
+    cu = np.concatenate([[0], np.cumsum(lens)]).tolist()
+    kept_l, ev_l = [], []
+    for r, (n, b) in enumerate(zip(lens, budgets)):
+        for h in range(Hkv):
+            sc = np.abs(synth.normal(synth.stream_key(93, r, h), n)) + 1e-3
+            a, e = orc.select(sc, mask[cu[r]:cu[r + 1]], b, 0)
+            kept_l.append(a)
+            ev_l.append(e)
+    kept = torch.from_numpy(np.concatenate(kept_l)).cuda()
+    ev = torch.from_numpy(np.concatenate(ev_l)).cuda()
+    n_ev = sum(Hkv * (n - b) for n, b in zip(lens, budgets))
+    assign = torch.zeros(n_ev, dtype=torch.int32, device="cuda")
+    sim = torch.zeros(n_ev, dtype=torch.float32, device="cuda")
+    lay = B.make_layout(None, k)
+    ws = B.alloc_workspace(lay, lens)
+    B.check(B.lookm_match(k, kept, ev, cu, budgets, lay, assign, sim, ws))
+    assert B.lookm_device_status(ws) == B.OK
+    a_got, s_got = assign.cpu().numpy(), sim.cpu().numpy().astype(np.float64)
+    at = 0
+    for r, (n, b) in enumerate(zip(lens, budgets)):
+        for h in range(Hkv):
+            E = n - b
+            a_ref, s_ref, S = orc.match(kf[cu[r]:cu[r + 1]], h, kept_l[r * Hkv + h], ev_l[r * Hkv + h], want_matrix=True)
+            assert np.allclose(s_got[at:at + E], s_ref, atol=2e-6, rtol=0)
+            for e in np.where(a_got[at:at + E] != a_ref)[0]:
+                assert S[e, a_ref[e]] - S[e, a_got[at + e]] <= 1e-4
+            at += E
+    # a position beyond the request is reported through the status word, never dereferenced
+    ev[5] = 100000
+    B.check(B.lookm_match(k, kept, ev, cu, budgets, lay, assign, sim, ws))
+    assert B.lookm_device_status(ws) == B.ERR_DEVICE_BAD_INDEX
+    assert B.lookm_device_status(ws) == B.OK
+
+
 # ------------------------------------------------------------------------------ merging ------
 
 @pytest.mark.parametrize("mode", [0, 1, 2])
