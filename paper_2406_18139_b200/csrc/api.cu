@@ -102,13 +102,21 @@ int build_plan(Plan& pl, const lookm_layout* lay, int n_req, const int* cu_seqle
     // table order: longest request first
     std::stable_sort(pl.reqs.begin(), pl.reqs.end(), [](const Req& a, const Req& b) { return a.L > b.L; });
     long long it0 = 0, it1 = 0, it2 = 0, slots = 0, units = 0;
-    // merge work units: about one per warp of the merge kernel (it reads n_kv_heads * T rows)
+    // Merge work units (the kernel reads n_kv_heads * T rows): every warp gets the same number of
+    // units, one if that keeps a unit within kMaxUnitEntries rows.  The units of a request are laid
+    // out heads fastest, so a wave of warps reads one token window of all heads; with very long
+    // units (a batch of many prompts) every warp would stream a far-away window of its own, and a
+    // unit count just above the warp count would leave a second, nearly empty wave.
     int unit_entries = kMinUnitEntries;
     {
         DeviceInfo di;
         const int sms = (device_info(di) == LOOKM_OK && di.sms > 0) ? di.sms : 148;
         const long long per_warp = ((long long)pl.n_kv_heads * pl.T) / ((long long)sms * merge_warps_per_sm());
-        if (per_warp > unit_entries) unit_entries = (int)std::min<long long>((per_warp + 7) / 8 * 8, 1 << 20);
+        if (per_warp > unit_entries) {
+            const long long per_warp_units = (per_warp + kMaxUnitEntries - 1) / kMaxUnitEntries;
+            const long long rows = (per_warp + per_warp_units - 1) / per_warp_units;
+            unit_entries = (int)std::max<long long>(kMinUnitEntries, (rows + 7) / 8 * 8);
+        }
     }
     for (Req& q : pl.reqs) {
         q.item_begin[kSweep1] = (int)it0;

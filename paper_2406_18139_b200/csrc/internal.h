@@ -12,6 +12,10 @@ namespace lookm {
 constexpr int kTile = 128;      // tokens per tile on either operand of the tensor-core kernels
 constexpr int kHeadDim = 128;   // only supported head_dim
 constexpr int kMinUnitEntries = 32; // least number of rows in a work unit of the merge kernel
+#ifndef LOOKM_MAX_UNIT_ENTRIES
+#define LOOKM_MAX_UNIT_ENTRIES 256
+#endif
+constexpr int kMaxUnitEntries = LOOKM_MAX_UNIT_ENTRIES;   // most rows in one
 // Digits of the assignment inversion's radix sort: the slot index of a request with B kept rows is
 // split into the fewest digits of at most max_bits bits, all of the same width (so B <= 2^max_bits
 // is sorted in one pass).  16-bit counters allow 11-bit digits, 32-bit counters 10-bit ones.

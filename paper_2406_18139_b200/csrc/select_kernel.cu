@@ -308,7 +308,9 @@ cudaError_t launch_select(const float* scores, const uint8_t* mask, const Req* r
         // leaves free, so that all of them run at once (a second wave would have to wait for the
         // selection CTAs, which run longest)
         const long long want = (T * n_kv_heads + kSelThreads / 16 - 1) / (kSelThreads / 16);
-        n_norm = (int)std::min<long long>(want, n_select < num_sms ? num_sms - n_select : num_sms);
+        // (with selection CTAs on more than half of the SMs the few SMs left would carry all the
+        // norms: then a full wave of norm CTAs follows the selection CTAs instead)
+        n_norm = (int)std::min<long long>(want, n_select < num_sms / 2 ? num_sms - n_select : num_sms);
     }
     return launch_chained(select_kernel, dim3(n_select + n_norm), dim3(kSelThreads), 0, stream,
                           scores, mask, reqs, n_select, n_kv_heads, T, kept_idx, evict_idx, rank,
