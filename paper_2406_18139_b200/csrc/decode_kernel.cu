@@ -278,8 +278,9 @@ decode_kernel(const __grid_constant__ DecodeBatch batch, const __nv_bfloat16* __
 }
 
 // Several splits: adds the partial results of one (request, KV head, pass, query head) in split
-// order.  One CTA of 128 threads per such unit, thread t owns feature t; the records of eight
-// splits are requested together (the loop is bound by the latency of these loads).  Launched
+// order.  One CTA of 128 threads per such unit, thread t owns feature t; the splits' reference
+// values are fetched in one round trip and the records of sixteen splits are requested together
+// (the kernel is bound by the latency of these loads).  Launched
 // behind decode_kernel with programmatic stream serialisation: no counters, no atomics, nothing in
 // the workspace has to be cleared, and the order of additions is fixed.
 __global__ void __launch_bounds__(kHeadDim)
@@ -295,15 +296,18 @@ decode_combine_kernel(const __grid_constant__ DecodeBatch batch, int gt, int n_p
     const long long part_stride = kHeadDim + 2;
     const float* base = parts + ((long long)rq.part_begin + (long long)unit * n_splits * gt + g) * part_stride;
     const long long step = (long long)gt * part_stride;          // between the records of two splits
-    constexpr int kBatch = 8;
+    // largest reference value over the splits: thread t looks at splits t, t + 128, ...; one round
+    // trip for up to 128 splits, then a block-wide maximum
+    __shared__ float warp_max[kHeadDim / 32];
     float mx = -INFINITY;
-    for (int s0 = 0; s0 < n_splits; s0 += kBatch) {
-        float mv[kBatch];
+    for (int sp = t; sp < n_splits; sp += kHeadDim) mx = fmaxf(mx, __ldcg(base + sp * step));
 #pragma unroll
-        for (int j = 0; j < kBatch; ++j) mv[j] = (s0 + j < n_splits) ? __ldcg(base + (s0 + j) * step) : -INFINITY;
-#pragma unroll
-        for (int j = 0; j < kBatch; ++j) mx = fmaxf(mx, mv[j]);
-    }
+    for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    if ((t & 31) == 0) warp_max[t >> 5] = mx;
+    __syncthreads();
+    mx = fmaxf(fmaxf(warp_max[0], warp_max[1]), fmaxf(warp_max[2], warp_max[3]));
+    // the records in split order, kBatch of them requested together
+    constexpr int kBatch = 16;
     float lsum = 0.f, osum = 0.f;
     for (int s0 = 0; s0 < n_splits; s0 += kBatch) {
         float mv[kBatch], lv[kBatch], ov[kBatch];
