@@ -201,6 +201,19 @@ __device__ __forceinline__ void tmem_ld_wait() {
     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
 
+// Read-only global loads that stay where they are written (the compiler may not sink them to their
+// first use): for values requested long before they are needed.
+__device__ __forceinline__ int ld_nc_s32(const int* p) {
+    int v;
+    asm volatile("ld.global.nc.s32 %0, [%1];" : "=r"(v) : "l"(p));
+    return v;
+}
+__device__ __forceinline__ float ld_nc_f32(const float* p) {
+    float v;
+    asm volatile("ld.global.nc.f32 %0, [%1];" : "=f"(v) : "l"(p));
+    return v;
+}
+
 // max of three in one instruction
 __device__ __forceinline__ float fmax3(float a, float b, float c) {
     float r;

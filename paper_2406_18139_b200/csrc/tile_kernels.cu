@@ -435,6 +435,22 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
             float acc0 = 0.f, acc1 = 0.f, acc2 = 0.f, acc3 = 0.f;   // sweep 2
             float best = -INFINITY;                          // match
             int best_slot = 0x7fffffff;
+            // match: 1 / |k| of this thread's evicted row takes two dependent loads (its position, then
+            // the norm).  They are requested here and after the part's first tile, not in the combine
+            // at the item's end, where the part that combines would sit out both round trips while
+            // its next accumulator stays full.
+            int row_at = 0;
+            float row_rnorm = 0.f;
+            bool rnorm_asked = false;
+            if (KIND == kMatch && pos < it.E) row_at = ptx::ld_nc_s32(p.evict_idx + it.ev0 + pos);
+            auto ask_rnorm = [&]() {
+                if (pos < it.E) {
+                    int at = row_at;
+                    if (at < 0 || at >= it.L) at = 0;       // reported by the gather warp
+                    row_rnorm = ptx::ld_nc_f32(p.rnorm_all + (long long)it.head * p.T + it.tok_begin + at);
+                }
+                rnorm_asked = true;
+            };
 
             for (int t = 0; t < it.nt; ++t, ++gb) {
                 if ((int)(gb % kGroups) != wg) continue;
@@ -518,6 +534,7 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                         }
                         columns16(rb, col0 + (2 * k + 1) * 16);
                     }
+                    if (!rnorm_asked) ask_rnorm();
                     continue;
                 }
                 // work on 32 columns of the accumulator, c0 = first column of the chunk
@@ -664,9 +681,7 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                         for (int g = 1; g < kParts; ++g) a += (g == part) ? own : cb[g][0][row];
                         p.scores[(long long)it.head * p.T + it.tok_begin + pos] = a;
                     } else {
-                        int at = p.evict_idx[it.ev0 + pos];      // position of this evicted row
-                        if (at < 0 || at >= it.L) at = 0;       // reported by the gather warp
-                        const long long gi = (long long)it.head * p.T + it.tok_begin + at;
+                        if (!rnorm_asked) ask_rnorm();           // a part without a tile in this item
                         const int e = pos;
                         {
                             float bb = (part == 0) ? best : cb[0][0][row];
@@ -678,7 +693,7 @@ tile_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                                 if (b1 > bb || (b1 == bb && s1 < bs)) { bb = b1; bs = s1; }
                             }
                             p.assign[it.ev0 + e] = bs;
-                            p.sim[it.ev0 + e] = bb * p.rnorm_all[gi];
+                            p.sim[it.ev0 + e] = bb * row_rnorm;
                         }
                     }
                 }
